@@ -1,0 +1,203 @@
+/* fmmoe.h -- C ABI of the B200 (sm_100a) FastMMoE MoE-layer hot path.
+ *
+ * The library implements, as hand-written CUDA kernels, the two components of
+ * FastMMoE's prefill path:
+ *   - Section 3.1: a mixture-of-experts layer in which vision tokens activate
+ *     K_v <= K routed experts (Eq. 1-5) from a start layer l_v on, and
+ *   - Section 3.2: routing-aware sliding-window pruning of vision tokens
+ *     (Eq. 6-18 and the drop rule stated after Eq. 18).
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise
+ *   - Tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned,
+ *     row-major and contiguous.  Pointers marked (host) are host arrays.
+ *   - Nothing is allocated on the device after fmmoe_create(); scratch memory is
+ *     the caller's `workspace`, sized by the matching *_workspace_bytes() call.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*) and the
+ *     call returns without synchronising, except where stated.
+ *   - Errors are return codes; arguments are validated on the host before any
+ *     launch.  A kernel whose bounded wait expired records FMMOE_ERR_TIMEOUT in
+ *     a device status word that fmmoe_get_status() reads back.
+ *   - There is no CPU or library fallback: unsupported shapes return
+ *     FMMOE_ERR_UNSUPPORTED.
+ *   - Tokens are rows.  is_visual[t] != 0 marks a vision token.  Experts are
+ *     numbered from 0.  All ties go to the lower index.
+ */
+#ifndef FMMOE_H_
+#define FMMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FMMOE_OK = 0,
+  FMMOE_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, negative size, K_v > K ...   */
+  FMMOE_ERR_UNSUPPORTED = 2,   /* shape outside what the kernels implement               */
+  FMMOE_ERR_WORKSPACE = 3,     /* workspace NULL, misaligned or too small                */
+  FMMOE_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                      */
+  FMMOE_ERR_TIMEOUT = 5,       /* a device-side bounded wait expired                     */
+  FMMOE_ERR_INTERNAL = 6
+} fmmoe_status;
+
+typedef enum { FMMOE_F32 = 0, FMMOE_BF16 = 1 } fmmoe_dtype;
+
+/* Limits of the kernels. */
+#define FMMOE_MAX_EXPERTS 256
+#define FMMOE_MAX_TOPK 16
+#define FMMOE_MAX_WINDOW 8
+#define FMMOE_MAX_SEQS_PER_LAUNCH 64
+
+/* flags of fmmoe_route / fmmoe_moe_forward */
+#define FMMOE_FLAG_REDUCE_ON 1u      /* layer index >= l_v: vision tokens use K_v (Section 3.1) */
+#define FMMOE_FLAG_RESIDUAL 2u       /* out = x + MoE(x)                                        */
+#define FMMOE_FLAG_DETERMINISTIC 4u  /* combine by a fixed-order gather instead of atomic adds  */
+
+/* Static shape of one MoE layer (Section 3.1: H, E, S_m, N_s, K, K_v). */
+typedef struct {
+  int32_t hidden;        /* H                                                    */
+  int32_t n_experts;     /* E routed experts, 1..FMMOE_MAX_EXPERTS               */
+  int32_t inter;         /* routed expert intermediate size S_m                  */
+  int32_t n_shared;      /* N_s shared experts (>= 0), always active, gate 1     */
+  int32_t shared_inter;  /* intermediate size of EACH shared expert              */
+  int32_t top_k;         /* K, 1..FMMOE_MAX_TOPK                                 */
+  int32_t top_k_vis;     /* K_v = pK, 0..K; 0 only if n_shared > 0 (Section 3.1) */
+  int32_t dtype;         /* fmmoe_dtype of x, out and all expert/router weights  */
+} fmmoe_layer_desc;
+
+/* Layer parameters (device, read-only).  nn.Linear layout: [out_features, in_features]. */
+typedef struct {
+  const void  *router_w;  /* W_E [E, H] dtype (Eq. 1)                                       */
+  const float *router_b;  /* [E] fp32 added to the logits before the softmax, or NULL       */
+  const void  *w_gate;    /* [E, S_m, H]                                                    */
+  const void  *w_up;      /* [E, S_m, H]                                                    */
+  const void  *w_down;    /* [E, H, S_m]                                                    */
+  const void  *ws_gate;   /* [N_s, S_s, H] or NULL                                          */
+  const void  *ws_up;     /* [N_s, S_s, H] or NULL                                          */
+  const void  *ws_down;   /* [N_s, H, S_s] or NULL                                          */
+} fmmoe_weights;
+
+/* Optional routing outputs (device).  Any pointer may be NULL = not wanted. */
+typedef struct {
+  float   *logits;      /* [T, E] fp32  Z (Eq. 1), as the kernel holds them                      */
+  float   *probs;       /* [T, E] fp32  P = softmax(Z) (Eq. 2); the R_v rows of Eq. 6            */
+  int32_t *topk_idx;    /* [T, K] Q (Eq. 3), descending probability; -1 beyond the token's k     */
+  float   *topk_w;      /* [T, K] g (Eq. 5), 0 beyond the token's k                              */
+  int32_t *expert_off;  /* [E+1] first row of each expert in the expert-grouped order            */
+  int32_t *row_token;   /* [T*K] token of each row (first expert_off[E] entries are valid)       */
+  int32_t *inv_row;     /* [T, K] row of each (token, slot), -1 for padded slots                 */
+} fmmoe_route_out;
+
+typedef struct fmmoe_handle fmmoe_handle;   /* opaque: device, SM count, status word, launch counter */
+
+/* Create a handle on CUDA device `device` (allocates a few hundred bytes of
+ * device memory for the status word).  Not thread-safe per handle. */
+fmmoe_status fmmoe_create(fmmoe_handle **handle, int device);
+fmmoe_status fmmoe_destroy(fmmoe_handle *handle);
+const char  *fmmoe_status_string(fmmoe_status s);
+
+/* Synchronises `cuda_stream`, reads and clears the device status word.
+ * Returns FMMOE_OK, FMMOE_ERR_TIMEOUT (a bounded wait expired in a kernel; its
+ * outputs are invalid) or FMMOE_ERR_CUDA. */
+fmmoe_status fmmoe_get_status(fmmoe_handle *handle, void *cuda_stream);
+
+/* Number of kernels this handle has launched so far (host counter). */
+int64_t fmmoe_launch_count(const fmmoe_handle *handle);
+
+/* Bytes of workspace fmmoe_route / fmmoe_moe_forward need for n_tokens tokens of
+ * this layer with these flags (only FMMOE_FLAG_DETERMINISTIC changes the size).
+ * Host-only, no GPU work.  Returns 0 for an invalid description. */
+size_t fmmoe_workspace_bytes(const fmmoe_layer_desc *desc, int64_t n_tokens, uint32_t flags);
+
+/* Section 3.1, Eq. 1-3 and 5: router logits, softmax, per-token top-k with
+ * k = K_v for vision tokens when FMMOE_FLAG_REDUCE_ON is set (K otherwise),
+ * gates renormalised over the selected set.  The selection is taken on the
+ * fp32 logits (softmax is monotone); equal logits go to the lower expert.
+ * If expert_off / row_token / inv_row are requested, the stable grouping of the
+ * (token, expert) pairs by expert (rows of one expert ascend by token) is
+ * produced too.  x: [T, H] dtype; is_visual: [T] bytes.  n_tokens may be 0. */
+fmmoe_status fmmoe_route(fmmoe_handle *handle, const fmmoe_layer_desc *desc, const fmmoe_weights *w,
+                         const void *x, const uint8_t *is_visual, int64_t n_tokens, uint32_t flags,
+                         const fmmoe_route_out *out, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream);
+
+/* Section 3.1, Eq. 1-5 (whole layer):
+ *   out[t] = sum_s FFN^s(x[t]) + sum_{j in Q_t} g_j FFN^e_j(x[t])   (+ x[t] with FMMOE_FLAG_RESIDUAL)
+ * with SwiGLU experts FFN(x) = W_down (silu(W_gate x) * (W_up x)).  Experts a
+ * token did not select are not evaluated for it.  bf16 layers run the expert
+ * contractions on tcgen05 tensor cores with fp32 accumulation and round the
+ * SwiGLU activations once to bf16; fp32 layers use fp32 FMA throughout.
+ * out: [T, H] dtype, must not alias x.  `route` (may be NULL) receives the
+ * routing record of the call.  bf16 requires H % 64 == 0, S_m % 64 == 0,
+ * S_s % 64 == 0. */
+fmmoe_status fmmoe_moe_forward(fmmoe_handle *handle, const fmmoe_layer_desc *desc, const fmmoe_weights *w,
+                               const void *x, const uint8_t *is_visual, int64_t n_tokens, uint32_t flags,
+                               void *out, const fmmoe_route_out *route, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream);
+
+/* Same layer as fmmoe_moe_forward with the step's activations in HOST memory:
+ * copies x_host [T,H] and is_visual_host [T] to the device, runs the layer, copies
+ * out back to out_host [T,H] and SYNCHRONISES the stream before returning.
+ * Pinned host buffers make the copies asynchronous.  `workspace` must hold
+ * fmmoe_workspace_bytes() + fmmoe_host_staging_bytes() bytes.  Weights stay on the device. */
+size_t fmmoe_host_staging_bytes(const fmmoe_layer_desc *desc, int64_t n_tokens);
+fmmoe_status fmmoe_moe_forward_host(fmmoe_handle *handle, const fmmoe_layer_desc *desc, const fmmoe_weights *w,
+                                    const void *x_host, const uint8_t *is_visual_host, int64_t n_tokens,
+                                    uint32_t flags, void *out_host, void *workspace, size_t workspace_bytes,
+                                    void *cuda_stream);
+
+/* Section 3.2 hyper-parameters. */
+typedef struct {
+  int32_t window;      /* W, 2..FMMOE_MAX_WINDOW                                                  */
+  int32_t sim_mode;    /* 0: mean pairwise cosine (Eq. 8); 1: cosine to the window mean (Eq. 9-10) */
+  int32_t merge_mode;  /* 0: mean rescaled to the largest member norm (Eq. 16-18); 1: plain mean;  */
+                       /* 2: no merging (gamma ignored, windows are only dropped)                  */
+  int32_t reserved;
+  double  alpha;       /* Eq. 13 trade-off, 0..1; ignored when attn == NULL                        */
+  double  gamma;       /* Eq. 14 merge rate, >= 0                                                  */
+} fmmoe_prune_params;
+
+/* Section 3.2.3 budget arithmetic (host only, data-independent): number of
+ * vision tokens left when n_vis tokens are pruned towards n_retain.
+ * eps = n_vis - n_retain; nothing happens unless eps > W; m = floor(n_retain*gamma)
+ * windows are merged (each removes W-1 tokens; m is clamped so no more than eps
+ * tokens go), then floor((eps - m(W-1)) / W) windows are dropped.
+ * Optionally returns m and the dropped-window count.  Returns -1 on invalid arguments. */
+int64_t fmmoe_prune_kept_count(int64_t n_vis, int64_t n_retain, const fmmoe_prune_params *p,
+                               int64_t *n_merge, int64_t *n_drop);
+
+size_t fmmoe_prune_workspace_bytes(int64_t n_tokens, int32_t n_seq);
+
+/* Section 3.2 on n_seq independent sequences laid out back to back:
+ * sequence b is tokens seq_off[b] .. seq_off[b+1]-1 and holds n_vis[b] vision
+ * tokens (must equal the number of set bytes of is_visual in that range; a
+ * mismatch is reported through the status word as FMMOE_ERR_INTERNAL).
+ * Windows of W consecutive vision tokens (in sequence order, wherever text sits)
+ * are scored C = alpha*S - (1-alpha)*A_bar (Eq. 8/10, 11-13) from the routing
+ * probabilities `probs` [T, E] fp32 and the attention importance `attn` [T] fp32
+ * (entries at vision tokens are used, Eq. 7).  With attn == NULL, C = S and the
+ * drop stage takes the most redundant remaining windows.  Scores are
+ * accumulated in fp64 and rounded once to fp32 before ranking.  The m highest-C
+ * windows are merged into one row at their first token's position (Eq. 15-18),
+ * then the d remaining windows with the smallest A_bar are dropped; the
+ * N_v mod W trailing vision tokens and all text tokens are kept.
+ * Outputs (device): x_out [T', H] dtype, is_visual_out [T'], keep_idx [T'] source
+ * token of each output row, kind [T'] (0 text, 1 kept, 2 merged); each may be
+ * NULL except x_out.  out_seq_off (host, [n_seq+1]) is filled before return:
+ * the counts do not depend on the data.  x_out must not alias x. */
+fmmoe_status fmmoe_prune_visual(fmmoe_handle *handle, const fmmoe_prune_params *p,
+                                const float *probs, int32_t n_experts, const float *attn,
+                                const void *x, int32_t dtype, int32_t hidden, const uint8_t *is_visual,
+                                const int64_t *seq_off /* host [n_seq+1] */,
+                                const int64_t *n_vis /* host [n_seq] */,
+                                const int64_t *n_retain /* host [n_seq] */, int32_t n_seq,
+                                void *x_out, uint8_t *is_visual_out, int32_t *keep_idx, uint8_t *kind,
+                                int64_t *out_seq_off /* host [n_seq+1] */,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FMMOE_H_ */

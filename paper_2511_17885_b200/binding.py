@@ -1,0 +1,252 @@
+"""ctypes binding over libfmmoe.so: same names as the C ABI (include/fmmoe.h).
+
+Argument marshalling only: torch supplies device memory, the current stream and
+dtypes; every step of the path runs in the library's CUDA kernels.  There is no
+fallback: a missing library raises ImportError at first use.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libfmmoe.so")
+
+FMMOE_OK = 0
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE", 4: "CUDA", 5: "TIMEOUT", 6: "INTERNAL"}
+F32, BF16 = 0, 1
+FLAG_REDUCE_ON, FLAG_RESIDUAL, FLAG_DETERMINISTIC = 1, 2, 4
+MAX_EXPERTS, MAX_TOPK, MAX_WINDOW = 256, 16, 8
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("n_experts", C.c_int32), ("inter", C.c_int32), ("n_shared", C.c_int32),
+                ("shared_inter", C.c_int32), ("top_k", C.c_int32), ("top_k_vis", C.c_int32), ("dtype", C.c_int32)]
+
+
+class Weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in
+                ("router_w", "router_b", "w_gate", "w_up", "w_down", "ws_gate", "ws_up", "ws_down")]
+
+
+class RouteOut(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in
+                ("logits", "probs", "topk_idx", "topk_w", "expert_off", "row_token", "inv_row")]
+
+
+class PruneParams(C.Structure):
+    _fields_ = [("window", C.c_int32), ("sim_mode", C.c_int32), ("merge_mode", C.c_int32), ("reserved", C.c_int32),
+                ("alpha", C.c_double), ("gamma", C.c_double)]
+
+
+class FmmoeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: FMMOE_ERR_{STATUS_NAMES.get(status, status)}")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libfmmoe.so (built by paper_2511_17885_b200.build).  No fallback."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2511_17885_b200.build` "
+                          "(there is no CPU or library fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, i32, u32, sz = C.c_void_p, C.c_int64, C.c_int32, C.c_uint32, C.c_size_t
+    L.fmmoe_create.argtypes = [C.POINTER(vp), C.c_int]; L.fmmoe_create.restype = C.c_int
+    L.fmmoe_destroy.argtypes = [vp]; L.fmmoe_destroy.restype = C.c_int
+    L.fmmoe_status_string.argtypes = [C.c_int]; L.fmmoe_status_string.restype = C.c_char_p
+    L.fmmoe_get_status.argtypes = [vp, vp]; L.fmmoe_get_status.restype = C.c_int
+    L.fmmoe_launch_count.argtypes = [vp]; L.fmmoe_launch_count.restype = i64
+    L.fmmoe_workspace_bytes.argtypes = [C.POINTER(LayerDesc), i64, u32]; L.fmmoe_workspace_bytes.restype = sz
+    L.fmmoe_host_staging_bytes.argtypes = [C.POINTER(LayerDesc), i64]; L.fmmoe_host_staging_bytes.restype = sz
+    L.fmmoe_route.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), vp, vp, i64, u32, C.POINTER(RouteOut), vp, sz, vp]
+    L.fmmoe_route.restype = C.c_int
+    L.fmmoe_moe_forward.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), vp, vp, i64, u32, vp,
+                                    C.POINTER(RouteOut), vp, sz, vp]
+    L.fmmoe_moe_forward.restype = C.c_int
+    L.fmmoe_moe_forward_host.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), vp, vp, i64, u32, vp, vp, sz, vp]
+    L.fmmoe_moe_forward_host.restype = C.c_int
+    L.fmmoe_prune_kept_count.argtypes = [i64, i64, C.POINTER(PruneParams), C.POINTER(i64), C.POINTER(i64)]
+    L.fmmoe_prune_kept_count.restype = i64
+    L.fmmoe_prune_workspace_bytes.argtypes = [i64, i32]; L.fmmoe_prune_workspace_bytes.restype = sz
+    L.fmmoe_prune_visual.argtypes = [vp, C.POINTER(PruneParams), vp, i32, vp, vp, i32, i32, vp,
+                                     C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), i32,
+                                     vp, vp, vp, vp, C.POINTER(i64), vp, sz, vp]
+    L.fmmoe_prune_visual.restype = C.c_int
+    _lib = L
+    return L
+
+
+def _check(st: int, where: str):
+    if st != FMMOE_OK:
+        raise FmmoeError(st, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_contiguous()
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t: torch.dtype) -> int:
+    return {torch.float32: F32, torch.bfloat16: BF16}[t]
+
+
+def prune_params(window: int, gamma: float, alpha: float = 1.0, sim_mode: int = 0, merge_mode: int = 0) -> PruneParams:
+    return PruneParams(window, sim_mode, merge_mode, 0, float(alpha), float(gamma))
+
+
+def fmmoe_prune_kept_count(n_vis: int, n_retain: int, p: PruneParams):
+    """Host-only budget arithmetic of Section 3.2.3 -> (kept, n_merge, n_drop)."""
+    m, d = C.c_int64(0), C.c_int64(0)
+    kept = lib().fmmoe_prune_kept_count(n_vis, n_retain, C.byref(p), C.byref(m), C.byref(d))
+    return int(kept), int(m.value), int(d.value)
+
+
+def fmmoe_workspace_bytes(desc: LayerDesc, n_tokens: int, flags: int = 0) -> int:
+    return int(lib().fmmoe_workspace_bytes(C.byref(desc), n_tokens, flags))
+
+
+def make_desc(hidden, n_experts, inter, n_shared, shared_inter, top_k, top_k_vis, dtype: torch.dtype) -> LayerDesc:
+    return LayerDesc(hidden, n_experts, inter, n_shared, shared_inter, top_k, top_k_vis, _dtype_code(dtype))
+
+
+def make_weights(w: Dict[str, Optional[torch.Tensor]]) -> Weights:
+    """Device tensors -> pointer struct.  The caller keeps the tensors alive."""
+    ws = Weights()
+    for name, _ in Weights._fields_:
+        t = w.get(name)
+        if t is not None:
+            assert t.is_cuda and t.is_contiguous(), name
+            setattr(ws, name, t.data_ptr())
+    return ws
+
+
+class Handle:
+    """fmmoe_handle plus a cached workspace tensor (device memory comes from torch)."""
+
+    def __init__(self, device: int = 0):
+        self._h = C.c_void_p()
+        self.device = device
+        _check(lib().fmmoe_create(C.byref(self._h), device), "fmmoe_create")
+        self._ws: Optional[torch.Tensor] = None
+
+    def close(self):
+        if self._h:
+            lib().fmmoe_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- plumbing
+    def workspace(self, nbytes: int) -> torch.Tensor:
+        if self._ws is None or self._ws.numel() < nbytes:
+            self._ws = torch.empty(int(nbytes) + 256, dtype=torch.uint8, device=f"cuda:{self.device}")
+        return self._ws
+
+    def _ws_args(self, nbytes: int):
+        ws = self.workspace(nbytes)
+        base = ws.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        return C.c_void_p(aligned), C.c_size_t(ws.numel() - (aligned - base))
+
+    def get_status(self) -> int:
+        return int(lib().fmmoe_get_status(self._h, _stream()))
+
+    def check_status(self, where: str = "fmmoe_get_status"):
+        _check(self.get_status(), where)
+
+    def launch_count(self) -> int:
+        return int(lib().fmmoe_launch_count(self._h))
+
+    # ---- Section 3.1
+    def fmmoe_route(self, desc: LayerDesc, w: Weights, x: torch.Tensor, is_visual: torch.Tensor, flags: int,
+                    want=("logits", "probs", "topk_idx", "topk_w", "expert_off", "row_token", "inv_row")):
+        """Eq. 1-3, 5 (+ grouping by expert).  Returns a dict of freshly allocated device tensors."""
+        T, E, K = x.shape[0], desc.n_experts, desc.top_k
+        dev = x.device
+        shapes = {"logits": ((T, E), torch.float32), "probs": ((T, E), torch.float32),
+                  "topk_idx": ((T, K), torch.int32), "topk_w": ((T, K), torch.float32),
+                  "expert_off": ((E + 1,), torch.int32), "row_token": ((T * K,), torch.int32),
+                  "inv_row": ((T, K), torch.int32)}
+        out = {k: torch.empty(shapes[k][0], dtype=shapes[k][1], device=dev) for k in want}
+        ro = RouteOut(**{k: v.data_ptr() for k, v in out.items()})
+        wsp, wsn = self._ws_args(fmmoe_workspace_bytes(desc, T, flags))
+        _check(lib().fmmoe_route(self._h, C.byref(desc), C.byref(w), _ptr(x), _ptr(is_visual), T, flags,
+                                 C.byref(ro), wsp, wsn, _stream()), "fmmoe_route")
+        return out
+
+    def fmmoe_moe_forward(self, desc: LayerDesc, w: Weights, x: torch.Tensor, is_visual: torch.Tensor, flags: int,
+                          out: Optional[torch.Tensor] = None, route: Optional[Dict[str, torch.Tensor]] = None):
+        """Eq. 1-5: out[T,H].  `route`: dict of preallocated tensors to receive the routing record."""
+        T = x.shape[0]
+        if out is None:
+            out = torch.empty_like(x)
+        ro = RouteOut(**{k: v.data_ptr() for k, v in route.items()}) if route else None
+        wsp, wsn = self._ws_args(fmmoe_workspace_bytes(desc, T, flags))
+        _check(lib().fmmoe_moe_forward(self._h, C.byref(desc), C.byref(w), _ptr(x), _ptr(is_visual), T, flags,
+                                       _ptr(out), C.byref(ro) if ro is not None else None, wsp, wsn, _stream()),
+               "fmmoe_moe_forward")
+        return out
+
+    def fmmoe_moe_forward_host(self, desc: LayerDesc, w: Weights, x_host: torch.Tensor, is_visual_host: torch.Tensor,
+                               flags: int, out_host: torch.Tensor):
+        """Host-buffer variant: H2D copy, layer, D2H copy, stream synchronised on return."""
+        T = x_host.shape[0]
+        assert not x_host.is_cuda and not out_host.is_cuda and x_host.is_contiguous() and out_host.is_contiguous()
+        need = fmmoe_workspace_bytes(desc, T, flags) + int(lib().fmmoe_host_staging_bytes(C.byref(desc), T))
+        wsp, wsn = self._ws_args(need)
+        _check(lib().fmmoe_moe_forward_host(self._h, C.byref(desc), C.byref(w), C.c_void_p(x_host.data_ptr()),
+                                            C.c_void_p(is_visual_host.data_ptr()), T, flags,
+                                            C.c_void_p(out_host.data_ptr()), wsp, wsn, _stream()),
+               "fmmoe_moe_forward_host")
+        return out_host
+
+    # ---- Section 3.2
+    def fmmoe_prune_visual(self, p: PruneParams, probs: torch.Tensor, attn: Optional[torch.Tensor], x: torch.Tensor,
+                           is_visual: torch.Tensor, seq_off, n_vis, n_retain, want_aux: bool = True):
+        """Eq. 6-18 + drop rule.  Returns dict(x_out, is_visual_out, keep_idx, kind, out_seq_off)."""
+        T, H = x.shape
+        B = len(n_vis)
+        arr = C.c_int64 * (B + 1)
+        so = arr(*[int(v) for v in seq_off])
+        nv = (C.c_int64 * max(B, 1))(*[int(v) for v in n_vis])
+        nr = (C.c_int64 * max(B, 1))(*[int(v) for v in n_retain])
+        oo = arr()
+        # output size is data-independent: compute it first, then allocate exactly
+        t_out = 0
+        for b in range(B):
+            kept, _, _ = fmmoe_prune_kept_count(int(n_vis[b]), int(n_retain[b]), p)
+            if kept < 0:
+                raise FmmoeError(1, "fmmoe_prune_kept_count")
+            t_out += int(seq_off[b + 1]) - int(seq_off[b]) - int(n_vis[b]) + kept
+        dev = x.device
+        x_out = torch.empty((t_out, H), dtype=x.dtype, device=dev)
+        vis_out = torch.empty(t_out, dtype=torch.uint8, device=dev) if want_aux else None
+        keep_idx = torch.empty(t_out, dtype=torch.int32, device=dev) if want_aux else None
+        kind = torch.empty(t_out, dtype=torch.uint8, device=dev) if want_aux else None
+        wsp, wsn = self._ws_args(int(lib().fmmoe_prune_workspace_bytes(T, B)))
+        _check(lib().fmmoe_prune_visual(self._h, C.byref(p), _ptr(probs), probs.shape[1] if probs is not None else 1,
+                                        _ptr(attn), _ptr(x), _dtype_code(x.dtype), H, _ptr(is_visual), so, nv, nr, B,
+                                        _ptr(x_out), _ptr(vis_out), _ptr(keep_idx), _ptr(kind), oo, wsp, wsn,
+                                        _stream()), "fmmoe_prune_visual")
+        return {"x_out": x_out, "is_visual_out": vis_out, "keep_idx": keep_idx, "kind": kind,
+                "out_seq_off": [int(v) for v in oo]}

@@ -1,0 +1,294 @@
+// C-ABI entry points: handle, workspace planning, argument validation, and the launch
+// sequence of one MoE layer (Section 3.1):
+//   clear -> route (Eq. 1-3, 5 + histogram) -> permute-by-expert -> [gather rows]
+//   -> GEMM-1 + SwiGLU -> GEMM-2 + combine (Eq. 4) -> finalize.
+#include <string.h>
+
+#include "internal.h"
+
+namespace fmmoe {
+
+static bool desc_ok(const fmmoe_layer_desc* d) {
+  if (!d) return false;
+  if (d->hidden < 1 || d->n_experts < 1 || d->n_experts > FMMOE_MAX_EXPERTS || d->inter < 1) return false;
+  if (d->n_shared < 0 || (d->n_shared > 0 && d->shared_inter < 1)) return false;
+  if (d->top_k < 1 || d->top_k > FMMOE_MAX_TOPK || d->top_k > d->n_experts) return false;
+  if (d->top_k_vis < 0 || d->top_k_vis > d->top_k) return false;
+  if (d->top_k_vis == 0 && d->n_shared == 0) return false;   // p = 0 needs shared experts (Section 3.1)
+  if (d->dtype != FMMOE_F32 && d->dtype != FMMOE_BF16) return false;
+  return true;
+}
+
+static fmmoe_status shape_supported(const fmmoe_layer_desc& d, bool forward) {
+  const int elem = d.dtype == FMMOE_BF16 ? 2 : 4;
+  if ((d.hidden * elem) % 16) return FMMOE_ERR_UNSUPPORTED;
+  if (d.dtype == FMMOE_BF16) {
+    if (d.hidden % 64) return FMMOE_ERR_UNSUPPORTED;
+    if (forward && (d.inter % 64 || (d.n_shared && d.shared_inter % 64))) return FMMOE_ERR_UNSUPPORTED;
+  } else if (forward && (d.hidden % 4 || d.inter % 4 || (d.n_shared && d.shared_inter % 4))) {
+    return FMMOE_ERR_UNSUPPORTED;
+  }
+  return FMMOE_OK;
+}
+
+bool plan_workspace(const fmmoe_layer_desc& d, int64_t T, uint32_t flags, WsPlan* p) {
+  if (T < 0) return false;
+  const size_t elem = d.dtype == FMMOE_BF16 ? 2 : 4;
+  const bool det = flags & FMMOE_FLAG_DETERMINISTIC;
+  const int block_m = d.dtype == FMMOE_BF16 ? TC_BLOCK_M : F32_BLOCK_M;
+  const size_t Tz = (size_t)T, K = d.top_k, H = d.hidden, I = d.inter;
+  const size_t P = Tz * K;
+  p->p_max = (int64_t)P;
+  p->max_mtiles = (int32_t)(d.n_experts + P / block_m + 1);
+  size_t o = 0;
+  auto take = [&](size_t bytes) { const size_t at = o; o = align_up(o + bytes, 256); return at; };
+  p->zero_off = 0;
+  p->counts_off = take(FMMOE_MAX_EXPERTS * 4);
+  p->misc_off = take(8 * 4);
+  p->acc_off = take(det ? 0 : Tz * H * 4);
+  p->zero_bytes = o;
+  p->topk_idx_off = take(P * 4);
+  p->topk_w_off = take(P * 4);
+  p->inv_row_off = take(P * 4);
+  p->expert_off_off = take((FMMOE_MAX_EXPERTS + 1) * 4);
+  p->row_token_off = take(P * 4);
+  p->row_gate_off = take(P * 4);
+  p->mtiles_off = take((size_t)p->max_mtiles * sizeof(MTile));
+  p->xp_off = take(d.dtype == FMMOE_BF16 ? P * H * elem : 0);
+  p->act_off = take(P * I * elem);
+  p->act_sh_off = take((size_t)d.n_shared * Tz * d.shared_inter * elem);
+  p->y_off = take(det ? P * H * 4 : 0);
+  p->ysh_off = take(det ? (size_t)d.n_shared * Tz * H * 4 : 0);
+  p->total = o;
+  return true;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+struct RoutePtrs {
+  float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row;
+  int32_t* expert_off; int32_t* row_token; float* row_gate; int32_t* counts; int32_t* misc; MTile* mtiles;
+};
+
+static RoutePtrs bind_route(const WsPlan& pl, char* ws, const fmmoe_route_out* out) {
+  RoutePtrs r;
+  r.logits = out ? out->logits : nullptr;
+  r.probs = out ? out->probs : nullptr;
+  r.topk_idx = (out && out->topk_idx) ? out->topk_idx : reinterpret_cast<int32_t*>(ws + pl.topk_idx_off);
+  r.topk_w = (out && out->topk_w) ? out->topk_w : reinterpret_cast<float*>(ws + pl.topk_w_off);
+  r.inv_row = (out && out->inv_row) ? out->inv_row : reinterpret_cast<int32_t*>(ws + pl.inv_row_off);
+  r.expert_off = (out && out->expert_off) ? out->expert_off : reinterpret_cast<int32_t*>(ws + pl.expert_off_off);
+  r.row_token = (out && out->row_token) ? out->row_token : reinterpret_cast<int32_t*>(ws + pl.row_token_off);
+  r.row_gate = reinterpret_cast<float*>(ws + pl.row_gate_off);
+  r.counts = reinterpret_cast<int32_t*>(ws + pl.counts_off);
+  r.misc = reinterpret_cast<int32_t*>(ws + pl.misc_off);
+  r.mtiles = reinterpret_cast<MTile*>(ws + pl.mtiles_off);
+  return r;
+}
+
+static fmmoe_status check_common(fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w, const void* x,
+                                 const uint8_t* is_visual, int64_t T, bool forward) {
+  if (!h || !desc_ok(d) || !w || T < 0) return FMMOE_ERR_INVALID_ARG;
+  if (T > (int64_t)0x7fffffff / d->top_k) return FMMOE_ERR_UNSUPPORTED;
+  const fmmoe_status st = shape_supported(*d, forward);
+  if (st != FMMOE_OK) return st;
+  if (!w->router_w || !aligned16(w->router_w)) return FMMOE_ERR_INVALID_ARG;
+  if (T > 0 && (!x || !is_visual || !aligned16(x))) return FMMOE_ERR_INVALID_ARG;
+  if (forward) {
+    if (!w->w_gate || !w->w_up || !w->w_down) return FMMOE_ERR_INVALID_ARG;
+    if (!aligned16(w->w_gate) || !aligned16(w->w_up) || !aligned16(w->w_down)) return FMMOE_ERR_INVALID_ARG;
+    if (d->n_shared) {
+      if (!w->ws_gate || !w->ws_up || !w->ws_down) return FMMOE_ERR_INVALID_ARG;
+      if (!aligned16(w->ws_gate) || !aligned16(w->ws_up) || !aligned16(w->ws_down)) return FMMOE_ERR_INVALID_ARG;
+    }
+  }
+  return FMMOE_OK;
+}
+
+static fmmoe_status run_route(fmmoe_handle* h, const fmmoe_layer_desc& d, const fmmoe_weights& w, const void* x,
+                              const uint8_t* is_visual, int64_t T, uint32_t flags, const RoutePtrs& r,
+                              bool need_permute, cudaStream_t s) {
+  RouteArgs ra;
+  ra.x = x; ra.router_w = w.router_w; ra.router_b = w.router_b; ra.is_visual = is_visual;
+  ra.T = T; ra.H = d.hidden; ra.E = d.n_experts; ra.K = d.top_k; ra.Kv = d.top_k_vis;
+  ra.reduce_on = (flags & FMMOE_FLAG_REDUCE_ON) ? 1 : 0; ra.dtype = d.dtype;
+  ra.logits = r.logits; ra.probs = r.probs; ra.topk_idx = r.topk_idx; ra.topk_w = r.topk_w;
+  ra.inv_row = r.inv_row; ra.counts = r.counts;
+  fmmoe_status st = launch_route(h, ra, s);
+  if (st != FMMOE_OK || !need_permute) return st;
+  PermuteArgs pa;
+  pa.topk_idx = r.topk_idx; pa.topk_w = r.topk_w; pa.counts = r.counts;
+  pa.T = T; pa.K = d.top_k; pa.E = d.n_experts;
+  pa.block_m = d.dtype == FMMOE_BF16 ? TC_BLOCK_M : F32_BLOCK_M;
+  pa.expert_off = r.expert_off; pa.row_token = r.row_token; pa.row_gate = r.row_gate; pa.inv_row = r.inv_row;
+  pa.mtiles = r.mtiles; pa.n_mtiles = r.misc;
+  return launch_permute(h, pa, s);
+}
+
+}  // namespace fmmoe
+
+using namespace fmmoe;
+
+extern "C" __attribute__((visibility("default"))) const char* fmmoe_status_string(fmmoe_status s) {
+  switch (s) {
+    case FMMOE_OK: return "ok";
+    case FMMOE_ERR_INVALID_ARG: return "invalid argument";
+    case FMMOE_ERR_UNSUPPORTED: return "unsupported shape or type";
+    case FMMOE_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case FMMOE_ERR_CUDA: return "CUDA call failed";
+    case FMMOE_ERR_TIMEOUT: return "device-side wait timed out";
+    case FMMOE_ERR_INTERNAL: return "internal consistency check failed";
+  }
+  return "unknown status";
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmoe_handle** out, int device) {
+  if (!out) return FMMOE_ERR_INVALID_ARG;
+  *out = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return FMMOE_ERR_CUDA;
+  FMMOE_CUDA_TRY(cudaSetDevice(device));
+  cudaDeviceProp prop;
+  FMMOE_CUDA_TRY(cudaGetDeviceProperties(&prop, device));
+  if (prop.major != 10) return FMMOE_ERR_UNSUPPORTED;   // kernels are built for sm_100a only
+  fmmoe_handle* h = new fmmoe_handle();
+  h->device = device;
+  h->sm_count = prop.multiProcessorCount;
+  h->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+  h->launches = 0;
+  h->d_status = nullptr; h->h_status = nullptr; h->encode_tiled = nullptr;
+  if (cudaMalloc(&h->d_status, 256) != cudaSuccess || cudaMemset(h->d_status, 0, 256) != cudaSuccess ||
+      cudaMallocHost(&h->h_status, 256) != cudaSuccess) {
+    if (h->d_status) cudaFree(h->d_status);
+    delete h;
+    return FMMOE_ERR_CUDA;
+  }
+  cudaDriverEntryPointQueryResult qres;
+  void* fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+      qres == cudaDriverEntryPointSuccess)
+    h->encode_tiled = fn;
+  *out = h;
+  return FMMOE_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_destroy(fmmoe_handle* h) {
+  if (!h) return FMMOE_OK;
+  cudaSetDevice(h->device);
+  if (h->d_status) cudaFree(h->d_status);
+  if (h->h_status) cudaFreeHost(h->h_status);
+  delete h;
+  return FMMOE_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_get_status(fmmoe_handle* h, void* cuda_stream) {
+  if (!h) return FMMOE_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  FMMOE_CUDA_TRY(cudaMemcpyAsync(h->h_status, h->d_status, 4, cudaMemcpyDeviceToHost, s));
+  FMMOE_CUDA_TRY(cudaMemsetAsync(h->d_status, 0, 4, s));
+  FMMOE_CUDA_TRY(cudaStreamSynchronize(s));
+  const int v = h->h_status[0];
+  if (v == 0) return FMMOE_OK;
+  return v == FMMOE_ERR_TIMEOUT ? FMMOE_ERR_TIMEOUT : FMMOE_ERR_INTERNAL;
+}
+
+extern "C" __attribute__((visibility("default"))) int64_t fmmoe_launch_count(const fmmoe_handle* h) { return h ? h->launches : -1; }
+
+extern "C" __attribute__((visibility("default"))) size_t fmmoe_workspace_bytes(const fmmoe_layer_desc* d, int64_t n_tokens, uint32_t flags) {
+  WsPlan p;
+  if (!desc_ok(d) || !plan_workspace(*d, n_tokens, flags, &p)) return 0;
+  return p.total + 256;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_route(fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w, const void* x,
+                                    const uint8_t* is_visual, int64_t T, uint32_t flags, const fmmoe_route_out* out,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  fmmoe_status st = check_common(h, d, w, x, is_visual, T, false);
+  if (st != FMMOE_OK) return st;
+  WsPlan pl;
+  plan_workspace(*d, T, flags, &pl);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < pl.total) return FMMOE_ERR_WORKSPACE;
+  if (T == 0) return FMMOE_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  FMMOE_CUDA_TRY(cudaMemsetAsync(ws + pl.counts_off, 0, pl.acc_off - pl.counts_off, s));
+  const RoutePtrs r = bind_route(pl, ws, out);
+  const bool need_permute = out && (out->expert_off || out->row_token || out->inv_row);
+  return run_route(h, *d, *w, x, is_visual, T, flags, r, need_permute, s);
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward(fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w,
+                                          const void* x, const uint8_t* is_visual, int64_t T, uint32_t flags, void* out,
+                                          const fmmoe_route_out* route, void* workspace, size_t workspace_bytes,
+                                          void* cuda_stream) {
+  fmmoe_status st = check_common(h, d, w, x, is_visual, T, true);
+  if (st != FMMOE_OK) return st;
+  if (T > 0 && (!out || !aligned16(out) || out == x)) return FMMOE_ERR_INVALID_ARG;
+  WsPlan pl;
+  plan_workspace(*d, T, flags, &pl);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < pl.total) return FMMOE_ERR_WORKSPACE;
+  if (T == 0) return FMMOE_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  const bool det = flags & FMMOE_FLAG_DETERMINISTIC;
+  FMMOE_CUDA_TRY(cudaMemsetAsync(ws + pl.zero_off, 0, pl.zero_bytes, s));
+  const RoutePtrs r = bind_route(pl, ws, route);
+  st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, s);
+  if (st != FMMOE_OK) return st;
+
+  FfnArgs fa = {};
+  fa.d = d; fa.w = w; fa.x = x; fa.T = T; fa.p_max = pl.p_max;
+  fa.mtiles = r.mtiles; fa.n_mtiles = r.misc; fa.max_mtiles = pl.max_mtiles;
+  fa.row_token = r.row_token; fa.row_gate = r.row_gate;
+  fa.xp = ws + pl.xp_off; fa.act = ws + pl.act_off; fa.act_sh = ws + pl.act_sh_off;
+  fa.acc = det ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off);
+  fa.y = det ? reinterpret_cast<float*>(ws + pl.y_off) : nullptr;
+  fa.ysh = det ? reinterpret_cast<float*>(ws + pl.ysh_off) : nullptr;
+  fa.deterministic = det; fa.d_status = h->d_status;
+  if (d->dtype == FMMOE_BF16) {
+    st = launch_gather_rows(h, x, r.row_token, r.expert_off, d->n_experts, pl.p_max, d->hidden, 2, fa.xp, s);
+    if (st != FMMOE_OK) return st;
+    st = launch_ffn_tc(h, fa, s);
+  } else {
+    st = launch_ffn_f32(h, fa, s);
+  }
+  if (st != FMMOE_OK) return st;
+
+  FinalizeArgs fin = {};
+  fin.x = x; fin.out = out; fin.T = T; fin.H = d->hidden; fin.K = d->top_k; fin.n_shared = d->n_shared;
+  fin.dtype = d->dtype; fin.add_residual = (flags & FMMOE_FLAG_RESIDUAL) ? 1 : 0; fin.deterministic = det;
+  fin.acc = fa.acc; fin.y = fa.y; fin.ysh = fa.ysh; fin.inv_row = r.inv_row; fin.topk_w = r.topk_w;
+  return launch_finalize(h, fin, s);
+}
+
+extern "C" __attribute__((visibility("default"))) size_t fmmoe_host_staging_bytes(const fmmoe_layer_desc* d, int64_t T) {
+  if (!desc_ok(d) || T < 0) return 0;
+  const size_t elem = d->dtype == FMMOE_BF16 ? 2 : 4;
+  return 2 * align_up((size_t)T * d->hidden * elem, 256) + align_up((size_t)T, 256);
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward_host(fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w,
+                                               const void* x_host, const uint8_t* is_visual_host, int64_t T,
+                                               uint32_t flags, void* out_host, void* workspace, size_t workspace_bytes,
+                                               void* cuda_stream) {
+  if (!h || !desc_ok(d) || T < 0) return FMMOE_ERR_INVALID_ARG;
+  if (T > 0 && (!x_host || !is_visual_host || !out_host)) return FMMOE_ERR_INVALID_ARG;
+  const size_t elem = d->dtype == FMMOE_BF16 ? 2 : 4;
+  const size_t xb = (size_t)T * d->hidden * elem;
+  const size_t stage = fmmoe_host_staging_bytes(d, T);
+  const size_t inner = fmmoe_workspace_bytes(d, T, flags);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < stage + inner) return FMMOE_ERR_WORKSPACE;
+  if (T == 0) return FMMOE_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  char* dx = ws;
+  char* dout = ws + align_up(xb, 256);
+  uint8_t* dvis = reinterpret_cast<uint8_t*>(ws + 2 * align_up(xb, 256));
+  FMMOE_CUDA_TRY(cudaMemcpyAsync(dx, x_host, xb, cudaMemcpyHostToDevice, s));
+  FMMOE_CUDA_TRY(cudaMemcpyAsync(dvis, is_visual_host, (size_t)T, cudaMemcpyHostToDevice, s));
+  const fmmoe_status st = fmmoe_moe_forward(h, d, w, dx, dvis, T, flags, dout, nullptr, ws + stage, workspace_bytes - stage, s);
+  if (st != FMMOE_OK) return st;
+  FMMOE_CUDA_TRY(cudaMemcpyAsync(out_host, dout, xb, cudaMemcpyDeviceToHost, s));
+  FMMOE_CUDA_TRY(cudaStreamSynchronize(s));
+  return FMMOE_OK;
+}

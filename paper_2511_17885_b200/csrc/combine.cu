@@ -1,0 +1,87 @@
+// Last step of Eq. 4: turn the fp32 combine result into the layer output.
+// Atomic mode: the GEMM-2 epilogue has already summed g_j * FFN_j(x) and the shared
+// experts into `acc`; this kernel adds the residual (optional) and rounds to the
+// storage type.  Deterministic mode: the per-pair outputs y were stored instead and
+// are summed here in a fixed order (slots 0..K-1, then shared experts 0..N_s-1).
+#include <cuda_bf16.h>
+
+#include "internal.h"
+
+namespace fmmoe {
+
+struct FinalizeDev {
+  const void* x; void* out; long long T; int H, K, n_shared, add_residual, deterministic;
+  const float* acc; const float* y; const float* ysh; const int32_t* inv_row; const float* topk_w;
+};
+
+template <typename T> struct Vec4;
+template <> struct Vec4<float> {
+  static __device__ __forceinline__ float4 load(const float* p) { return *reinterpret_cast<const float4*>(p); }
+  static __device__ __forceinline__ void store(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+};
+template <> struct Vec4<__nv_bfloat16> {
+  static __device__ __forceinline__ float4 load(const __nv_bfloat16* p) {
+    const uint2 u = *reinterpret_cast<const uint2*>(p);
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+  }
+  static __device__ __forceinline__ void store(__nv_bfloat16* p, float4 v) {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    uint2 u;
+    u.x = *reinterpret_cast<const uint32_t*>(&a);
+    u.y = *reinterpret_cast<const uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(p) = u;
+  }
+};
+
+template <typename T>
+__global__ void finalize_kernel(const FinalizeDev a) {
+  const int hv = a.H / 4;
+  const long long n = a.T * hv;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const long long t = i / hv;
+    const int c = (int)(i - t * hv) * 4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (!a.deterministic) {
+      v = *reinterpret_cast<const float4*>(a.acc + t * a.H + c);
+    } else {
+      for (int s = 0; s < a.K; ++s) {
+        const int row = a.inv_row[t * a.K + s];
+        if (row < 0) continue;
+        const float g = a.topk_w[t * a.K + s];
+        const float4 yv = *reinterpret_cast<const float4*>(a.y + (long long)row * a.H + c);
+        v.x = fmaf(g, yv.x, v.x); v.y = fmaf(g, yv.y, v.y); v.z = fmaf(g, yv.z, v.z); v.w = fmaf(g, yv.w, v.w);
+      }
+      for (int s = 0; s < a.n_shared; ++s) {
+        const float4 yv = *reinterpret_cast<const float4*>(a.ysh + ((long long)s * a.T + t) * a.H + c);
+        v.x += yv.x; v.y += yv.y; v.z += yv.z; v.w += yv.w;
+      }
+    }
+    if (a.add_residual) {
+      const float4 xv = Vec4<T>::load(static_cast<const T*>(a.x) + t * a.H + c);
+      v.x += xv.x; v.y += xv.y; v.z += xv.z; v.w += xv.w;
+    }
+    Vec4<T>::store(static_cast<T*>(a.out) + t * a.H + c, v);
+  }
+}
+
+fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_t s) {
+  if (a.T == 0) return FMMOE_OK;
+  FinalizeDev d;
+  d.x = a.x; d.out = a.out; d.T = a.T; d.H = a.H; d.K = a.K; d.n_shared = a.n_shared;
+  d.add_residual = a.add_residual; d.deterministic = a.deterministic;
+  d.acc = a.acc; d.y = a.y; d.ysh = a.ysh; d.inv_row = a.inv_row; d.topk_w = a.topk_w;
+  const long long n = a.T * (a.H / 4);
+  const int threads = 256;
+  long long blocks = (n + threads - 1) / threads;
+  const long long cap = (long long)h->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  if (a.dtype == FMMOE_BF16) finalize_kernel<__nv_bfloat16><<<(int)blocks, threads, 0, s>>>(d);
+  else finalize_kernel<float><<<(int)blocks, threads, 0, s>>>(d);
+  FMMOE_CUDA_TRY(cudaGetLastError());
+  h->launches += 1;
+  return FMMOE_OK;
+}
+
+}  // namespace fmmoe

@@ -1,0 +1,363 @@
+// Expert FFNs on the 5th-generation tensor cores (tcgen05), bf16 in / fp32 accumulate.
+//
+// Eq. 4 needs, for every routed (token, expert) pair and every (token, shared expert)
+// pair, y = W_down (silu(W_gate x) * (W_up x)).  With the pairs grouped by expert
+// this is two grouped GEMMs:
+//   GEMM-1  [rows_e, H] x [H, 2*S_m]  -> SwiGLU in the epilogue -> act [rows, S_m] bf16
+//   GEMM-2  [rows_e, S_m] x [S_m, H]  -> gate-weighted combine in the epilogue
+// Both run in one persistent, warp-specialised kernel template:
+//   warp 0    : TMA producer  (A tile 128x64 + two B boxes 128x64 per stage, 128B swizzle)
+//   warp 1    : UMMA issuer   (one thread; 128x256x16 tcgen05.mma, accumulators in TMEM)
+//   warps 2-5 : epilogue      (tcgen05.ld -> registers -> global), overlapped with the next
+//               tile's main loop through two TMEM accumulator stages (2 x 256 columns).
+// A tile is (M-tile of 128 grouped rows) x (N-block).  Tile ids run N-block-major so
+// that CTAs working at the same time share weight tiles through L2.
+// GEMM-1's B tile is 128 gate rows + 128 up rows of the same expert, so one thread
+// holds gate and up of the same (row, column) in TMEM columns c and 128+c.
+// Every wait is bounded; on expiry the CTA records FMMOE_ERR_TIMEOUT and leaves.
+#include <cuda_bf16.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace fmmoe {
+
+constexpr int G_BM = TC_BLOCK_M;   // 128
+constexpr int G_BK = 64;           // one 128-byte swizzle atom of bf16
+constexpr int G_STAGES = 4;
+constexpr int G_A_BYTES = G_BM * G_BK * 2;          // 16 KB
+constexpr int G_B_BYTES = 2 * 128 * G_BK * 2;       // 32 KB (two 128-row boxes)
+constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;
+constexpr int G_THREADS = 192;
+constexpr int G_TMEM_COLS = 512;
+constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+
+struct Segment {          // routed experts (0) or shared experts (1)
+  int n_nblocks;          // N-blocks per group
+  int k_blocks;           // K / 64
+  int b_rows_per_group;   // rows of the B tensor per group (S_m for GEMM-1, H for GEMM-2)
+  int n_valid;            // valid output columns per group (S_m for GEMM-1, H for GEMM-2)
+  int a_group_stride;     // rows added to the A row per group index (shared experts only)
+  int out_group_stride;   // rows added to the output row per group index
+  int ld_out;             // leading dimension of the output (elements)
+};
+
+struct GemmParams {
+  const MTile* mtiles;        // routed M-tiles
+  const int32_t* n_mtiles;    // device: number of routed M-tiles
+  int n_experts;
+  int shared_mtiles;          // N_s * ceil(T/128), host-known
+  int mt_per_shared;          // ceil(T/128)
+  long long T;
+  Segment seg[2];
+  // epilogue
+  __nv_bfloat16* act[2];      // MODE 0: activation outputs (routed, shared)
+  const int32_t* row_token;   // MODE 1
+  const float* row_gate;      // MODE 1
+  float* acc;                 // MODE 1 atomic:  [T, H]
+  float* y[2];                // MODE 1 deterministic: routed [P, H], shared [N_s*T, H]
+  int deterministic;
+  int* status;
+};
+
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+struct TileInfo {
+  int seg, group_local, row0, rows, nb;
+};
+
+__device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, int tile, int n_mt_r) {
+  TileInfo ti;
+  const int routed_tiles = n_mt_r * p.seg[0].n_nblocks;
+  if (tile < routed_tiles) {
+    ti.seg = 0;
+    ti.nb = tile / n_mt_r;
+    const MTile m = p.mtiles[tile - ti.nb * n_mt_r];
+    ti.group_local = m.group; ti.row0 = m.row0; ti.rows = m.rows;
+  } else {
+    const int t2 = tile - routed_tiles;
+    ti.seg = 1;
+    ti.nb = t2 / p.shared_mtiles;
+    const int mt = t2 - ti.nb * p.shared_mtiles;
+    ti.group_local = mt / p.mt_per_shared;
+    const int mb = mt - ti.group_local * p.mt_per_shared;
+    ti.row0 = mb * G_BM;
+    const long long left = p.T - (long long)ti.row0;
+    ti.rows = left < G_BM ? (int)left : G_BM;
+  }
+  return ti;
+}
+
+// MODE 0: GEMM-1 + SwiGLU.  MODE 1: GEMM-2 + combine.
+template <int MODE>
+__global__ void __launch_bounds__(G_THREADS, 1)
+ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__ CUtensorMap tmA_s,
+              const __grid_constant__ CUtensorMap tmB0_r, const __grid_constant__ CUtensorMap tmB1_r,
+              const __grid_constant__ CUtensorMap tmB0_s, const __grid_constant__ CUtensorMap tmB1_s,
+              const GemmParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  unsigned char* smem = smem_raw + ((1024 - (raw & 1023)) & 1023);   // 1024-byte aligned tiles (128B swizzle)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G_STAGES * G_STAGE_BYTES);
+  uint64_t* full_bar = bars;                   // [G_STAGES]
+  uint64_t* empty_bar = bars + G_STAGES;       // [G_STAGES]
+  uint64_t* tfull_bar = bars + 2 * G_STAGES;   // [2]
+  uint64_t* tempty_bar = tfull_bar + 2;        // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < G_STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&tfull_bar[i], 1); mbar_init(&tempty_bar[i], 128); }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, G_TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_mt_r = p.n_mtiles ? *p.n_mtiles : 0;
+  const int total_tiles = n_mt_r * p.seg[0].n_nblocks + p.shared_mtiles * p.seg[1].n_nblocks;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmA_r); tma_prefetch_desc(&tmB0_r); tma_prefetch_desc(&tmB1_r);
+      if (p.shared_mtiles) { tma_prefetch_desc(&tmA_s); tma_prefetch_desc(&tmB0_s); tma_prefetch_desc(&tmB1_s); }
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const TileInfo ti = decode_tile(p, tile, n_mt_r);
+        const Segment& sg = p.seg[ti.seg];
+        const CUtensorMap* mA = ti.seg ? &tmA_s : &tmA_r;
+        const CUtensorMap* mB0 = ti.seg ? &tmB0_s : &tmB0_r;
+        const CUtensorMap* mB1 = ti.seg ? &tmB1_s : &tmB1_r;
+        const int a_row = ti.row0 + ti.group_local * sg.a_group_stride;
+        const int b_y0 = ti.group_local * sg.b_rows_per_group + ti.nb * (MODE == 0 ? 128 : 256);
+        const int b_y1 = MODE == 0 ? b_y0 : b_y0 + 128;
+        for (int kb = 0; kb < sg.k_blocks; ++kb) {
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
+          unsigned char* sA = smem + stage * G_STAGE_BYTES;
+          mbar_arrive_expect_tx(&full_bar[stage], G_STAGE_BYTES);
+          tma_load_2d(sA, mA, &full_bar[stage], kb * G_BK, a_row);
+          tma_load_2d(sA + G_A_BYTES, mB0, &full_bar[stage], kb * G_BK, b_y0);
+          tma_load_2d(sA + G_A_BYTES + G_B_BYTES / 2, mB1, &full_bar[stage], kb * G_BK, b_y1);
+          if (++stage == G_STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ UMMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(G_BM, 256);
+      int stage = 0; uint32_t phase = 0;
+      int as = 0; uint32_t aphase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const TileInfo ti = decode_tile(p, tile, n_mt_r);
+        const int k_blocks = p.seg[ti.seg].k_blocks;
+        if (!mbar_wait(&tempty_bar[as], aphase ^ 1)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + as * 256;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&full_bar[stage], phase)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sA = smem_u32(smem + stage * G_STAGE_BYTES);
+          const uint64_t da = umma_desc_sw128(sA);
+          const uint64_t db = umma_desc_sw128(sA + G_A_BYTES);
+#pragma unroll
+          for (int k = 0; k < G_BK / 16; ++k)
+            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);   // +32 bytes per K=16 step
+          umma_commit(&empty_bar[stage]);   // stage reusable once these MMAs have read it
+          if (++stage == G_STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        umma_commit(&tfull_bar[as]);        // accumulator complete
+        if (++as == 2) { as = 0; aphase ^= 1; }
+      }
+      if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;                 // TMEM lane quarter this warp may access
+    const int r = q * 32 + lane;            // row of the tile held by this thread
+    int as = 0; uint32_t aphase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const TileInfo ti = decode_tile(p, tile, n_mt_r);
+      const Segment& sg = p.seg[ti.seg];
+      if (!mbar_wait(&tfull_bar[as], aphase)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + as * 256 + (static_cast<uint32_t>(q * 32) << 16);
+      const bool row_ok = r < ti.rows;
+      if (MODE == 0) {
+        const long long out_row = (long long)ti.row0 + r + (long long)ti.group_local * sg.out_group_stride;
+        __nv_bfloat16* dst = p.act[ti.seg] + out_row * sg.ld_out + ti.nb * 128;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          if (ti.nb * 128 + c * 32 >= sg.n_valid) break;   // warp-uniform
+          uint32_t g[32], u[32];
+          tmem_ld32(taddr + c * 32, g);
+          tmem_ld32(taddr + 128 + c * 32, u);
+          tmem_ld_wait();
+          uint32_t o[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+            const float a0 = g0 / (1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
+            const float a1 = g1 / (1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
+            const __nv_bfloat162 h = __floats2bfloat162_rn(a0, a1);
+            o[i] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+          if (row_ok) {
+            uint4* d4 = reinterpret_cast<uint4*>(dst + c * 32);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) d4[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+          }
+        }
+      } else {
+        long long tok; float gate;
+        if (ti.seg == 0) {
+          tok = row_ok ? p.row_token[ti.row0 + r] : 0;
+          gate = row_ok ? p.row_gate[ti.row0 + r] : 0.f;
+        } else {
+          tok = ti.row0 + r; gate = 1.f;
+        }
+        float* dst;
+        if (p.deterministic) {
+          const long long out_row = (long long)ti.row0 + r + (long long)ti.group_local * sg.out_group_stride;
+          dst = p.y[ti.seg] + out_row * sg.ld_out + ti.nb * 256;
+          gate = 1.f;   // gates are applied by the ordered gather
+        } else {
+          dst = p.acc + tok * sg.ld_out + ti.nb * 256;
+        }
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+          if (ti.nb * 256 + c * 32 >= sg.n_valid) break;   // warp-uniform
+          uint32_t v[32];
+          tmem_ld32(taddr + c * 32, v);
+          tmem_ld_wait();
+          if (row_ok) {
+            if (p.deterministic) {
+              float4* d4 = reinterpret_cast<float4*>(dst + c * 32);
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                d4[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                    __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+            } else {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                red_add_v4(dst + c * 32 + 4 * i, gate * __uint_as_float(v[4 * i]), gate * __uint_as_float(v[4 * i + 1]),
+                           gate * __uint_as_float(v[4 * i + 2]), gate * __uint_as_float(v[4 * i + 3]));
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(&tempty_bar[as]);
+      if (++as == 2) { as = 0; aphase ^= 1; }
+    }
+    if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // give copies still in flight time to land before the shared memory is released
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, G_TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 row-major [rows, cols] tensor, box = 64 columns x box_rows rows, 128-byte swizzle.
+static bool make_map(fmmoe_handle* h, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  if (rows == 0) rows = 1;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {G_BK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(h->encode_tiled)(
+      m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
+  const fmmoe_layer_desc& d = *a.d;
+  const int H = d.hidden, I = d.inter, E = d.n_experts, Ns = d.n_shared, Is = d.shared_inter;
+  if (!h->encode_tiled) return FMMOE_ERR_CUDA;
+  if (a.T == 0) return FMMOE_OK;
+  const int mtps = (int)((a.T + G_BM - 1) / G_BM);
+  const uint64_t p_rows = (uint64_t)a.p_max;
+
+  CUtensorMap A1r, A1s, G1r, U1r, G1s, U1s, A2r, A2s, D2r, D2s;
+  bool ok = true;
+  ok &= make_map(h, &A1r, a.xp, p_rows, H, 128);
+  ok &= make_map(h, &G1r, a.w->w_gate, (uint64_t)E * I, H, 128);
+  ok &= make_map(h, &U1r, a.w->w_up, (uint64_t)E * I, H, 128);
+  ok &= make_map(h, &A2r, a.act, p_rows, I, 128);
+  ok &= make_map(h, &D2r, a.w->w_down, (uint64_t)E * H, I, 128);
+  if (Ns) {
+    ok &= make_map(h, &A1s, a.x, (uint64_t)a.T, H, 128);
+    ok &= make_map(h, &G1s, a.w->ws_gate, (uint64_t)Ns * Is, H, 128);
+    ok &= make_map(h, &U1s, a.w->ws_up, (uint64_t)Ns * Is, H, 128);
+    ok &= make_map(h, &A2s, a.act_sh, (uint64_t)Ns * a.T, Is, 128);
+    ok &= make_map(h, &D2s, a.w->ws_down, (uint64_t)Ns * H, Is, 128);
+  } else {
+    A1s = A1r; G1s = G1r; U1s = U1r; A2s = A2r; D2s = D2r;
+  }
+  if (!ok) return FMMOE_ERR_CUDA;
+
+  GemmParams p1 = {};
+  p1.mtiles = a.mtiles; p1.n_mtiles = a.n_mtiles; p1.n_experts = E;
+  p1.shared_mtiles = Ns * mtps; p1.mt_per_shared = mtps; p1.T = a.T;
+  p1.seg[0] = Segment{(I + 127) / 128, H / G_BK, I, I, 0, 0, I};
+  p1.seg[1] = Segment{Ns ? (Is + 127) / 128 : 0, H / G_BK, Is, Is, 0, (int)a.T, Is};
+  p1.act[0] = static_cast<__nv_bfloat16*>(a.act); p1.act[1] = static_cast<__nv_bfloat16*>(a.act_sh);
+  p1.status = a.d_status;
+
+  GemmParams p2 = p1;
+  p2.seg[0] = Segment{(H + 255) / 256, I / G_BK, H, H, 0, 0, H};
+  p2.seg[1] = Segment{Ns ? (H + 255) / 256 : 0, Ns ? Is / G_BK : 0, H, H, (int)a.T, (int)a.T, H};
+  p2.row_token = a.row_token; p2.row_gate = a.row_gate; p2.acc = a.acc;
+  p2.y[0] = a.y; p2.y[1] = a.ysh; p2.deterministic = a.deterministic;
+
+  static bool attr_set = false;
+  if (!attr_set) {
+    FMMOE_CUDA_TRY(cudaFuncSetAttribute(ffn_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES));
+    FMMOE_CUDA_TRY(cudaFuncSetAttribute(ffn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES));
+    attr_set = true;
+  }
+  const int grid = h->sm_count;
+  ffn_tc_kernel<0><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(A1r, A1s, G1r, U1r, G1s, U1s, p1);
+  FMMOE_CUDA_TRY(cudaGetLastError());
+  ffn_tc_kernel<1><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(A2r, A2s, D2r, D2r, D2s, D2s, p2);
+  FMMOE_CUDA_TRY(cudaGetLastError());
+  h->launches += 2;
+  return FMMOE_OK;
+}
+
+}  // namespace fmmoe

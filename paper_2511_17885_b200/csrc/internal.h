@@ -1,0 +1,101 @@
+// Internal declarations shared by the library's translation units (host side).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/fmmoe.h"
+
+struct fmmoe_handle {
+  int device;
+  int sm_count;
+  int max_smem_optin;
+  int* d_status;        // device status word (0 = ok)
+  int* h_status;        // pinned host mirror
+  int64_t launches;     // kernels launched through this handle
+  void* encode_tiled;   // cuTensorMapEncodeTiled entry point
+};
+
+namespace fmmoe {
+
+// Device-side status codes written to the status word (first writer wins).
+enum : int { DEV_OK = 0, DEV_TIMEOUT = FMMOE_ERR_TIMEOUT, DEV_INTERNAL = FMMOE_ERR_INTERNAL };
+
+constexpr int TC_BLOCK_M = 128;   // token rows per tile on the tensor-core path
+constexpr int F32_BLOCK_M = 32;   // token rows per tile on the fp32 FMA path
+
+// One M-tile of the expert-grouped row space.
+struct MTile {
+  int32_t group;  // expert id
+  int32_t row0;   // first row (in the grouped order)
+  int32_t rows;   // valid rows in this tile (1..block_m)
+  int32_t pad;
+};
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Workspace layout of fmmoe_route / fmmoe_moe_forward (byte offsets).
+struct WsPlan {
+  size_t zero_off, zero_bytes;  // region cleared at the start of every call
+  size_t counts_off;            // int32 [FMMOE_MAX_EXPERTS] expert histogram
+  size_t misc_off;              // int32 [8]: [0] number of routed M-tiles
+  size_t acc_off;               // fp32 [T,H] combine accumulator (atomic mode)
+  size_t topk_idx_off, topk_w_off, inv_row_off;
+  size_t expert_off_off, row_token_off, row_gate_off, mtiles_off;
+  size_t xp_off;                // dtype [P_max,H] rows gathered by expert (bf16 path)
+  size_t act_off;               // dtype [P_max,I] SwiGLU activations
+  size_t act_sh_off;            // dtype [N_s*T,I_s]
+  size_t y_off;                 // fp32 [P_max,H]    (deterministic mode)
+  size_t ysh_off;               // fp32 [N_s*T,H]    (deterministic mode)
+  size_t total;
+  int64_t p_max;
+  int32_t max_mtiles;
+};
+bool plan_workspace(const fmmoe_layer_desc& d, int64_t T, uint32_t flags, WsPlan* p);
+
+#define FMMOE_CUDA_TRY(expr)                         \
+  do {                                               \
+    cudaError_t _e = (expr);                         \
+    if (_e != cudaSuccess) return FMMOE_ERR_CUDA;    \
+  } while (0)
+
+// ---- launchers (each returns after enqueueing; *launches is incremented per kernel) ----
+struct RouteArgs {
+  const void* x; const void* router_w; const float* router_b; const uint8_t* is_visual;
+  int64_t T; int H, E, K, Kv; int reduce_on; int dtype;
+  float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row; int32_t* counts;
+};
+fmmoe_status launch_route(fmmoe_handle* h, const RouteArgs& a, cudaStream_t s);
+
+struct PermuteArgs {
+  const int32_t* topk_idx; const float* topk_w; const int32_t* counts;
+  int64_t T; int K, E; int block_m;
+  int32_t* expert_off; int32_t* row_token; float* row_gate; int32_t* inv_row;
+  MTile* mtiles; int32_t* n_mtiles;
+};
+fmmoe_status launch_permute(fmmoe_handle* h, const PermuteArgs& a, cudaStream_t s);
+fmmoe_status launch_gather_rows(fmmoe_handle* h, const void* x, const int32_t* row_token, const int32_t* expert_off,
+                                int E, int64_t p_max, int H, int elem_bytes, void* xp, cudaStream_t s);
+
+struct FfnArgs {   // both paths
+  const fmmoe_layer_desc* d; const fmmoe_weights* w;
+  const void* x; int64_t T; int64_t p_max;
+  const MTile* mtiles; const int32_t* n_mtiles; int32_t max_mtiles;
+  const int32_t* row_token; const float* row_gate;
+  void* xp; void* act; void* act_sh;
+  float* acc;            // atomic mode
+  float* y; float* ysh;  // deterministic mode
+  int deterministic;
+  int* d_status;
+};
+fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05
+fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);   // fp32 FMA
+
+struct FinalizeArgs {
+  const void* x; void* out; int64_t T; int H, K, n_shared; int dtype; int add_residual; int deterministic;
+  const float* acc; const float* y; const float* ysh; const int32_t* inv_row; const float* topk_w;
+};
+fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_t s);
+
+}  // namespace fmmoe

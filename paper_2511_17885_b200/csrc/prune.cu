@@ -1,0 +1,559 @@
+// Routing-aware sliding-window pruning of vision tokens (Section 3.2).
+//   vis_index_kernel   : rank of every vision token inside its sequence (scan of the mask)
+//   window_score_kernel: per window, routing similarity S (Eq. 8 or Eq. 9-10) and the
+//                        attention sum (Eq. 11); one warp per window, fp64 accumulation
+//   select_kernel      : per sequence, A_bar (Eq. 12), C (Eq. 13) rounded once to fp32,
+//                        merge set = m highest C (Eq. 15), drop set = d smallest A_bar among
+//                        the rest, then the stable compaction map (scan of keep flags)
+//   compact_kernel     : copies kept rows; a merged window becomes mean(rows) rescaled to the
+//                        largest member norm (Eq. 16-18) at its first token's position
+// Ranks are computed by counting, on (value, index) pairs, so the keep-set does not depend
+// on thread order; ties go to the lower window index.
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "internal.h"
+
+namespace fmmoe {
+
+constexpr int MAXS = FMMOE_MAX_SEQS_PER_LAUNCH;
+constexpr int MAXW = FMMOE_MAX_WINDOW;
+
+struct PruneSeqs {
+  int n_seq;
+  int n_vis[MAXS], m[MAXS], d[MAXS];
+  int win_off[MAXS + 1];          // first window of each sequence in this launch
+  long long seq_off[MAXS + 1];    // token offsets
+  long long out_off[MAXS + 1];    // output row offsets
+};
+
+struct PruneDev {
+  const float* probs; const float* attn; const void* x; const uint8_t* is_visual;
+  int E, H, W, sim_mode, merge_mode, dtype;
+  double alpha;
+  // workspace
+  int32_t* vrank;      // [T] rank of a vision token inside its sequence, -1 for text
+  int32_t* vis_list;   // [T] token index of the v-th vision token of sequence b at seq_off[b]+v
+  double* sim;         // [windows]
+  double* asum;        // [windows]
+  uint8_t* action;     // [windows] 0 keep, 1 merge, 2 drop
+  // outputs
+  void* x_out; uint8_t* is_visual_out; int32_t* keep_idx; uint8_t* kind;
+  int32_t* keep_idx_ws; uint8_t* kind_ws;   // always-present copies in the workspace
+  int* status;
+};
+
+// ------------------------------------------------------------------ vision ranks
+__global__ void __launch_bounds__(1024) vis_index_kernel(const PruneDev a, const PruneSeqs sq) {
+  __shared__ int s_warp[32];
+  __shared__ int s_running;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long lo = sq.seq_off[b], hi = sq.seq_off[b + 1];
+  if (tid == 0) s_running = 0;
+  __syncthreads();
+  for (long long t0 = lo; t0 < hi; t0 += 1024) {
+    const long long t = t0 + tid;
+    const bool v = t < hi && a.is_visual[t] != 0;
+    const unsigned bal = __ballot_sync(0xffffffffu, v);
+    if (lane == 0) s_warp[warp] = __popc(bal);
+    __syncthreads();
+    if (warp == 0) {
+      int c = s_warp[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, c, o);
+        if (lane >= o) c += n;
+      }
+      s_warp[lane] = c;
+    }
+    __syncthreads();
+    const int running = s_running;
+    if (t < hi) {
+      int rank = -1;
+      if (v) {
+        rank = running + (warp ? s_warp[warp - 1] : 0) + __popc(bal & ((1u << lane) - 1u));
+        a.vis_list[lo + rank] = (int32_t)t;
+      }
+      a.vrank[t] = rank;
+    }
+    __syncthreads();
+    if (tid == 0) s_running = running + s_warp[31];
+    __syncthreads();
+  }
+  if (tid == 0 && s_running != sq.n_vis[b]) atomicCAS(a.status, 0, DEV_INTERNAL);
+}
+
+// ------------------------------------------------------------------ window scores
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+template <int W>
+__device__ __forceinline__ void score_window(const PruneDev& a, const int32_t* members, int lane, double* sim_out,
+                                             double* asum_out) {
+  // dots[i][j] for j <= i (norms on the diagonal), partial over this lane's experts
+  double dots[W * (W + 1) / 2];
+#pragma unroll
+  for (int i = 0; i < W * (W + 1) / 2; ++i) dots[i] = 0.0;
+  const float* rows[W];
+#pragma unroll
+  for (int i = 0; i < W; ++i) rows[i] = a.probs + (long long)members[i] * a.E;
+  for (int e = lane; e < a.E; e += 32) {
+    double v[W];
+#pragma unroll
+    for (int i = 0; i < W; ++i) v[i] = (double)rows[i][e];
+    int q = 0;
+#pragma unroll
+    for (int i = 0; i < W; ++i)
+#pragma unroll
+      for (int j = 0; j <= i; ++j) { dots[q] = fma(v[i], v[j], dots[q]); ++q; }
+  }
+#pragma unroll
+  for (int i = 0; i < W * (W + 1) / 2; ++i) dots[i] = warp_sum_d(dots[i]);
+  // every lane now holds the full dot products
+  auto D = [&](int i, int j) { return dots[i * (i + 1) / 2 + j]; };   // j <= i
+  double s = 0.0;
+  if (a.sim_mode == 0) {
+#pragma unroll
+    for (int i = 0; i < W; ++i)
+#pragma unroll
+      for (int j = 0; j < i; ++j) s += D(i, j) / (sqrt(D(i, i)) * sqrt(D(j, j)));
+    s = s / (double)(W * (W - 1) / 2);
+  } else {
+    // mean row rbar = sum(rows)/W:  rows_i . rbar = sum_j D(i,j)/W ;  rbar . rbar = sum_ij D(i,j)/W^2
+    double rr = 0.0;
+    double rd[W];
+#pragma unroll
+    for (int i = 0; i < W; ++i) {
+      double t = 0.0;
+#pragma unroll
+      for (int j = 0; j < W; ++j) t += (j <= i) ? D(i, j) : D(j, i);
+      rd[i] = t / (double)W;
+      rr += t;
+    }
+    rr = rr / (double)(W * W);
+#pragma unroll
+    for (int i = 0; i < W; ++i) s += rd[i] / (sqrt(D(i, i)) * sqrt(rr));
+    s = s / (double)W;
+  }
+  double asum = 0.0;
+  if (a.attn) {
+#pragma unroll
+    for (int i = 0; i < W; ++i) asum += (double)a.attn[members[i]];
+  }
+  if (lane == 0) { *sim_out = s; *asum_out = asum; }
+}
+
+__global__ void __launch_bounds__(256) window_score_kernel(const PruneDev a, const PruneSeqs sq) {
+  const int lane = threadIdx.x & 31;
+  const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (gw >= sq.win_off[sq.n_seq]) return;
+  int b = 0;
+  while (b + 1 < sq.n_seq && gw >= sq.win_off[b + 1]) ++b;
+  const int i = gw - sq.win_off[b];
+  int32_t members[MAXW];
+#pragma unroll
+  for (int k = 0; k < MAXW; ++k)
+    members[k] = k < a.W ? a.vis_list[sq.seq_off[b] + (long long)i * a.W + k] : 0;
+  switch (a.W) {
+    case 2: score_window<2>(a, members, lane, a.sim + gw, a.asum + gw); break;
+    case 3: score_window<3>(a, members, lane, a.sim + gw, a.asum + gw); break;
+    case 4: score_window<4>(a, members, lane, a.sim + gw, a.asum + gw); break;
+    case 5: score_window<5>(a, members, lane, a.sim + gw, a.asum + gw); break;
+    case 6: score_window<6>(a, members, lane, a.sim + gw, a.asum + gw); break;
+    case 7: score_window<7>(a, members, lane, a.sim + gw, a.asum + gw); break;
+    case 8: score_window<8>(a, members, lane, a.sim + gw, a.asum + gw); break;
+    default: break;
+  }
+}
+
+// ------------------------------------------------------------------ select + compaction map
+__global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const PruneSeqs sq) {
+  extern __shared__ float s_f[];   // C32[n_f], A32[n_f]
+  __shared__ double s_red[32];
+  __shared__ int s_warp[32];
+  __shared__ int s_running;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_f = sq.n_vis[b] / a.W;
+  const int w0 = sq.win_off[b];
+  const int m = sq.m[b], d = sq.d[b];
+  float* C32 = s_f;
+  float* A32 = s_f + n_f;
+  const bool have_attn = a.attn != nullptr;
+
+  // Eq. 12: divide by the largest window sum (0 if all sums are 0)
+  double amax = 0.0;
+  if (have_attn) {
+    for (int i = tid; i < n_f; i += 1024) amax = fmax(amax, a.asum[w0 + i]);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) amax = fmax(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if (lane == 0) s_red[warp] = amax;
+    __syncthreads();
+    amax = s_red[0];
+    for (int i = 1; i < 32; ++i) amax = fmax(amax, s_red[i]);
+  }
+  for (int i = tid; i < n_f; i += 1024) {
+    const double S = a.sim[w0 + i];
+    if (have_attn) {
+      const double ab = amax > 0.0 ? a.asum[w0 + i] / amax : 0.0;
+      // Eq. 13 in fp64 without contraction, then ONE rounding to fp32
+      const double c = __dsub_rn(__dmul_rn(a.alpha, S), __dmul_rn(__dsub_rn(1.0, a.alpha), ab));
+      C32[i] = (float)c;
+      A32[i] = (float)ab;
+    } else {
+      C32[i] = (float)S;
+      A32[i] = 0.f;
+    }
+  }
+  __syncthreads();
+  // ranks by counting
+  for (int i = tid; i < n_f; i += 1024) {
+    const float ci = C32[i];
+    int rc = 0;
+    for (int j = 0; j < n_f; ++j) {
+      const float cj = C32[j];
+      rc += (cj > ci) || (cj == ci && j < i);
+    }
+    uint8_t act = 0;
+    if (rc < m) act = 1;
+    else if (!have_attn && rc < m + d) act = 2;
+    a.action[w0 + i] = act;
+  }
+  if (have_attn && d > 0) {
+    __syncthreads();
+    for (int i = tid; i < n_f; i += 1024) {
+      if (a.action[w0 + i] == 1) continue;
+      const float ai = A32[i];
+      int ra = 0;
+      for (int j = 0; j < n_f; ++j) {
+        if (a.action[w0 + j] == 1) continue;
+        const float aj = A32[j];
+        ra += (aj < ai) || (aj == ai && j < i);
+      }
+      if (ra < d) a.action[w0 + i] = 2;   // concurrent readers only test for "== 1"
+    }
+  }
+  __syncthreads();
+
+  // stable compaction map over the sequence's tokens
+  const long long lo = sq.seq_off[b], hi = sq.seq_off[b + 1];
+  if (tid == 0) s_running = 0;
+  __syncthreads();
+  for (long long t0 = lo; t0 < hi; t0 += 1024) {
+    const long long t = t0 + tid;
+    int kd = -1;   // kind of the emitted row, -1 = nothing emitted
+    if (t < hi) {
+      const int v = a.vrank[t];
+      if (v < 0) kd = 0;
+      else {
+        const int w = v / a.W;
+        if (w >= n_f) kd = 1;
+        else {
+          const uint8_t act = a.action[w0 + w];
+          if (act == 0) kd = 1;
+          else if (act == 1 && v - w * a.W == 0) kd = 2;
+        }
+      }
+    }
+    const unsigned bal = __ballot_sync(0xffffffffu, kd >= 0);
+    if (lane == 0) s_warp[warp] = __popc(bal);
+    __syncthreads();
+    if (warp == 0) {
+      int c = s_warp[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, c, o);
+        if (lane >= o) c += n;
+      }
+      s_warp[lane] = c;
+    }
+    __syncthreads();
+    const int running = s_running;
+    if (kd >= 0) {
+      const long long pos = sq.out_off[b] + running + (warp ? s_warp[warp - 1] : 0) + __popc(bal & ((1u << lane) - 1u));
+      if (pos < sq.out_off[b + 1]) {
+        a.keep_idx_ws[pos] = (int32_t)t;
+        a.kind_ws[pos] = (uint8_t)kd;
+        if (a.keep_idx) a.keep_idx[pos] = (int32_t)t;
+        if (a.kind) a.kind[pos] = (uint8_t)kd;
+        if (a.is_visual_out) a.is_visual_out[pos] = kd != 0;
+      }
+    }
+    __syncthreads();
+    if (tid == 0) s_running = running + s_warp[31];
+    __syncthreads();
+  }
+  if (tid == 0 && s_running != (int)(sq.out_off[b + 1] - sq.out_off[b])) atomicCAS(a.status, 0, DEV_INTERNAL);
+}
+
+// ------------------------------------------------------------------ gather / merge rows
+template <typename T> struct Row8;   // 8 elements (bf16) or 4 elements (fp32) per 16 bytes
+template <> struct Row8<__nv_bfloat16> {
+  static constexpr int N = 8;
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float* f) {
+    const uint4 u = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+      f[2 * i] = v.x; f[2 * i + 1] = v.y;
+    }
+  }
+  static __device__ __forceinline__ void store(__nv_bfloat16* p, const float* f) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      w[i] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+template <> struct Row8<float> {
+  static constexpr int N = 4;
+  static __device__ __forceinline__ void load(const float* p, float* f) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+  }
+  static __device__ __forceinline__ void store(float* p, const float* f) {
+    *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+  }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const PruneSeqs sq, long long row_base, long long n_rows) {
+  constexpr int N = Row8<T>::N;
+  __shared__ float s_red[8][MAXW + 1];
+  __shared__ float s_scale;
+  const long long row = row_base + blockIdx.x;
+  if (blockIdx.x >= n_rows) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const T* X = static_cast<const T*>(a.x);
+  T* O = static_cast<T*>(a.x_out) + row * a.H;
+  const long long t0 = a.keep_idx_ws[row];
+  const int kd = a.kind_ws[row];
+  if (kd != 2) {
+    const uint4* src = reinterpret_cast<const uint4*>(X + t0 * a.H);
+    uint4* dst = reinterpret_cast<uint4*>(O);
+    for (int i = tid; i < a.H / N; i += 256) dst[i] = src[i];
+    return;
+  }
+  int b = 0;
+  while (b + 1 < sq.n_seq && row >= sq.out_off[b + 1]) ++b;
+  const int v0 = a.vrank[t0];
+  long long mem[MAXW];
+#pragma unroll
+  for (int k = 0; k < MAXW; ++k) mem[k] = k < a.W ? a.vis_list[sq.seq_off[b] + v0 + k] : 0;
+  const float invW = 1.f / (float)a.W;
+  // pass 1: squared norms of the members and of the mean
+  float part[MAXW + 1];
+#pragma unroll
+  for (int k = 0; k <= MAXW; ++k) part[k] = 0.f;
+  for (int i = tid; i < a.H / N; i += 256) {
+    float mean[N];
+#pragma unroll
+    for (int j = 0; j < N; ++j) mean[j] = 0.f;
+#pragma unroll
+    for (int k = 0; k < MAXW; ++k) {
+      if (k < a.W) {
+        float f[N];
+        Row8<T>::load(X + mem[k] * a.H + i * N, f);
+#pragma unroll
+        for (int j = 0; j < N; ++j) { part[k] = fmaf(f[j], f[j], part[k]); mean[j] += f[j]; }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < N; ++j) { const float mv = mean[j] * invW; part[MAXW] = fmaf(mv, mv, part[MAXW]); }
+  }
+#pragma unroll
+  for (int k = 0; k <= MAXW; ++k) {
+    float v = part[k];
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == 0) s_red[warp][k] = v;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    float tot[MAXW + 1];
+    for (int k = 0; k <= MAXW; ++k) { tot[k] = 0.f; for (int w = 0; w < 8; ++w) tot[k] += s_red[w][k]; }
+    float nmax = 0.f;
+    for (int k = 0; k < a.W; ++k) nmax = fmaxf(nmax, sqrtf(tot[k]));
+    const float nb = sqrtf(tot[MAXW]);
+    s_scale = a.merge_mode == 1 ? 1.f : (nb > 0.f ? nmax / nb : 0.f);   // Eq. 18
+  }
+  __syncthreads();
+  const float scale = s_scale * invW;
+  for (int i = tid; i < a.H / N; i += 256) {
+    float mean[N];
+#pragma unroll
+    for (int j = 0; j < N; ++j) mean[j] = 0.f;
+#pragma unroll
+    for (int k = 0; k < MAXW; ++k) {
+      if (k < a.W) {
+        float f[N];
+        Row8<T>::load(X + mem[k] * a.H + i * N, f);
+#pragma unroll
+        for (int j = 0; j < N; ++j) mean[j] += f[j];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < N; ++j) mean[j] *= scale;
+    Row8<T>::store(O + i * N, mean);
+  }
+}
+
+static int64_t counts_for(int64_t n_vis, int64_t n_retain, const fmmoe_prune_params* p, int64_t* m_out, int64_t* d_out) {
+  const int64_t W = p->window;
+  const int64_t eps = n_vis - n_retain;
+  const int64_t n_f = n_vis / W;
+  int64_t m = 0, d = 0;
+  if (!(n_retain >= n_vis || eps <= W)) {
+    if (p->merge_mode != 2) {
+      m = (int64_t)floor((double)n_retain * p->gamma + 1e-9);
+      if (m > eps / (W - 1)) m = eps / (W - 1);
+      if (m > n_f) m = n_f;
+      if (m < 0) m = 0;
+    }
+    const int64_t u = eps - m * (W - 1);
+    d = u / W;
+    if (d > n_f - m) d = n_f - m;
+  }
+  if (m_out) *m_out = m;
+  if (d_out) *d_out = d;
+  return n_vis - m * (W - 1) - d * W;
+}
+
+}  // namespace fmmoe
+
+using namespace fmmoe;
+
+static bool prune_params_ok(const fmmoe_prune_params* p) {
+  return p && p->window >= 2 && p->window <= FMMOE_MAX_WINDOW && p->sim_mode >= 0 && p->sim_mode <= 1 &&
+         p->merge_mode >= 0 && p->merge_mode <= 2 && p->alpha >= 0.0 && p->alpha <= 1.0 && p->gamma >= 0.0;
+}
+
+extern "C" __attribute__((visibility("default"))) int64_t fmmoe_prune_kept_count(int64_t n_vis, int64_t n_retain, const fmmoe_prune_params* p,
+                                          int64_t* n_merge, int64_t* n_drop) {
+  if (!prune_params_ok(p) || n_vis < 0 || n_retain < 0) return -1;
+  return counts_for(n_vis, n_retain, p, n_merge, n_drop);
+}
+
+namespace {
+struct PruneWs { size_t vrank, vis_list, sim, asum, action, keep_idx, kind, total; };
+PruneWs plan_prune(int64_t T) {
+  PruneWs w; size_t o = 0;
+  const size_t nw = (size_t)T / 2 + 1;
+  w.vrank = o; o = align_up(o + (size_t)T * 4, 256);
+  w.vis_list = o; o = align_up(o + (size_t)T * 4, 256);
+  w.sim = o; o = align_up(o + nw * 8, 256);
+  w.asum = o; o = align_up(o + nw * 8, 256);
+  w.action = o; o = align_up(o + nw, 256);
+  w.keep_idx = o; o = align_up(o + (size_t)T * 4, 256);
+  w.kind = o; o = align_up(o + (size_t)T, 256);
+  w.total = o;
+  return w;
+}
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) size_t fmmoe_prune_workspace_bytes(int64_t n_tokens, int32_t n_seq) {
+  (void)n_seq;
+  if (n_tokens < 0) return 0;
+  return plan_prune(n_tokens).total + 256;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visual(fmmoe_handle* h, const fmmoe_prune_params* p, const float* probs,
+                                           int32_t n_experts, const float* attn, const void* x, int32_t dtype,
+                                           int32_t hidden, const uint8_t* is_visual, const int64_t* seq_off,
+                                           const int64_t* n_vis, const int64_t* n_retain, int32_t n_seq, void* x_out,
+                                           uint8_t* is_visual_out, int32_t* keep_idx, uint8_t* kind,
+                                           int64_t* out_seq_off, void* workspace, size_t workspace_bytes,
+                                           void* cuda_stream) {
+  if (!h || !prune_params_ok(p) || !seq_off || !n_vis || !n_retain || !out_seq_off || n_seq < 0)
+    return FMMOE_ERR_INVALID_ARG;
+  if (n_experts < 1 || hidden < 1 || (dtype != FMMOE_F32 && dtype != FMMOE_BF16)) return FMMOE_ERR_INVALID_ARG;
+  const int elem = dtype == FMMOE_BF16 ? 2 : 4;
+  if ((hidden * elem) % 16 != 0) return FMMOE_ERR_UNSUPPORTED;
+  int64_t max_nf = 0;
+  out_seq_off[0] = 0;
+  for (int b = 0; b < n_seq; ++b) {
+    const int64_t L = seq_off[b + 1] - seq_off[b];
+    if (L < 0 || n_vis[b] < 0 || n_vis[b] > L || n_retain[b] < 0) return FMMOE_ERR_INVALID_ARG;
+    const int64_t kept = counts_for(n_vis[b], n_retain[b], p, nullptr, nullptr);
+    out_seq_off[b + 1] = out_seq_off[b] + (L - n_vis[b]) + kept;
+    if (n_vis[b] / p->window > max_nf) max_nf = n_vis[b] / p->window;
+  }
+  const int64_t T = n_seq ? seq_off[n_seq] : 0;
+  if (n_seq && seq_off[0] != 0) return FMMOE_ERR_INVALID_ARG;
+  if (T > 0x7fffffff) return FMMOE_ERR_UNSUPPORTED;
+  if (T == 0) return FMMOE_OK;
+  if (!probs || !x || !is_visual || !x_out) return FMMOE_ERR_INVALID_ARG;
+  if (x == x_out) return FMMOE_ERR_INVALID_ARG;
+  if (((uintptr_t)x | (uintptr_t)x_out | (uintptr_t)probs) & 15) return FMMOE_ERR_INVALID_ARG;
+  const PruneWs wp = plan_prune(T);
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < wp.total) return FMMOE_ERR_WORKSPACE;
+  const size_t sel_smem = (size_t)max_nf * 8;
+  if (sel_smem > (size_t)h->max_smem_optin - 1024) return FMMOE_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+
+  PruneDev a = {};
+  a.probs = probs; a.attn = attn; a.x = x; a.is_visual = is_visual;
+  a.E = n_experts; a.H = hidden; a.W = p->window; a.sim_mode = p->sim_mode; a.merge_mode = p->merge_mode;
+  a.dtype = dtype; a.alpha = p->alpha;
+  a.vrank = reinterpret_cast<int32_t*>(ws + wp.vrank); a.vis_list = reinterpret_cast<int32_t*>(ws + wp.vis_list);
+  a.sim = reinterpret_cast<double*>(ws + wp.sim); a.asum = reinterpret_cast<double*>(ws + wp.asum);
+  a.action = reinterpret_cast<uint8_t*>(ws + wp.action);
+  a.keep_idx_ws = reinterpret_cast<int32_t*>(ws + wp.keep_idx); a.kind_ws = reinterpret_cast<uint8_t*>(ws + wp.kind);
+  a.x_out = x_out; a.is_visual_out = is_visual_out; a.keep_idx = keep_idx; a.kind = kind;
+  a.status = h->d_status;
+
+  if (sel_smem > 48 * 1024)
+    FMMOE_CUDA_TRY(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_smem));
+
+  int win_base = 0;
+  for (int b0 = 0; b0 < n_seq; b0 += MAXS) {
+    const int nb = n_seq - b0 < MAXS ? n_seq - b0 : MAXS;
+    PruneSeqs sq = {};
+    sq.n_seq = nb;
+    sq.win_off[0] = win_base;
+    for (int i = 0; i < nb; ++i) {
+      const int b = b0 + i;
+      int64_t m, d;
+      counts_for(n_vis[b], n_retain[b], p, &m, &d);
+      sq.n_vis[i] = (int)n_vis[b]; sq.m[i] = (int)m; sq.d[i] = (int)d;
+      sq.win_off[i + 1] = sq.win_off[i] + (int)(n_vis[b] / p->window);
+      sq.seq_off[i] = seq_off[b]; sq.out_off[i] = out_seq_off[b];
+    }
+    sq.seq_off[nb] = seq_off[b0 + nb]; sq.out_off[nb] = out_seq_off[b0 + nb];
+    const int n_win = sq.win_off[nb] - win_base;
+    // window ids inside a launch are relative to the launch's first window
+    PruneSeqs rel = sq;
+    for (int i = 0; i <= nb; ++i) rel.win_off[i] -= win_base;
+    PruneDev al = a;
+    al.sim = a.sim + win_base; al.asum = a.asum + win_base; al.action = a.action + win_base;
+    vis_index_kernel<<<nb, 1024, 0, s>>>(al, rel);
+    FMMOE_CUDA_TRY(cudaGetLastError());
+    h->launches += 1;
+    if (n_win > 0) {
+      window_score_kernel<<<(n_win + 7) / 8, 256, 0, s>>>(al, rel);
+      FMMOE_CUDA_TRY(cudaGetLastError());
+      h->launches += 1;
+    }
+    select_kernel<<<nb, 1024, sel_smem, s>>>(al, rel);
+    FMMOE_CUDA_TRY(cudaGetLastError());
+    h->launches += 1;
+    const long long rows = rel.out_off[nb] - rel.out_off[0];
+    if (rows > 0) {
+      if (dtype == FMMOE_BF16)
+        compact_kernel<__nv_bfloat16><<<(unsigned)rows, 256, 0, s>>>(al, rel, rel.out_off[0], rows);
+      else
+        compact_kernel<float><<<(unsigned)rows, 256, 0, s>>>(al, rel, rel.out_off[0], rows);
+      FMMOE_CUDA_TRY(cudaGetLastError());
+      h->launches += 1;
+    }
+    win_base += n_win;
+  }
+  return FMMOE_OK;
+}

@@ -1,0 +1,149 @@
+"""GPU parity: the whole MoE layer (Eq. 1-5) through the C ABI against the CPU oracle.
+Tolerances: fp32 layers 1e-4, bf16 layers 2e-2, both as max over token rows of
+|y - ref|_inf / |ref|_inf.  The oracle is teacher-forced on the kernel's fp32 logits for
+the (integer) selection, so a near-tie cannot turn into a large output difference."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fmmoe_oracle as O
+from paper_2511_17885_b200 import binding as B
+from paper_2511_17885_b200 import inputs as I
+from gpu_util import dev, handle, host, row_rel_err, upload_weights, TDT
+
+pytestmark = pytest.mark.gpu
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+
+
+def random_layer(r, dtype, H, E, I_, Ns, Is, std=0.05):
+    def d(shape):
+        return I.round_to_storage(std * r.standard_normal(shape), dtype)
+    w = {"router_w": d((E, H)), "router_b": None, "w_gate": d((E, I_, H)), "w_up": d((E, I_, H)),
+         "w_down": d((E, H, I_)), "ws_gate": None, "ws_up": None, "ws_down": None}
+    if Ns:
+        w["ws_gate"] = d((Ns, Is, H)); w["ws_up"] = d((Ns, Is, H)); w["ws_down"] = d((Ns, H, Is))
+    return w
+
+
+def run_layer(dtype, x, mask, w, K, Kv, flags, Ns=0, Is=0):
+    td = TDT[dtype]
+    T, H = x.shape
+    E, I_ = w["w_gate"].shape[0], w["w_gate"].shape[1]
+    desc = B.make_desc(H, E, I_, Ns, Is, K, Kv, td)
+    wd = upload_weights(w, dtype)
+    ws = B.make_weights(wd)
+    route = {"logits": torch.empty(T, E, dtype=torch.float32, device="cuda"),
+             "topk_idx": torch.empty(T, K, dtype=torch.int32, device="cuda"),
+             "topk_w": torch.empty(T, K, dtype=torch.float32, device="cuda")}
+    out = handle().fmmoe_moe_forward(desc, ws, dev(x, td), dev(mask), flags, route=route)
+    handle().check_status()
+    return host(out), {k: host(v) for k, v in route.items()}
+
+
+def check_layer(dtype, T, H, E, I_, K, Kv, Ns=0, Is=0, flags=B.FLAG_REDUCE_ON, seed=0, mask=None, bias=False):
+    r = np.random.default_rng(seed)
+    x = I.round_to_storage(r.standard_normal((T, H)), dtype)
+    mask = (r.random(T) < 0.7).astype(np.uint8) if mask is None else mask
+    w = random_layer(r, dtype, H, E, I_, Ns, Is)
+    if bias:
+        w["router_b"] = (0.7 * r.standard_normal(E)).astype(np.float32)
+    y, route = run_layer(dtype, x, mask, w, K, Kv, flags, Ns, Is)
+    ref = O.moe_forward(x, mask, w, K, Kv, bool(flags & B.FLAG_REDUCE_ON), bool(flags & B.FLAG_RESIDUAL),
+                        logits32=route["logits"])
+    assert np.array_equal(route["topk_idx"], ref["topk_idx"])
+    err = row_rel_err(y, ref["out"])
+    assert err < TOL[dtype], f"row-relative error {err}"
+    return y, ref
+
+
+SMALL = [
+    # dtype, T, H, E, I, K, Kv, Ns, Is
+    ("f32", 256, 256, 8, 512, 2, 1, 0, 0),
+    ("f32", 70, 64, 5, 36, 3, 1, 1, 20),
+    ("bf16", 300, 128, 8, 128, 2, 1, 0, 0),
+    ("bf16", 1000, 256, 16, 192, 4, 2, 2, 192),
+    ("bf16", 515, 512, 40, 320, 6, 3, 1, 128),
+    ("bf16", 129, 64, 4, 64, 2, 0, 1, 64),
+]
+
+
+@pytest.mark.parametrize("case", SMALL)
+@pytest.mark.parametrize("det", [0, B.FLAG_DETERMINISTIC])
+def test_layer_small(case, det):
+    dtype, T, H, E, I_, K, Kv, Ns, Is = case
+    check_layer(dtype, T, H, E, I_, K, Kv, Ns, Is, flags=B.FLAG_REDUCE_ON | det)
+
+
+def test_layer_residual_and_reduce_off():
+    check_layer("bf16", 200, 128, 8, 128, 3, 1, flags=B.FLAG_REDUCE_ON | B.FLAG_RESIDUAL)
+    check_layer("bf16", 200, 128, 8, 128, 3, 1, flags=0)
+    check_layer("f32", 90, 64, 6, 64, 2, 1, flags=B.FLAG_RESIDUAL)
+
+
+def test_layer_edge_masks_and_empty_experts():
+    T = 260
+    check_layer("bf16", T, 128, 8, 128, 2, 1, mask=np.ones(T, np.uint8))
+    check_layer("bf16", T, 128, 8, 128, 2, 1, mask=np.zeros(T, np.uint8))
+    # a strong bias empties several experts and overloads others (multi-tile groups)
+    r = np.random.default_rng(3)
+    x = I.round_to_storage(r.standard_normal((T, 128)), "bf16")
+    w = random_layer(r, "bf16", 128, 16, 128, 0, 0)
+    w["router_b"] = np.array([8, 8, 8] + [-30] * 13, np.float32)
+    mask = (r.random(T) < 0.5).astype(np.uint8)
+    y, route = run_layer("bf16", x, mask, w, 3, 1, B.FLAG_REDUCE_ON)
+    ref = O.moe_forward(x, mask, w, 3, 1, True, logits32=route["logits"])
+    assert set(np.unique(route["topk_idx"][route["topk_idx"] >= 0]).tolist()) <= {0, 1, 2}
+    assert row_rel_err(y, ref["out"]) < 2e-2
+
+
+def test_layer_kv_equals_k_reproduces_dense():
+    r = np.random.default_rng(4)
+    T, H, E, I_ = 150, 128, 8, 128
+    x = I.round_to_storage(r.standard_normal((T, H)), "bf16")
+    mask = (r.random(T) < 0.6).astype(np.uint8)
+    w = random_layer(r, "bf16", H, E, I_, 0, 0)
+    a, _ = run_layer("bf16", x, mask, w, 3, 3, B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC)
+    b, _ = run_layer("bf16", x, mask, w, 3, 1, B.FLAG_DETERMINISTIC)      # reduce off: K for everyone
+    assert np.array_equal(a, b)
+
+
+def test_layer_deterministic_mode_is_reproducible():
+    r = np.random.default_rng(6)
+    T, H, E, I_ = 400, 256, 16, 128
+    x = I.round_to_storage(r.standard_normal((T, H)), "bf16")
+    mask = (r.random(T) < 0.6).astype(np.uint8)
+    w = random_layer(r, "bf16", H, E, I_, 1, 128)
+    a, _ = run_layer("bf16", x, mask, w, 4, 2, B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC, 1, 128)
+    b, _ = run_layer("bf16", x, mask, w, 4, 2, B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC, 1, 128)
+    assert np.array_equal(a, b)
+
+
+def test_layer_c0_full_config():
+    cfg = I.C0
+    x, m, _, _ = I.make_tokens(cfg)
+    w = I.make_weights(cfg)
+    y, route = run_layer("f32", x, m, w, cfg.top_k, cfg.top_k_vis, B.FLAG_REDUCE_ON)
+    ref = O.moe_forward(x, m, w, cfg.top_k, cfg.top_k_vis, True, logits32=route["logits"])
+    assert np.array_equal(route["topk_idx"], ref["topk_idx"])
+    assert row_rel_err(y, ref["out"]) < 1e-4
+    assert int((ref["topk_idx"] >= 0).sum()) == 224 * 1 + 32 * 2
+
+
+def test_forward_host_variant_and_empty():
+    r = np.random.default_rng(7)
+    T, H, E, I_ = 200, 128, 8, 128
+    x = I.round_to_storage(r.standard_normal((T, H)), "bf16")
+    mask = (r.random(T) < 0.6).astype(np.uint8)
+    w = random_layer(r, "bf16", H, E, I_, 0, 0)
+    desc = B.make_desc(H, E, I_, 0, 0, 2, 1, torch.bfloat16)
+    wd = upload_weights(w, "bf16"); ws = B.make_weights(wd)
+    xh = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    mh = torch.from_numpy(mask).pin_memory()
+    oh = torch.empty_like(xh).pin_memory()
+    handle().fmmoe_moe_forward_host(desc, ws, xh, mh, B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC, oh)
+    y, _ = run_layer("bf16", x, mask, w, 2, 1, B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC)
+    assert np.array_equal(oh.float().numpy(), y)
+    # T = 0
+    out = handle().fmmoe_moe_forward(desc, ws, torch.zeros(0, H, dtype=torch.bfloat16, device="cuda"),
+                                     torch.zeros(0, dtype=torch.uint8, device="cuda"), 1)
+    assert out.shape == (0, H)
