@@ -488,7 +488,8 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
   if (n_seq && seq_off[0] != 0) return FMMOE_ERR_INVALID_ARG;
   if (T > 0x7fffffff) return FMMOE_ERR_UNSUPPORTED;
   if (T == 0) return FMMOE_OK;
-  if (!probs || !x || !is_visual || !x_out) return FMMOE_ERR_INVALID_ARG;
+  const int64_t T_out = out_seq_off[n_seq];
+  if (!probs || !x || !is_visual || (T_out > 0 && !x_out)) return FMMOE_ERR_INVALID_ARG;
   if (x == x_out) return FMMOE_ERR_INVALID_ARG;
   if (((uintptr_t)x | (uintptr_t)x_out | (uintptr_t)probs) & 15) return FMMOE_ERR_INVALID_ARG;
   const PruneWs wp = plan_prune(T);
