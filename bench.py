@@ -1,0 +1,340 @@
+#!/usr/bin/env python
+"""Benchmark of the FastMMoE MoE-layer hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1] [--impl reference]
+
+One "step" = one pass of the whole hot path over one batch of synthetic tokens:
+router + top-k + gates, permute-by-expert, grouped SwiGLU expert GEMMs + shared
+experts, weighted combine (fmmoe_moe_forward), then routing-aware pruning of the layer
+output with that layer's routing probabilities (fmmoe_prune_visual).
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "MoE-layer prefill tokens/s"
+UNIT = "tokens/s"
+WORKLOADS = ("C0", "C1", "C2", "C2x4", "C3")
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
+# ncu captures summarised under profiles/ (null until a capture for that workload exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "tf_burst": float(d["bf16_tflops"]),
+                "tf_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tf_burst": 1590.0, "tf_sustained": 1400.0, "source": "fallback"}
+
+
+def workload_cfg(name):
+    from paper_2511_17885_b200 import inputs as I
+    cfg = I.CONFIGS[name]
+    # pruning stage of the step: the workload's own 50%-retention setting (C3/C2: the sweep's middle point)
+    prune = None
+    for pc in cfg.prune:
+        if abs(pc.retain - 0.5) < 1e-9:
+            prune = pc
+    if prune is None and cfg.prune:
+        prune = cfg.prune[0]
+    return cfg, prune
+
+
+def describe(name, cfg, prune):
+    return {"workload": f"{name}: {cfg.name}, {cfg.batch} x ({cfg.n_vis} visual + {cfg.n_text} text) tokens, "
+                        f"H={cfg.hidden} E={cfg.n_experts} I={cfg.inter} shared={cfg.n_shared} K={cfg.top_k} "
+                        f"K_v={cfg.top_k_vis} (reduction on); then pruning to {int(prune.retain * 100)}% "
+                        f"(W={prune.window}, gamma={prune.gamma}, attention-free score)",
+            "tokens_per_step": cfg.n_tokens,
+            "l2": "inputs larger than L2: every step streams the layer's expert weights "
+                  f"({weight_bytes(cfg) / 1e6:.0f} MB) from HBM"}
+
+
+def weight_bytes(cfg):
+    e = 2 if cfg.dtype == "bf16" else 4
+    return (3 * cfg.hidden * cfg.inter * cfg.n_experts + 3 * cfg.hidden * cfg.shared_inter * cfg.n_shared
+            + cfg.n_experts * cfg.hidden) * e
+
+
+# ------------------------------------------------------------------ algorithmic work per launch
+def kernel_work(cfg, kernel, P, touched, t_out=None):
+    """(bytes, flops) one launch of `kernel` must move / compute for this workload.
+    P = routed pairs, touched = experts with at least one row."""
+    e = 2 if cfg.dtype == "bf16" else 4
+    T, H, E, I_, Ns, Is, K = cfg.n_tokens, cfg.hidden, cfg.n_experts, cfg.inter, cfg.n_shared, cfg.shared_inter, cfg.top_k
+    if kernel == "gemm1":
+        b = touched * 2 * H * I_ * e + Ns * 2 * H * Is * e + T * H * e + (P * I_ + Ns * T * Is) * e
+        f = 4 * H * I_ * P + 4 * H * Is * Ns * T
+    elif kernel == "gemm2":
+        b = touched * H * I_ * e + Ns * H * Is * e + (P * I_ + Ns * T * Is) * e + T * H * e
+        f = 2 * H * I_ * P + 2 * H * Is * Ns * T
+    elif kernel == "route":
+        b = T * H * e + E * H * e + T * K * 8 + T * E * 4
+        f = 2 * T * H * E
+    elif kernel == "gather":
+        b = T * H * e + P * H * e
+        f = 0
+    elif kernel == "finalize":
+        b = T * H * 4 + T * H * e
+        f = 0
+    else:
+        b, f = 0, 0
+    return float(b), float(f)
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and clock-event reasons while the timed region runs (read-only NVML)."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz, self.ok = [], set(), None, False
+        self._stop = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+        self.th = None
+
+    def sample_once(self):
+        if not self.ok:
+            return
+        try:
+            self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.dev, self.nv.NVML_CLOCK_SM)))
+            try:
+                r = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev))
+            except Exception:
+                r = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev))
+            for bit, name in self.REASONS.items():
+                if r & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample_once()
+            time.sleep(0.002)
+
+    def start(self):
+        if self.ok:
+            self.th = threading.Thread(target=self._run, daemon=True)
+            self.th.start()
+
+    def stop(self):
+        self._stop.set()
+        if self.th is not None:
+            self.th.join(timeout=2)
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ oracle timing
+def oracle_sample(name, cfg, prune, frac):
+    """Inputs of a bounded sample: the first `frac` of every sequence's visual and text tokens."""
+    from paper_2511_17885_b200 import inputs as I
+    x, mask, seq_off, n_vis = I.make_tokens(cfg)
+    w = I.make_weights(cfg)
+    idx = []
+    for b in range(cfg.batch):
+        lo = int(seq_off[b])
+        nv = max(prune.window * 4, int(cfg.n_vis * frac))
+        nt = max(1, int(cfg.n_text * frac))
+        idx += list(range(lo, lo + min(nv, cfg.n_vis))) + list(range(lo + cfg.n_vis, lo + cfg.n_vis + min(nt, cfg.n_text)))
+    idx = np.array(idx)
+    xs, ms = x[idx], mask[idx]
+    per = len(idx) // cfg.batch
+    so = np.arange(cfg.batch + 1, dtype=np.int64) * per
+    nvs = np.array([int(ms[so[b]:so[b + 1]].sum()) for b in range(cfg.batch)], np.int64)
+    return xs, ms, so, nvs, w
+
+
+def oracle_step(cfg, prune, xs, ms, so, nvs, w):
+    from oracle import fmmoe_oracle as O
+    from paper_2511_17885_b200 import inputs as I
+    r = O.moe_forward(xs, ms, w, cfg.top_k, cfg.top_k_vis, True)
+    O.prune_visual(r["out"], ms, r["probs"], None, so, I.retain_counts(nvs, prune.retain), prune.window,
+                   prune.alpha, prune.gamma)
+
+
+def time_oracle(name, cfg, prune, frac, steps, warmup):
+    import torch
+    xs, ms, so, nvs, w = oracle_sample(name, cfg, prune, frac)
+    for _ in range(warmup):
+        oracle_step(cfg, prune, xs, ms, so, nvs, w)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(cfg, prune, xs, ms, so, nvs, w)
+    dt = time.perf_counter() - t0
+    cores = min(len(os.sched_getaffinity(0)), torch.get_num_threads() if torch.get_num_threads() > 0 else 1)
+    try:
+        from threadpoolctl import threadpool_info
+        nt = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if nt:
+            cores = max(nt)
+    except Exception:
+        pass
+    sample = (f"{xs.shape[0]} of {cfg.n_tokens} tokens of the workload (first {frac:.3g} of each sequence's visual "
+              f"and text tokens), route + experts + combine + pruning, fp64 numpy, {steps} pass(es)")
+    return xs.shape[0] * steps / dt, dt / max(steps, 1), int(cores), sample
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return 0
+    cfg, prune = workload_cfg(args.workload)
+    frac = 1.0 if cfg.n_tokens <= 4096 else 4096.0 / cfg.n_tokens
+    value, spp, cores, sample = time_oracle(args.workload, cfg, prune, frac, max(args.steps, 1), args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": spp * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": describe(args.workload, cfg, prune),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------ the CUDA arm
+def run_ours(args):
+    import torch
+    from paper_2511_17885_b200 import binding as B
+    from paper_2511_17885_b200 import dist as D
+    from paper_2511_17885_b200.workload import LayerWorkload
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    rank, local, world = D.init("nccl") if int(os.environ.get("WORLD_SIZE", 1)) > 1 else (0, 0, 1)
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    cfg, prune = workload_cfg(args.workload)
+    peaks = load_peaks()
+    h = B.Handle(local)
+    wl = LayerWorkload(cfg, h, device=local, prune=prune, token_seed=D.token_seed_for_rank(cfg.seed, rank))
+    K, W = args.steps, max(args.warmup, 0)
+
+    for _ in range(max(W, 1)):
+        wl.step()
+    h.check_status("warm-up")
+    P, touched = wl.routing_stats()
+
+    # ---- device-resident timed region
+    clocks = ClockSampler(local)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h.profile_reset()
+    h.profile_enable(True)
+    D.barrier(); torch.cuda.synchronize()
+    clocks.start()
+    n0 = h.launch_count()
+    ev0.record()
+    for _ in range(K):
+        wl.step()
+    ev1.record()
+    clocks.sample_once()
+    torch.cuda.synchronize(); D.barrier()
+    clocks.stop()
+    launches = h.launch_count() - n0
+    h.profile_enable(False)
+    prof = h.profile_read()
+    h.check_status("timed region")
+    secs = ev0.elapsed_time(ev1) * 1e-3
+    value, tmax = D.aggregate_throughput(cfg.n_tokens * K, secs, dev)
+
+    # ---- end-to-end region (host buffers in, host buffers out)
+    for _ in range(min(max(W, 1), 3)):
+        wl.step_host()
+    D.barrier(); torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(K):
+        wl.step_host()
+    e1.record()
+    torch.cuda.synchronize(); D.barrier()
+    e2e_value, _ = D.aggregate_throughput(cfg.n_tokens * K, e0.elapsed_time(e1) * 1e-3, dev)
+    h.check_status("end-to-end region")
+
+    # ---- roofline of the dominant kernel
+    dom = max(prof, key=lambda k: prof[k]["ms"])
+    per_launch_s = prof[dom]["ms"] * 1e-3 / max(prof[dom]["launches"], 1)
+    b, f = kernel_work(cfg, dom, P, touched)
+    t_hbm, t_tc = b / (peaks["hbm_gbs"] * 1e9), f / (peaks["tf_sustained"] * 1e12)
+    if t_hbm >= t_tc:
+        roof = {"bound": "hbm", "achieved": b / per_launch_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "tensor", "achieved": f / per_launch_s / 1e12, "peak": peaks["tf_sustained"], "unit": "TFLOP/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.workload, {}).get(dom)
+    roof.update({"kernel": dom, "us_per_launch": per_launch_s * 1e6, "algorithmic_bytes": b, "algorithmic_flops": f,
+                 "peak_source": peaks["source"]})
+    # whole step against the slower of (activated FLOPs at tensor peak, algorithmic bytes at HBM bandwidth)
+    tot_b = sum(kernel_work(cfg, k, P, touched)[0] for k in ("route", "gemm1", "gemm2")) \
+        - 2 * cfg.n_tokens * cfg.hidden * (2 if cfg.dtype == "bf16" else 4)   # X is read once, not three times
+    tot_f = sum(kernel_work(cfg, k, P, touched)[1] for k in ("route", "gemm1", "gemm2"))
+    t_step = max(tot_b / (peaks["hbm_gbs"] * 1e9), tot_f / (peaks["tf_sustained"] * 1e12))
+    step_s = tmax / K
+    kernels = {k: {"us_per_step": v["ms"] * 1e3 / K, "launches_per_step": v["launches"] / K,
+                   "share": v["ms"] / max(sum(x["ms"] for x in prof.values()), 1e-12)}
+               for k, v in prof.items() if v["launches"]}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        frac = 1.0 if cfg.n_tokens <= 4096 else 4096.0 / cfg.n_tokens
+        v, spp, cores, sample = time_oracle(args.workload, cfg, prune, frac, 3, 0)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+
+    if rank == 0:
+        conf = describe(args.workload, cfg, prune)
+        conf.update({"routed_pairs": P, "experts_touched": touched, "parallelism": f"replicas x{world} (no collective)"})
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": cfg.dtype, "data": "synthetic", "config": conf,
+                "clocks": clocks.summary(),
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(),
+                        "d2h_bytes_per_step": wl.d2h_bytes()},
+                "gpu_launches": int(launches),
+                "roofline": roof,
+                "step_roofline": {"frac": t_step / step_s, "t_bound_us": t_step * 1e6, "algorithmic_bytes": tot_b,
+                                  "activated_flops": tot_f, "peak_source": peaks["source"]},
+                "kernels": kernels,
+                "cpu_baseline": cpu}
+        print(json.dumps(line))
+    D.shutdown()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C1", choices=WORKLOADS)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    sys.exit(run_reference(args) if args.impl == "reference" else run_ours(args))
+
+
+if __name__ == "__main__":
+    main()

@@ -141,12 +141,29 @@ fmmoe_status fmmoe_moe_forward(fmmoe_handle *handle, const fmmoe_layer_desc *des
  * copies x_host [T,H] and is_visual_host [T] to the device, runs the layer, copies
  * out back to out_host [T,H] and SYNCHRONISES the stream before returning.
  * Pinned host buffers make the copies asynchronous.  `workspace` must hold
- * fmmoe_workspace_bytes() + fmmoe_host_staging_bytes() bytes.  Weights stay on the device. */
+ * fmmoe_workspace_bytes() + fmmoe_host_staging_bytes() bytes.  Weights stay on the device.
+ * Optional DEVICE outputs for a caller that continues on the GPU (e.g. with
+ * fmmoe_prune_visual): `route` as in fmmoe_moe_forward, `out_dev` [T,H] receives the
+ * layer output, `is_visual_dev` [T] the uploaded mask.  Each may be NULL. */
 size_t fmmoe_host_staging_bytes(const fmmoe_layer_desc *desc, int64_t n_tokens);
 fmmoe_status fmmoe_moe_forward_host(fmmoe_handle *handle, const fmmoe_layer_desc *desc, const fmmoe_weights *w,
                                     const void *x_host, const uint8_t *is_visual_host, int64_t n_tokens,
-                                    uint32_t flags, void *out_host, void *workspace, size_t workspace_bytes,
+                                    uint32_t flags, void *out_host, const fmmoe_route_out *route, void *out_dev,
+                                    uint8_t *is_visual_dev, void *workspace, size_t workspace_bytes,
                                     void *cuda_stream);
+
+/* Optional per-kernel timeline.  While enabled, every kernel the handle launches is
+ * bracketed by CUDA events on the launching stream (host-side event objects only; no
+ * device memory).  fmmoe_profile_read synchronises the device and returns the summed
+ * duration and the number of launches of one kernel since the last reset. */
+enum {
+  FMMOE_KERNEL_ROUTE = 0, FMMOE_KERNEL_PERMUTE = 1, FMMOE_KERNEL_GATHER = 2, FMMOE_KERNEL_GEMM1 = 3,
+  FMMOE_KERNEL_GEMM2 = 4, FMMOE_KERNEL_FINALIZE = 5, FMMOE_KERNEL_PRUNE_INDEX = 6, FMMOE_KERNEL_PRUNE_SCORE = 7,
+  FMMOE_KERNEL_PRUNE_SELECT = 8, FMMOE_KERNEL_PRUNE_COMPACT = 9, FMMOE_KERNEL_COUNT = 10
+};
+fmmoe_status fmmoe_profile_enable(fmmoe_handle *handle, int enable);
+fmmoe_status fmmoe_profile_reset(fmmoe_handle *handle);
+fmmoe_status fmmoe_profile_read(fmmoe_handle *handle, int kernel_id, double *total_ms, int64_t *launches);
 
 /* Section 3.2 hyper-parameters. */
 typedef struct {

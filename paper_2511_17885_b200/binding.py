@@ -73,8 +73,13 @@ def lib() -> C.CDLL:
     L.fmmoe_moe_forward.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), vp, vp, i64, u32, vp,
                                     C.POINTER(RouteOut), vp, sz, vp]
     L.fmmoe_moe_forward.restype = C.c_int
-    L.fmmoe_moe_forward_host.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), vp, vp, i64, u32, vp, vp, sz, vp]
+    L.fmmoe_moe_forward_host.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), vp, vp, i64, u32, vp,
+                                         C.POINTER(RouteOut), vp, vp, vp, sz, vp]
     L.fmmoe_moe_forward_host.restype = C.c_int
+    L.fmmoe_profile_enable.argtypes = [vp, C.c_int]; L.fmmoe_profile_enable.restype = C.c_int
+    L.fmmoe_profile_reset.argtypes = [vp]; L.fmmoe_profile_reset.restype = C.c_int
+    L.fmmoe_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_double), C.POINTER(i64)]
+    L.fmmoe_profile_read.restype = C.c_int
     L.fmmoe_prune_kept_count.argtypes = [i64, i64, C.POINTER(PruneParams), C.POINTER(i64), C.POINTER(i64)]
     L.fmmoe_prune_kept_count.restype = i64
     L.fmmoe_prune_workspace_bytes.argtypes = [i64, i32]; L.fmmoe_prune_workspace_bytes.restype = sz
@@ -177,6 +182,24 @@ class Handle:
     def launch_count(self) -> int:
         return int(lib().fmmoe_launch_count(self._h))
 
+    KERNELS = ("route", "permute", "gather", "gemm1", "gemm2", "finalize", "prune_index", "prune_score",
+               "prune_select", "prune_compact")
+
+    def profile_enable(self, on: bool = True):
+        _check(lib().fmmoe_profile_enable(self._h, 1 if on else 0), "fmmoe_profile_enable")
+
+    def profile_reset(self):
+        _check(lib().fmmoe_profile_reset(self._h), "fmmoe_profile_reset")
+
+    def profile_read(self) -> Dict[str, Dict[str, float]]:
+        """Per kernel: summed milliseconds and launches since the last reset."""
+        out = {}
+        for i, name in enumerate(self.KERNELS):
+            ms, n = C.c_double(0), C.c_int64(0)
+            _check(lib().fmmoe_profile_read(self._h, i, C.byref(ms), C.byref(n)), "fmmoe_profile_read")
+            out[name] = {"ms": ms.value, "launches": int(n.value)}
+        return out
+
     # ---- Section 3.1
     def fmmoe_route(self, desc: LayerDesc, w: Weights, x: torch.Tensor, is_visual: torch.Tensor, flags: int,
                     want=("logits", "probs", "topk_idx", "topk_w", "expert_off", "row_token", "inv_row")):
@@ -208,15 +231,18 @@ class Handle:
         return out
 
     def fmmoe_moe_forward_host(self, desc: LayerDesc, w: Weights, x_host: torch.Tensor, is_visual_host: torch.Tensor,
-                               flags: int, out_host: torch.Tensor):
+                               flags: int, out_host: torch.Tensor, route: Optional[Dict[str, torch.Tensor]] = None,
+                               out_dev: Optional[torch.Tensor] = None, is_visual_dev: Optional[torch.Tensor] = None):
         """Host-buffer variant: H2D copy, layer, D2H copy, stream synchronised on return."""
         T = x_host.shape[0]
+        ro = RouteOut(**{k: v.data_ptr() for k, v in route.items()}) if route else None
         assert not x_host.is_cuda and not out_host.is_cuda and x_host.is_contiguous() and out_host.is_contiguous()
         need = fmmoe_workspace_bytes(desc, T, flags) + int(lib().fmmoe_host_staging_bytes(C.byref(desc), T))
         wsp, wsn = self._ws_args(need)
         _check(lib().fmmoe_moe_forward_host(self._h, C.byref(desc), C.byref(w), C.c_void_p(x_host.data_ptr()),
                                             C.c_void_p(is_visual_host.data_ptr()), T, flags,
-                                            C.c_void_p(out_host.data_ptr()), wsp, wsn, _stream()),
+                                            C.c_void_p(out_host.data_ptr()), C.byref(ro) if ro is not None else None,
+                                            _ptr(out_dev), _ptr(is_visual_dev), wsp, wsn, _stream()),
                "fmmoe_moe_forward_host")
         return out_host
 

@@ -157,6 +157,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
   h->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
   h->launches = 0;
   h->d_status = nullptr; h->h_status = nullptr; h->encode_tiled = nullptr;
+  h->tc_attr_set = false; h->profiling = false; h->ev_used = 0;
   if (cudaMalloc(&h->d_status, 256) != cudaSuccess || cudaMemset(h->d_status, 0, 256) != cudaSuccess ||
       cudaMallocHost(&h->h_status, 256) != cudaSuccess) {
     if (h->d_status) cudaFree(h->d_status);
@@ -177,6 +178,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_destroy(fmm
   cudaSetDevice(h->device);
   if (h->d_status) cudaFree(h->d_status);
   if (h->h_status) cudaFreeHost(h->h_status);
+  for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   delete h;
   return FMMOE_OK;
 }
@@ -269,8 +271,9 @@ extern "C" __attribute__((visibility("default"))) size_t fmmoe_host_staging_byte
 
 extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward_host(fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w,
                                                const void* x_host, const uint8_t* is_visual_host, int64_t T,
-                                               uint32_t flags, void* out_host, void* workspace, size_t workspace_bytes,
-                                               void* cuda_stream) {
+                                               uint32_t flags, void* out_host, const fmmoe_route_out* route,
+                                               void* out_dev, uint8_t* is_visual_dev, void* workspace,
+                                               size_t workspace_bytes, void* cuda_stream) {
   if (!h || !desc_ok(d) || T < 0) return FMMOE_ERR_INVALID_ARG;
   if (T > 0 && (!x_host || !is_visual_host || !out_host)) return FMMOE_ERR_INVALID_ARG;
   const size_t elem = d->dtype == FMMOE_BF16 ? 2 : 4;
@@ -282,13 +285,45 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);
   char* dx = ws;
-  char* dout = ws + align_up(xb, 256);
-  uint8_t* dvis = reinterpret_cast<uint8_t*>(ws + 2 * align_up(xb, 256));
+  char* dout = out_dev ? static_cast<char*>(out_dev) : ws + align_up(xb, 256);
+  uint8_t* dvis = is_visual_dev ? is_visual_dev : reinterpret_cast<uint8_t*>(ws + 2 * align_up(xb, 256));
   FMMOE_CUDA_TRY(cudaMemcpyAsync(dx, x_host, xb, cudaMemcpyHostToDevice, s));
   FMMOE_CUDA_TRY(cudaMemcpyAsync(dvis, is_visual_host, (size_t)T, cudaMemcpyHostToDevice, s));
-  const fmmoe_status st = fmmoe_moe_forward(h, d, w, dx, dvis, T, flags, dout, nullptr, ws + stage, workspace_bytes - stage, s);
+  const fmmoe_status st = fmmoe_moe_forward(h, d, w, dx, dvis, T, flags, dout, route, ws + stage, workspace_bytes - stage, s);
   if (st != FMMOE_OK) return st;
   FMMOE_CUDA_TRY(cudaMemcpyAsync(out_host, dout, xb, cudaMemcpyDeviceToHost, s));
   FMMOE_CUDA_TRY(cudaStreamSynchronize(s));
+  return FMMOE_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_profile_enable(fmmoe_handle* h, int enable) {
+  if (!h) return FMMOE_ERR_INVALID_ARG;
+  h->profiling = enable != 0;
+  return FMMOE_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_profile_reset(fmmoe_handle* h) {
+  if (!h) return FMMOE_ERR_INVALID_ARG;
+  FMMOE_CUDA_TRY(cudaDeviceSynchronize());
+  h->prof.clear();
+  h->ev_used = 0;
+  return FMMOE_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_profile_read(fmmoe_handle* h, int kernel_id,
+                                                                                  double* total_ms, int64_t* launches) {
+  if (!h || kernel_id < 0 || kernel_id >= FMMOE_KERNEL_COUNT || !total_ms || !launches) return FMMOE_ERR_INVALID_ARG;
+  FMMOE_CUDA_TRY(cudaDeviceSynchronize());
+  double tot = 0.0;
+  int64_t n = 0;
+  for (const auto& r : h->prof) {
+    if (r.id != kernel_id) continue;
+    float ms = 0.f;
+    FMMOE_CUDA_TRY(cudaEventElapsedTime(&ms, h->ev_pool[r.start], h->ev_pool[r.stop]));
+    tot += ms;
+    ++n;
+  }
+  *total_ms = tot;
+  *launches = n;
   return FMMOE_OK;
 }

@@ -77,8 +77,11 @@ fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_
   long long blocks = (n + threads - 1) / threads;
   const long long cap = (long long)h->sm_count * 16;
   if (blocks > cap) blocks = cap;
-  if (a.dtype == FMMOE_BF16) finalize_kernel<__nv_bfloat16><<<(int)blocks, threads, 0, s>>>(d);
-  else finalize_kernel<float><<<(int)blocks, threads, 0, s>>>(d);
+  {
+    ProfScope ps(h, FMMOE_KERNEL_FINALIZE, s);
+    if (a.dtype == FMMOE_BF16) finalize_kernel<__nv_bfloat16><<<(int)blocks, threads, 0, s>>>(d);
+    else finalize_kernel<float><<<(int)blocks, threads, 0, s>>>(d);
+  }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 1;
   return FMMOE_OK;

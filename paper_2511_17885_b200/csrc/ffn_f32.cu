@@ -124,14 +124,14 @@ fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   p.b0 = static_cast<const float*>(a.w->w_gate); p.b1 = static_cast<const float*>(a.w->w_up);
   p.out = static_cast<float*>(a.act);
   if (a.max_mtiles > 0) {
-    ffn_f32_kernel<0><<<dim3(a.max_mtiles, (I + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(p);
+    { ProfScope prof_(h, FMMOE_KERNEL_GEMM1, s); ffn_f32_kernel<0><<<dim3(a.max_mtiles, (I + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(p); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     // routed GEMM-2
     F32Params q = p;
     q.K = I; q.N = H; q.a = static_cast<const float*>(a.act);
     q.b0 = static_cast<const float*>(a.w->w_down); q.b1 = nullptr;
     q.out = a.y; q.acc = a.acc; q.deterministic = a.deterministic;
-    ffn_f32_kernel<1><<<dim3(a.max_mtiles, (H + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(q);
+    { ProfScope prof_(h, FMMOE_KERNEL_GEMM2, s); ffn_f32_kernel<1><<<dim3(a.max_mtiles, (H + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(q); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     h->launches += 2;
   }
@@ -140,13 +140,13 @@ fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
     ps.mt_per_shared = mtps; ps.T = a.T; ps.K = H; ps.N = Is; ps.a = static_cast<const float*>(a.x);
     ps.b0 = static_cast<const float*>(a.w->ws_gate); ps.b1 = static_cast<const float*>(a.w->ws_up);
     ps.out = static_cast<float*>(a.act_sh);
-    ffn_f32_kernel<0><<<dim3(Ns * mtps, (Is + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(ps);
+    { ProfScope prof_(h, FMMOE_KERNEL_GEMM1, s); ffn_f32_kernel<0><<<dim3(Ns * mtps, (Is + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(ps); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     F32Params qs = ps;
     qs.K = Is; qs.N = H; qs.a = static_cast<const float*>(a.act_sh);
     qs.b0 = static_cast<const float*>(a.w->ws_down); qs.b1 = nullptr;
     qs.out = a.ysh; qs.acc = a.acc; qs.deterministic = a.deterministic;
-    ffn_f32_kernel<1><<<dim3(Ns * mtps, (H + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(qs);
+    { ProfScope prof_(h, FMMOE_KERNEL_GEMM2, s); ffn_f32_kernel<1><<<dim3(Ns * mtps, (H + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(qs); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     h->launches += 2;
   }

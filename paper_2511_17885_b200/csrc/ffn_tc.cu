@@ -345,16 +345,15 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   p2.row_token = a.row_token; p2.row_gate = a.row_gate; p2.acc = a.acc;
   p2.y[0] = a.y; p2.y[1] = a.ysh; p2.deterministic = a.deterministic;
 
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (!h->tc_attr_set) {
     FMMOE_CUDA_TRY(cudaFuncSetAttribute(ffn_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES));
     FMMOE_CUDA_TRY(cudaFuncSetAttribute(ffn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES));
-    attr_set = true;
+    h->tc_attr_set = true;
   }
   const int grid = h->sm_count;
-  ffn_tc_kernel<0><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(A1r, A1s, G1r, U1r, G1s, U1s, p1);
+  { ProfScope ps(h, FMMOE_KERNEL_GEMM1, s); ffn_tc_kernel<0><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(A1r, A1s, G1r, U1r, G1s, U1s, p1); }
   FMMOE_CUDA_TRY(cudaGetLastError());
-  ffn_tc_kernel<1><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(A2r, A2s, D2r, D2r, D2s, D2s, p2);
+  { ProfScope ps(h, FMMOE_KERNEL_GEMM2, s); ffn_tc_kernel<1><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(A2r, A2s, D2r, D2r, D2s, D2s, p2); }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 2;
   return FMMOE_OK;

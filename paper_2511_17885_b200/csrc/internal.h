@@ -5,6 +5,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "../../include/fmmoe.h"
 
 struct fmmoe_handle {
@@ -15,6 +17,13 @@ struct fmmoe_handle {
   int* h_status;        // pinned host mirror
   int64_t launches;     // kernels launched through this handle
   void* encode_tiled;   // cuTensorMapEncodeTiled entry point
+  bool tc_attr_set;     // dynamic shared memory opt-in done for the tensor-core kernels
+  // optional kernel timeline
+  bool profiling;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used;
+  struct ProfRec { int id; size_t start, stop; };
+  std::vector<ProfRec> prof;
 };
 
 namespace fmmoe {
@@ -53,6 +62,27 @@ struct WsPlan {
   int32_t max_mtiles;
 };
 bool plan_workspace(const fmmoe_layer_desc& d, int64_t T, uint32_t flags, WsPlan* p);
+
+// Brackets one kernel launch with events when the handle's timeline is on.
+struct ProfScope {
+  fmmoe_handle* h; cudaStream_t s; size_t rec; bool on;
+  ProfScope(fmmoe_handle* h_, int id, cudaStream_t s_) : h(h_), s(s_), rec(0), on(h_->profiling) {
+    if (!on) return;
+    while (h->ev_pool.size() < h->ev_used + 2) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+      h->ev_pool.push_back(e);
+    }
+    fmmoe_handle::ProfRec r{id, h->ev_used, h->ev_used + 1};
+    h->ev_used += 2;
+    h->prof.push_back(r);
+    rec = h->prof.size() - 1;
+    cudaEventRecord(h->ev_pool[r.start], s);
+  }
+  ~ProfScope() {
+    if (on) cudaEventRecord(h->ev_pool[h->prof[rec].stop], s);
+  }
+};
 
 #define FMMOE_CUDA_TRY(expr)                         \
   do {                                               \

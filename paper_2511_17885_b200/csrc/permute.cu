@@ -125,7 +125,7 @@ fmmoe_status launch_permute(fmmoe_handle* h, const PermuteArgs& a, cudaStream_t 
   d.T = a.T; d.K = a.K; d.E = a.E; d.block_m = a.block_m;
   d.expert_off = a.expert_off; d.row_token = a.row_token; d.row_gate = a.row_gate; d.inv_row = a.inv_row;
   d.mtiles = a.mtiles; d.n_mtiles = a.n_mtiles;
-  permute_kernel<<<a.E, P_THREADS, 0, s>>>(d);
+  { ProfScope ps(h, FMMOE_KERNEL_PERMUTE, s); permute_kernel<<<a.E, P_THREADS, 0, s>>>(d); }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 1;
   return FMMOE_OK;
@@ -139,8 +139,11 @@ fmmoe_status launch_gather_rows(fmmoe_handle* h, const void* x, const int32_t* r
   long long blocks = (p_max + 7) / 8;
   const long long cap = (long long)h->sm_count * 8;
   if (blocks > cap) blocks = cap;
-  gather_rows_kernel<<<(int)blocks, threads, 0, s>>>(static_cast<const uint4*>(x), row_token, expert_off, E, p_max,
-                                                     row_vec, static_cast<uint4*>(xp));
+  {
+    ProfScope ps(h, FMMOE_KERNEL_GATHER, s);
+    gather_rows_kernel<<<(int)blocks, threads, 0, s>>>(static_cast<const uint4*>(x), row_token, expert_off, E, p_max,
+                                                       row_vec, static_cast<uint4*>(xp));
+  }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 1;
   return FMMOE_OK;

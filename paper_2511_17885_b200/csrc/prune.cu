@@ -534,19 +534,20 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
     for (int i = 0; i <= nb; ++i) rel.win_off[i] -= win_base;
     PruneDev al = a;
     al.sim = a.sim + win_base; al.asum = a.asum + win_base; al.action = a.action + win_base;
-    vis_index_kernel<<<nb, 1024, 0, s>>>(al, rel);
+    { ProfScope ps(h, FMMOE_KERNEL_PRUNE_INDEX, s); vis_index_kernel<<<nb, 1024, 0, s>>>(al, rel); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     h->launches += 1;
     if (n_win > 0) {
-      window_score_kernel<<<(n_win + 7) / 8, 256, 0, s>>>(al, rel);
+      { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SCORE, s); window_score_kernel<<<(n_win + 7) / 8, 256, 0, s>>>(al, rel); }
       FMMOE_CUDA_TRY(cudaGetLastError());
       h->launches += 1;
     }
-    select_kernel<<<nb, 1024, sel_smem, s>>>(al, rel);
+    { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SELECT, s); select_kernel<<<nb, 1024, sel_smem, s>>>(al, rel); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     h->launches += 1;
     const long long rows = rel.out_off[nb] - rel.out_off[0];
     if (rows > 0) {
+      ProfScope ps(h, FMMOE_KERNEL_PRUNE_COMPACT, s);
       if (dtype == FMMOE_BF16)
         compact_kernel<__nv_bfloat16><<<(unsigned)rows, 256, 0, s>>>(al, rel, rel.out_off[0], rows);
       else

@@ -273,16 +273,18 @@ __global__ void __launch_bounds__(R_THREADS) route_f32_kernel(const RouteDev a) 
 }
 
 template <int NT>
-static fmmoe_status launch_nt(const RouteDev& d, int dtype, int grid, cudaStream_t s) {
+static fmmoe_status launch_nt(fmmoe_handle* h, const RouteDev& d, int dtype, int grid, cudaStream_t s) {
   const int e_pad = NT * 32;
   const size_t tail = (size_t)R_BM * (e_pad + 1) * 4 + (size_t)e_pad * 4;
   if (dtype == FMMOE_BF16) {
     const size_t smem = (size_t)R_STAGES * (R_BM + e_pad) * R_LDS * 2 + tail;
     FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_bf16_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
     route_bf16_kernel<NT><<<grid, R_THREADS, smem, s>>>(d);
   } else {
     const size_t smem = (size_t)(R_BM + e_pad) * 33 * 4 + tail;
     FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_f32_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
     route_f32_kernel<NT><<<grid, R_THREADS, smem, s>>>(d);
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
@@ -300,14 +302,14 @@ fmmoe_status launch_route(fmmoe_handle* h, const RouteArgs& a, cudaStream_t s) {
   const int grid = (int)((a.T + R_BM - 1) / R_BM);
   fmmoe_status st;
   switch (d.e_pad / 32) {
-    case 1: st = launch_nt<1>(d, a.dtype, grid, s); break;
-    case 2: st = launch_nt<2>(d, a.dtype, grid, s); break;
-    case 3: st = launch_nt<3>(d, a.dtype, grid, s); break;
-    case 4: st = launch_nt<4>(d, a.dtype, grid, s); break;
-    case 5: st = launch_nt<5>(d, a.dtype, grid, s); break;
-    case 6: st = launch_nt<6>(d, a.dtype, grid, s); break;
-    case 7: st = launch_nt<7>(d, a.dtype, grid, s); break;
-    case 8: st = launch_nt<8>(d, a.dtype, grid, s); break;
+    case 1: st = launch_nt<1>(h, d, a.dtype, grid, s); break;
+    case 2: st = launch_nt<2>(h, d, a.dtype, grid, s); break;
+    case 3: st = launch_nt<3>(h, d, a.dtype, grid, s); break;
+    case 4: st = launch_nt<4>(h, d, a.dtype, grid, s); break;
+    case 5: st = launch_nt<5>(h, d, a.dtype, grid, s); break;
+    case 6: st = launch_nt<6>(h, d, a.dtype, grid, s); break;
+    case 7: st = launch_nt<7>(h, d, a.dtype, grid, s); break;
+    case 8: st = launch_nt<8>(h, d, a.dtype, grid, s); break;
     default: return FMMOE_ERR_UNSUPPORTED;
   }
   if (st == FMMOE_OK) h->launches += 1;
