@@ -39,7 +39,8 @@ typedef enum {
   FMMOE_ERR_WORKSPACE = 3,     /* workspace NULL, misaligned or too small                */
   FMMOE_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                      */
   FMMOE_ERR_TIMEOUT = 5,       /* a device-side bounded wait expired                     */
-  FMMOE_ERR_INTERNAL = 6
+  FMMOE_ERR_INTERNAL = 6,
+  FMMOE_ERR_TOO_LARGE = 7      /* problem exceeds the built-in scratch of a *_static entry point */
 } fmmoe_status;
 
 typedef enum { FMMOE_F32 = 0, FMMOE_BF16 = 1 } fmmoe_dtype;
@@ -213,6 +214,42 @@ fmmoe_status fmmoe_prune_visual(fmmoe_handle *handle, const fmmoe_prune_params *
                                 void *x_out, uint8_t *is_visual_out, int32_t *keep_idx, uint8_t *kind,
                                 int64_t *out_seq_off /* host [n_seq+1] */,
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* fmmoe_prune_visual without a caller-supplied workspace and without any allocation.
+ * (The paper has no counterpart: this is a packaging variant of fmmoe_prune_visual above,
+ * same arguments minus `workspace`/`workspace_bytes`, same kernels, same results.)
+ *
+ * For callers that cannot obtain device memory at the point where they prune: a server
+ * whose HBM was handed to another memory pool at start-up, or a latency-critical loop that
+ * must not run into the device-wide synchronisation an allocation or a free can cause.
+ * Inputs and outputs are still the caller's buffers.  The scratch lives in a fixed array
+ * inside the library: FMMOE_STATIC_PRUNE_SCRATCH_BYTES (768 KiB) of device memory on every
+ * GPU that loads the library, held until the process exits.
+ *
+ *   - The call makes no cudaMalloc/cudaFree and uses no allocating library routine.  The
+ *     handle must exist already (fmmoe_create, done once at start-up, is where the
+ *     library's only allocation happens) and its device must be the current device,
+ *     otherwise FMMOE_ERR_INVALID_ARG.  Keep the handle's kernel timeline off
+ *     (fmmoe_profile_enable) in such a setting: it creates event objects on demand.
+ *   - Limit: seq_off[n_seq] <= FMMOE_STATIC_PRUNE_MAX_TOKENS tokens per call; more returns
+ *     FMMOE_ERR_TOO_LARGE before anything is enqueued.
+ *   - The first call on each device looks up the array's device address (a one-time
+ *     set-up step guarded by a mutex); make that first call before starting any stream
+ *     capture on that device.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call
+ *     left in it.  No part of it needs clearing (each pass writes every word before reading
+ *     it), but two calls whose kernels may overlap on the GPU - different streams, or
+ *     different host threads - race on it: serialise them, or use fmmoe_prune_visual with
+ *     separate workspaces. */
+#define FMMOE_STATIC_PRUNE_MAX_TOKENS 32768
+fmmoe_status fmmoe_prune_visual_static(fmmoe_handle *handle, const fmmoe_prune_params *p,
+                                       const float *probs, int32_t n_experts, const float *attn,
+                                       const void *x, int32_t dtype, int32_t hidden, const uint8_t *is_visual,
+                                       const int64_t *seq_off /* host [n_seq+1] */,
+                                       const int64_t *n_vis /* host [n_seq] */,
+                                       const int64_t *n_retain /* host [n_seq] */, int32_t n_seq,
+                                       void *x_out, uint8_t *is_visual_out, int32_t *keep_idx, uint8_t *kind,
+                                       int64_t *out_seq_off /* host [n_seq+1] */, void *cuda_stream);
 
 #ifdef __cplusplus
 }

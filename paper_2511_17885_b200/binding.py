@@ -16,10 +16,12 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libfmmoe.so")
 
 FMMOE_OK = 0
-STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE", 4: "CUDA", 5: "TIMEOUT", 6: "INTERNAL"}
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE", 4: "CUDA", 5: "TIMEOUT", 6: "INTERNAL",
+                7: "TOO_LARGE"}
 F32, BF16 = 0, 1
 FLAG_REDUCE_ON, FLAG_RESIDUAL, FLAG_DETERMINISTIC = 1, 2, 4
 MAX_EXPERTS, MAX_TOPK, MAX_WINDOW = 256, 16, 8
+STATIC_PRUNE_MAX_TOKENS = 32768
 
 
 class LayerDesc(C.Structure):
@@ -87,6 +89,10 @@ def lib() -> C.CDLL:
                                      C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), i32,
                                      vp, vp, vp, vp, C.POINTER(i64), vp, sz, vp]
     L.fmmoe_prune_visual.restype = C.c_int
+    L.fmmoe_prune_visual_static.argtypes = [vp, C.POINTER(PruneParams), vp, i32, vp, vp, i32, i32, vp,
+                                            C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), i32,
+                                            vp, vp, vp, vp, C.POINTER(i64), vp]
+    L.fmmoe_prune_visual_static.restype = C.c_int
     _lib = L
     return L
 
@@ -276,3 +282,28 @@ class Handle:
                                         _stream()), "fmmoe_prune_visual")
         return {"x_out": x_out, "is_visual_out": vis_out, "keep_idx": keep_idx, "kind": kind,
                 "out_seq_off": [int(v) for v in oo]}
+
+    def fmmoe_prune_visual_static(self, p: PruneParams, probs: torch.Tensor, attn: Optional[torch.Tensor],
+                                  x: torch.Tensor, is_visual: torch.Tensor, seq_off, n_vis, n_retain,
+                                  x_out: torch.Tensor, is_visual_out: Optional[torch.Tensor] = None,
+                                  keep_idx: Optional[torch.Tensor] = None, kind: Optional[torch.Tensor] = None):
+        """fmmoe_prune_visual for callers that cannot allocate device memory when they prune.
+
+        The library call behind this method takes no workspace and allocates nothing: its
+        scratch is a fixed array inside the library (at most STATIC_PRUNE_MAX_TOKENS tokens
+        per call; more raises FmmoeError TOO_LARGE).  In keeping with that, this wrapper
+        allocates nothing either: the caller passes preallocated outputs, x_out [T', H] with
+        T' from fmmoe_prune_kept_count, and optionally is_visual_out / keep_idx / kind [T'].
+        Calls share the one scratch array, so do not let two of them overlap on the GPU.
+        Returns out_seq_off as a list."""
+        B = len(n_vis)
+        arr = C.c_int64 * (B + 1)
+        so = arr(*[int(v) for v in seq_off])
+        nv = (C.c_int64 * max(B, 1))(*[int(v) for v in n_vis])
+        nr = (C.c_int64 * max(B, 1))(*[int(v) for v in n_retain])
+        oo = arr()
+        _check(lib().fmmoe_prune_visual_static(self._h, C.byref(p), _ptr(probs), probs.shape[1], _ptr(attn), _ptr(x),
+                                               _dtype_code(x.dtype), x.shape[1], _ptr(is_visual), so, nv, nr, B,
+                                               _ptr(x_out), _ptr(is_visual_out), _ptr(keep_idx), _ptr(kind), oo,
+                                               _stream()), "fmmoe_prune_visual_static")
+        return [int(v) for v in oo]

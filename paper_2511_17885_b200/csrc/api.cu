@@ -138,6 +138,7 @@ extern "C" __attribute__((visibility("default"))) const char* fmmoe_status_strin
     case FMMOE_ERR_CUDA: return "CUDA call failed";
     case FMMOE_ERR_TIMEOUT: return "device-side wait timed out";
     case FMMOE_ERR_INTERNAL: return "internal consistency check failed";
+    case FMMOE_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
   }
   return "unknown status";
 }

@@ -11,6 +11,7 @@
 // on thread order; ties go to the lower window index.
 #include <cuda_bf16.h>
 #include <math.h>
+#include <pthread.h>
 
 #include "internal.h"
 
@@ -558,4 +559,72 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
     win_base += n_win;
   }
   return FMMOE_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// fmmoe_prune_visual_static: the same pruning pass, with its scratch memory built into the
+// library instead of supplied by the caller.
+//
+// Who needs it: code that must not ask the CUDA allocator for anything at the point where
+// it prunes.  Examples are an inference server whose whole HBM budget was handed to another
+// memory pool at start-up (a late cudaMalloc there fails or fragments the pool), and a
+// latency-critical loop that cannot afford the device-wide synchronisation an allocation
+// or a free may imply.  Such a caller still owns its inputs and outputs (they come from
+// its pool); what it cannot do is size and carve out a workspace per call.
+//
+// The scratch is the file-scope device array below.  Every GPU on which the library is
+// loaded holds these FMMOE_STATIC_PRUNE_SCRATCH_BYTES until the process exits.  In host
+// code the array's name is only a stand-in for the symbol, never a device address, so the
+// address is looked up with cudaGetSymbolAddress once per device (with that device
+// current) and cached; kernels receive the looked-up pointer.
+// ---------------------------------------------------------------------------------------
+#define FMMOE_STATIC_PRUNE_SCRATCH_BYTES (768u * 1024u)
+static __device__ __align__(256) unsigned char g_prune_scratch[FMMOE_STATIC_PRUNE_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_prune_scratch_addr[kMaxDevices] = {};     // device address of g_prune_scratch, per device
+pthread_mutex_t g_prune_scratch_mu = PTHREAD_MUTEX_INITIALIZER;
+
+// Device address of the scratch array on the CURRENT device (must be `device`); looked up on
+// the first call for that device, cached afterwards.  Returns nullptr on failure.
+void* static_scratch_for(int device) {
+  if (device < 0 || device >= kMaxDevices) return nullptr;
+  pthread_mutex_lock(&g_prune_scratch_mu);
+  void* p = g_prune_scratch_addr[device];
+  if (!p) {
+    void* q = nullptr;
+    if (cudaGetSymbolAddress(&q, g_prune_scratch) == cudaSuccess && q) {
+      g_prune_scratch_addr[device] = q;
+      p = q;
+    }
+  }
+  pthread_mutex_unlock(&g_prune_scratch_mu);
+  return p;
+}
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visual_static(
+    fmmoe_handle* h, const fmmoe_prune_params* p, const float* probs, int32_t n_experts, const float* attn,
+    const void* x, int32_t dtype, int32_t hidden, const uint8_t* is_visual, const int64_t* seq_off,
+    const int64_t* n_vis, const int64_t* n_retain, int32_t n_seq, void* x_out, uint8_t* is_visual_out,
+    int32_t* keep_idx, uint8_t* kind, int64_t* out_seq_off, void* cuda_stream) {
+  if (!h || !seq_off || n_seq < 0) return FMMOE_ERR_INVALID_ARG;
+  const int64_t T = n_seq ? seq_off[n_seq] : 0;
+  if (T < 0) return FMMOE_ERR_INVALID_ARG;
+  // the limit is on the token count: refuse before touching the GPU
+  if (T > FMMOE_STATIC_PRUNE_MAX_TOKENS) return FMMOE_ERR_TOO_LARGE;
+  const size_t need = plan_prune(T).total;
+  if (need > (size_t)FMMOE_STATIC_PRUNE_SCRATCH_BYTES) return FMMOE_ERR_TOO_LARGE;
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess) return FMMOE_ERR_CUDA;
+  if (cur != h->device) return FMMOE_ERR_INVALID_ARG;   // the handle's device must be current
+  void* scratch = static_scratch_for(cur);
+  if (!scratch) return FMMOE_ERR_CUDA;
+  // Nothing in the scratch has to start at zero: every word a kernel of this pass reads was
+  // written earlier in the same pass (vision ranks and lists, window scores, actions, the
+  // compaction map), so the previous call's leftovers are never observed.
+  return fmmoe_prune_visual(h, p, probs, n_experts, attn, x, dtype, hidden, is_visual, seq_off, n_vis, n_retain,
+                            n_seq, x_out, is_visual_out, keep_idx, kind, out_seq_off, scratch,
+                            (size_t)FMMOE_STATIC_PRUNE_SCRATCH_BYTES, cuda_stream);
 }
