@@ -242,6 +242,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward
   FfnArgs fa = {};
   fa.d = d; fa.w = w; fa.x = x; fa.T = T; fa.p_max = pl.p_max;
   fa.mtiles = r.mtiles; fa.n_mtiles = r.misc; fa.max_mtiles = pl.max_mtiles;
+  fa.tile_counters = r.misc + 1;
   fa.row_token = r.row_token; fa.row_gate = r.row_gate;
   fa.xp = ws + pl.xp_off; fa.act = ws + pl.act_off; fa.act_sh = ws + pl.act_sh_off;
   fa.acc = det ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off);

@@ -6,12 +6,23 @@
 //   GEMM-1  [rows_e, H] x [H, 2*S_m]  -> SwiGLU in the epilogue -> act [rows, S_m] bf16
 //   GEMM-2  [rows_e, S_m] x [S_m, H]  -> gate-weighted combine in the epilogue
 // Both run in one persistent, warp-specialised kernel template:
-//   warp 0    : TMA producer  (A tile 128x64 + two B boxes 128x64 per stage, 128B swizzle)
+//   warp 0    : tile scheduler + TMA producer (A tile 128x64 + two B boxes 128x64 per stage,
+//               128B swizzle, L2 eviction hints)
 //   warp 1    : UMMA issuer   (one thread; 128x256x16 tcgen05.mma, accumulators in TMEM)
-//   warps 2-5 : epilogue      (tcgen05.ld -> registers -> global), overlapped with the next
-//               tile's main loop through two TMEM accumulator stages (2 x 256 columns).
-// A tile is (M-tile of 128 grouped rows) x (N-block).  Tile ids run N-block-major so
-// that CTAs working at the same time share weight tiles through L2.
+//   warps 2-5 : epilogue      (tcgen05.ld -> registers -> shared-memory transpose -> coalesced
+//               global stores / reductions), overlapped with the next tile's main loop
+//               through two TMEM accumulator stages (2 x 256 columns).
+// A tile is (M-tile of 128 grouped rows) x (N-block).  Tiles are handed out dynamically (an
+// atomic counter; the producer publishes each tile id to the other roles through a small
+// shared-memory ring), in an order that
+//   - walks the routed tiles M-tile-major, so the 128 activation rows of an M-tile are
+//     re-read from L2 by CTAs running at the same time while every weight tile streams
+//     from HBM once,
+//   - walks the shared-expert tiles N-block-major, so the CTAs running at the same time
+//     share one weight tile, and
+//   - interleaves the two kinds evenly: at small batch routed tiles are bound by the
+//     weight stream and shared-expert tiles by the tensor pipe, and mixing them keeps both
+//     busy.
 // GEMM-1's B tile is 128 gate rows + 128 up rows of the same expert, so one thread
 // holds gate and up of the same (row, column) in TMEM columns c and 128+c.
 // Every wait is bounded; on expiry the CTA records FMMOE_ERR_TIMEOUT and leaves.
@@ -25,12 +36,15 @@ namespace fmmoe {
 constexpr int G_BM = TC_BLOCK_M;   // 128
 constexpr int G_BK = 64;           // one 128-byte swizzle atom of bf16
 constexpr int G_STAGES = 4;
+constexpr int G_SCHED = 4;         // slots of the tile-id ring
 constexpr int G_A_BYTES = G_BM * G_BK * 2;          // 16 KB
 constexpr int G_B_BYTES = 2 * 128 * G_BK * 2;       // 32 KB (two 128-row boxes)
 constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;
 constexpr int G_THREADS = 192;
 constexpr int G_TMEM_COLS = 512;
-constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int G_EPI_LD = 33;                                 // padded row of the epilogue transpose buffer
+constexpr int G_EPI_BYTES = 4 * 32 * G_EPI_LD * 4;           // one 32x32 fp32 block per epilogue warp
+constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 
 struct Segment {          // routed experts (0) or shared experts (1)
   int n_nblocks;          // N-blocks per group
@@ -45,6 +59,7 @@ struct Segment {          // routed experts (0) or shared experts (1)
 struct GemmParams {
   const MTile* mtiles;        // routed M-tiles
   const int32_t* n_mtiles;    // device: number of routed M-tiles
+  int32_t* tile_counter;      // device: next tile to hand out (zero at launch)
   int n_experts;
   int shared_mtiles;          // N_s * ceil(T/128), host-known
   int mt_per_shared;          // ceil(T/128)
@@ -68,16 +83,23 @@ struct TileInfo {
   int seg, group_local, row0, rows, nb;
 };
 
+// Position `tile` of the interleaved order -> (segment, M-tile, N-block).
 __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, int tile, int n_mt_r) {
   TileInfo ti;
-  const int routed_tiles = n_mt_r * p.seg[0].n_nblocks;
-  if (tile < routed_tiles) {
+  const unsigned long long R = (unsigned long long)n_mt_r * p.seg[0].n_nblocks;
+  const unsigned long long S = (unsigned long long)p.shared_mtiles * p.seg[1].n_nblocks;
+  const unsigned long long N = R + S;
+  const unsigned long long sb = (unsigned long long)tile * S / N;          // shared tiles before this position
+  const unsigned long long sb1 = (unsigned long long)(tile + 1) * S / N;
+  if (sb1 == sb) {
+    const int r = tile - (int)sb;
+    const int mt = r / p.seg[0].n_nblocks;
     ti.seg = 0;
-    ti.nb = tile / n_mt_r;
-    const MTile m = p.mtiles[tile - ti.nb * n_mt_r];
+    ti.nb = r - mt * p.seg[0].n_nblocks;
+    const MTile m = p.mtiles[mt];
     ti.group_local = m.group; ti.row0 = m.row0; ti.rows = m.rows;
   } else {
-    const int t2 = tile - routed_tiles;
+    const int t2 = (int)sb;
     ti.seg = 1;
     ti.nb = t2 / p.shared_mtiles;
     const int mt = t2 - ti.nb * p.shared_mtiles;
@@ -100,12 +122,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char* smem = smem_raw + ((1024 - (raw & 1023)) & 1023);   // 1024-byte aligned tiles (128B swizzle)
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G_STAGES * G_STAGE_BYTES);
+  float* epi = reinterpret_cast<float*>(smem + G_STAGES * G_STAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G_STAGES * G_STAGE_BYTES + G_EPI_BYTES);
   uint64_t* full_bar = bars;                   // [G_STAGES]
   uint64_t* empty_bar = bars + G_STAGES;       // [G_STAGES]
   uint64_t* tfull_bar = bars + 2 * G_STAGES;   // [2]
   uint64_t* tempty_bar = tfull_bar + 2;        // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  uint64_t* sfull_bar = tempty_bar + 2;        // [G_SCHED]
+  uint64_t* sempty_bar = sfull_bar + G_SCHED;  // [G_SCHED]
+  volatile int* ring = reinterpret_cast<volatile int*>(sempty_bar + G_SCHED);   // [G_SCHED]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(ring) + G_SCHED);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -113,6 +139,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   if (threadIdx.x == 0) {
     for (int i = 0; i < G_STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&tfull_bar[i], 1); mbar_init(&tempty_bar[i], 128); }
+    for (int i = 0; i < G_SCHED; ++i) { mbar_init(&sfull_bar[i], 1); mbar_init(&sempty_bar[i], 5); }   // issuer + 4 epilogue warps
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -129,28 +156,46 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   const int total_tiles = n_mt_r * p.seg[0].n_nblocks + p.shared_mtiles * p.seg[1].n_nblocks;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------ scheduler + TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tmA_r); tma_prefetch_desc(&tmB0_r); tma_prefetch_desc(&tmB1_r);
       if (p.shared_mtiles) { tma_prefetch_desc(&tmA_s); tma_prefetch_desc(&tmB0_s); tma_prefetch_desc(&tmB1_s); }
+      const uint64_t pol_stream = l2_policy_evict_first();
+      const uint64_t pol_keep = l2_policy_evict_last();
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (uint32_t it = 0; ok; ++it) {
+        const int slot = it % G_SCHED;
+        const uint32_t sph = (it / G_SCHED) & 1;
+        if (!mbar_wait(&sempty_bar[slot], sph ^ 1, abort_flag)) { ok = false; break; }
+        int tile = atomicAdd(p.tile_counter, 1);
+        if (tile >= total_tiles) tile = -1;
+        ring[slot] = tile;
+        mbar_arrive(&sfull_bar[slot]);
+        if (tile < 0) break;
         const TileInfo ti = decode_tile(p, tile, n_mt_r);
         const Segment& sg = p.seg[ti.seg];
         const CUtensorMap* mA = ti.seg ? &tmA_s : &tmA_r;
         const CUtensorMap* mB0 = ti.seg ? &tmB0_s : &tmB0_r;
         const CUtensorMap* mB1 = ti.seg ? &tmB1_s : &tmB1_r;
+        // routed weights are read once per M-tile of their expert: let them leave L2 first;
+        // shared-expert weights are reused by every M-tile: default priority
+        const bool stream_b = ti.seg == 0;
         const int a_row = ti.row0 + ti.group_local * sg.a_group_stride;
         const int b_y0 = ti.group_local * sg.b_rows_per_group + ti.nb * (MODE == 0 ? 128 : 256);
         const int b_y1 = MODE == 0 ? b_y0 : b_y0 + 128;
         for (int kb = 0; kb < sg.k_blocks; ++kb) {
-          if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           unsigned char* sA = smem + stage * G_STAGE_BYTES;
           mbar_arrive_expect_tx(&full_bar[stage], G_STAGE_BYTES);
-          tma_load_2d(sA, mA, &full_bar[stage], kb * G_BK, a_row);
-          tma_load_2d(sA + G_A_BYTES, mB0, &full_bar[stage], kb * G_BK, b_y0);
-          tma_load_2d(sA + G_A_BYTES + G_B_BYTES / 2, mB1, &full_bar[stage], kb * G_BK, b_y1);
+          tma_load_2d_hint(sA, mA, &full_bar[stage], kb * G_BK, a_row, pol_keep);
+          if (stream_b) {
+            tma_load_2d_hint(sA + G_A_BYTES, mB0, &full_bar[stage], kb * G_BK, b_y0, pol_stream);
+            tma_load_2d_hint(sA + G_A_BYTES + G_B_BYTES / 2, mB1, &full_bar[stage], kb * G_BK, b_y1, pol_stream);
+          } else {
+            tma_load_2d(sA + G_A_BYTES, mB0, &full_bar[stage], kb * G_BK, b_y0);
+            tma_load_2d(sA + G_A_BYTES + G_B_BYTES / 2, mB1, &full_bar[stage], kb * G_BK, b_y1);
+          }
           if (++stage == G_STAGES) { stage = 0; phase ^= 1; }
         }
       }
@@ -163,14 +208,20 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
       int stage = 0; uint32_t phase = 0;
       int as = 0; uint32_t aphase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (uint32_t it = 0; ok; ++it) {
+        const int slot = it % G_SCHED;
+        const uint32_t sph = (it / G_SCHED) & 1;
+        if (!mbar_wait(&sfull_bar[slot], sph, abort_flag)) { ok = false; break; }
+        const int tile = ring[slot];
+        mbar_arrive(&sempty_bar[slot]);
+        if (tile < 0) break;
         const TileInfo ti = decode_tile(p, tile, n_mt_r);
         const int k_blocks = p.seg[ti.seg].k_blocks;
-        if (!mbar_wait(&tempty_bar[as], aphase ^ 1)) { ok = false; break; }
+        if (!mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + as * 256;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(&full_bar[stage], phase)) { ok = false; break; }
+          if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sA = smem_u32(smem + stage * G_STAGE_BYTES);
           const uint64_t da = umma_desc_sw128(sA);
@@ -191,18 +242,27 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int q = warp & 3;                 // TMEM lane quarter this warp may access
     const int r = q * 32 + lane;            // row of the tile held by this thread
+    float* stg = epi + q * 32 * G_EPI_LD;   // this warp's 32 x 32 transpose block
     int as = 0; uint32_t aphase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    for (uint32_t it = 0; ok; ++it) {
+      const int slot = it % G_SCHED;
+      const uint32_t sph = (it / G_SCHED) & 1;
+      if (!mbar_wait(&sfull_bar[slot], sph, abort_flag)) { ok = false; break; }
+      const int tile = ring[slot];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sempty_bar[slot]);
+      if (tile < 0) break;
       const TileInfo ti = decode_tile(p, tile, n_mt_r);
       const Segment& sg = p.seg[ti.seg];
-      if (!mbar_wait(&tfull_bar[as], aphase)) { ok = false; break; }
+      if (!mbar_wait(&tfull_bar[as], aphase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + as * 256 + (static_cast<uint32_t>(q * 32) << 16);
-      const bool row_ok = r < ti.rows;
+      const int rows_w = ti.rows - q * 32;   // valid rows among this warp's 32 (may be <= 0)
+      const long long out_row0 = (long long)ti.row0 + q * 32 + (long long)ti.group_local * sg.out_group_stride;
       if (MODE == 0) {
-        const long long out_row = (long long)ti.row0 + r + (long long)ti.group_local * sg.out_group_stride;
-        __nv_bfloat16* dst = p.act[ti.seg] + out_row * sg.ld_out + ti.nb * 128;
+        uint32_t* stg32 = reinterpret_cast<uint32_t*>(stg);   // [32][17] packed bf16 pairs
+        __nv_bfloat16* dst0 = p.act[ti.seg] + out_row0 * sg.ld_out + ti.nb * 128;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
           if (ti.nb * 128 + c * 32 >= sg.n_valid) break;   // warp-uniform
@@ -210,57 +270,65 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
           tmem_ld32(taddr + c * 32, g);
           tmem_ld32(taddr + 128 + c * 32, u);
           tmem_ld_wait();
-          uint32_t o[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
             const float a0 = g0 / (1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
             const float a1 = g1 / (1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
             const __nv_bfloat162 h = __floats2bfloat162_rn(a0, a1);
-            o[i] = *reinterpret_cast<const uint32_t*>(&h);
+            stg32[lane * 17 + i] = *reinterpret_cast<const uint32_t*>(&h);
           }
-          if (row_ok) {
-            uint4* d4 = reinterpret_cast<uint4*>(dst + c * 32);
+          __syncwarp();
+          // 4 lanes x 16 bytes cover the 64-byte row segment; 8 rows per instruction
 #pragma unroll
-            for (int i = 0; i < 4; ++i) d4[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+          for (int rr = 0; rr < 4; ++rr) {
+            const int row = rr * 8 + (lane >> 2);
+            const int w4 = (lane & 3) * 4;
+            if (row < rows_w) {
+              const uint32_t* sp = stg32 + row * 17 + w4;
+              *reinterpret_cast<uint4*>(dst0 + (long long)row * sg.ld_out + c * 32 + w4 * 2) =
+                  make_uint4(sp[0], sp[1], sp[2], sp[3]);
+            }
           }
+          __syncwarp();
         }
       } else {
-        long long tok; float gate;
+        int tok; float gate;
         if (ti.seg == 0) {
+          const bool row_ok = lane < rows_w;
           tok = row_ok ? p.row_token[ti.row0 + r] : 0;
           gate = row_ok ? p.row_gate[ti.row0 + r] : 0.f;
         } else {
           tok = ti.row0 + r; gate = 1.f;
         }
-        float* dst;
-        if (p.deterministic) {
-          const long long out_row = (long long)ti.row0 + r + (long long)ti.group_local * sg.out_group_stride;
-          dst = p.y[ti.seg] + out_row * sg.ld_out + ti.nb * 256;
-          gate = 1.f;   // gates are applied by the ordered gather
-        } else {
-          dst = p.acc + tok * sg.ld_out + ti.nb * 256;
-        }
+        if (p.deterministic) gate = 1.f;   // gates are applied by the ordered gather
+        float* ybase = p.deterministic ? p.y[ti.seg] + out_row0 * sg.ld_out + ti.nb * 256 : nullptr;
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
           if (ti.nb * 256 + c * 32 >= sg.n_valid) break;   // warp-uniform
           uint32_t v[32];
           tmem_ld32(taddr + c * 32, v);
           tmem_ld_wait();
-          if (row_ok) {
-            if (p.deterministic) {
-              float4* d4 = reinterpret_cast<float4*>(dst + c * 32);
 #pragma unroll
-              for (int i = 0; i < 8; ++i)
-                d4[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                    __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-            } else {
+          for (int j = 0; j < 32; ++j) stg[lane * G_EPI_LD + j] = gate * __uint_as_float(v[j]);
+          __syncwarp();
+          // 8 lanes x 16 bytes cover a row's 128-byte segment; 4 rows per instruction
 #pragma unroll
-              for (int i = 0; i < 8; ++i)
-                red_add_v4(dst + c * 32 + 4 * i, gate * __uint_as_float(v[4 * i]), gate * __uint_as_float(v[4 * i + 1]),
-                           gate * __uint_as_float(v[4 * i + 2]), gate * __uint_as_float(v[4 * i + 3]));
+          for (int rr = 0; rr < 8; ++rr) {
+            const int row = rr * 4 + (lane >> 3);
+            const int col = (lane & 7) * 4;
+            const int tok_r = __shfl_sync(0xffffffffu, tok, row);
+            if (row < rows_w) {
+              const float* sp = stg + row * G_EPI_LD + col;
+              if (p.deterministic) {
+                *reinterpret_cast<float4*>(ybase + (long long)row * sg.ld_out + c * 32 + col) =
+                    make_float4(sp[0], sp[1], sp[2], sp[3]);
+              } else {
+                red_add_v4(p.acc + (long long)tok_r * sg.ld_out + ti.nb * 256 + c * 32 + col, sp[0], sp[1], sp[2], sp[3]);
+              }
             }
           }
+          __syncwarp();
         }
       }
       tc_fence_before();
@@ -338,12 +406,14 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   p1.seg[1] = Segment{Ns ? (Is + 127) / 128 : 0, H / G_BK, Is, Is, 0, (int)a.T, Is};
   p1.act[0] = static_cast<__nv_bfloat16*>(a.act); p1.act[1] = static_cast<__nv_bfloat16*>(a.act_sh);
   p1.status = a.d_status;
+  p1.tile_counter = a.tile_counters;
 
   GemmParams p2 = p1;
   p2.seg[0] = Segment{(H + 255) / 256, I / G_BK, H, H, 0, 0, H};
   p2.seg[1] = Segment{Ns ? (H + 255) / 256 : 0, Ns ? Is / G_BK : 0, H, H, (int)a.T, (int)a.T, H};
   p2.row_token = a.row_token; p2.row_gate = a.row_gate; p2.acc = a.acc;
   p2.y[0] = a.y; p2.y[1] = a.ysh; p2.deterministic = a.deterministic;
+  p2.tile_counter = a.tile_counters + 1;
 
   if (!h->tc_attr_set) {
     FMMOE_CUDA_TRY(cudaFuncSetAttribute(ffn_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES));

@@ -48,7 +48,7 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 struct WsPlan {
   size_t zero_off, zero_bytes;  // region cleared at the start of every call
   size_t counts_off;            // int32 [FMMOE_MAX_EXPERTS] expert histogram
-  size_t misc_off;              // int32 [8]: [0] number of routed M-tiles
+  size_t misc_off;              // int32 [8]: [0] number of routed M-tiles, [1],[2] GEMM tile counters
   size_t acc_off;               // fp32 [T,H] combine accumulator (atomic mode)
   size_t topk_idx_off, topk_w_off, inv_row_off;
   size_t expert_off_off, row_token_off, row_gate_off, mtiles_off;
@@ -112,6 +112,7 @@ struct FfnArgs {   // both paths
   const fmmoe_layer_desc* d; const fmmoe_weights* w;
   const void* x; int64_t T; int64_t p_max;
   const MTile* mtiles; const int32_t* n_mtiles; int32_t max_mtiles;
+  int32_t* tile_counters;   // [2] zeroed per call: tile schedulers of GEMM-1 and GEMM-2
   const int32_t* row_token; const float* row_gate;
   void* xp; void* act; void* act_sh;
   float* acc;            // atomic mode
