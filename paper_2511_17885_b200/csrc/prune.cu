@@ -4,10 +4,11 @@
 //                        attention sum (Eq. 11); one warp per window, fp64 accumulation
 //   select_kernel      : per sequence, A_bar (Eq. 12), C (Eq. 13) rounded once to fp32,
 //                        merge set = m highest C (Eq. 15), drop set = d smallest A_bar among
-//                        the rest, then the stable compaction map (scan of keep flags)
+//                        the rest (both by an in-CTA bitonic sort of (score, window) keys),
+//                        then the stable compaction map (scan of keep flags)
 //   compact_kernel     : copies kept rows; a merged window becomes mean(rows) rescaled to the
 //                        largest member norm (Eq. 16-18) at its first token's position
-// Ranks are computed by counting, on (value, index) pairs, so the keep-set does not depend
+// Ranks come from sorting unique (value, window index) keys, so the keep-set does not depend
 // on thread order; ties go to the lower window index.
 #include <cuda_bf16.h>
 #include <math.h>
@@ -171,18 +172,45 @@ __global__ void __launch_bounds__(256) window_score_kernel(const PruneDev a, con
 }
 
 // ------------------------------------------------------------------ select + compaction map
+// Order-preserving map float -> uint32 (-0 is folded onto +0 so that equal values tie).
+__device__ __forceinline__ uint32_t ordered_bits(float f) {
+  if (f == 0.f) f = 0.f;
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Ascending bitonic sort of n (a power of two) 64-bit keys in shared memory by the whole CTA.
+// Keys are unique (the window index is part of them), so the result does not depend on the
+// network's comparison order.
+__device__ __forceinline__ void bitonic_sort_u64(unsigned long long* keys, int n) {
+  for (int k = 2; k <= n; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int idx = threadIdx.x; idx < n; idx += blockDim.x) {
+        const int ixj = idx ^ j;
+        if (ixj > idx) {
+          const unsigned long long x = keys[idx], y = keys[ixj];
+          const bool up = (idx & k) == 0;
+          if ((x > y) == up) { keys[idx] = y; keys[ixj] = x; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// One CTA per sequence.  Eq. 12-13 (one rounding to fp32), then the merge set (Eq. 15) and the
+// drop set by SORTING (score, window index) keys: position p of the sorted order is rank p.
 __global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const PruneSeqs sq) {
-  extern __shared__ float s_f[];   // C32[n_f], A32[n_f]
+  extern __shared__ unsigned long long s_keys[];   // [n_pad]
   __shared__ double s_red[32];
   __shared__ int s_warp[32];
-  __shared__ int s_running;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_f = sq.n_vis[b] / a.W;
   const int w0 = sq.win_off[b];
   const int m = sq.m[b], d = sq.d[b];
-  float* C32 = s_f;
-  float* A32 = s_f + n_f;
   const bool have_attn = a.attn != nullptr;
+  int n_pad = 2;
+  while (n_pad < n_f) n_pad <<= 1;
 
   // Eq. 12: divide by the largest window sum (0 if all sums are 0)
   double amax = 0.0;
@@ -195,98 +223,101 @@ __global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const Pr
     amax = s_red[0];
     for (int i = 1; i < 32; ++i) amax = fmax(amax, s_red[i]);
   }
-  for (int i = tid; i < n_f; i += 1024) {
-    const double S = a.sim[w0 + i];
-    if (have_attn) {
-      const double ab = amax > 0.0 ? a.asum[w0 + i] / amax : 0.0;
-      // Eq. 13 in fp64 without contraction, then ONE rounding to fp32
-      const double c = __dsub_rn(__dmul_rn(a.alpha, S), __dmul_rn(__dsub_rn(1.0, a.alpha), ab));
-      C32[i] = (float)c;
-      A32[i] = (float)ab;
-    } else {
-      C32[i] = (float)S;
-      A32[i] = 0.f;
-    }
-  }
-  __syncthreads();
-  // ranks by counting
-  for (int i = tid; i < n_f; i += 1024) {
-    const float ci = C32[i];
-    int rc = 0;
-    for (int j = 0; j < n_f; ++j) {
-      const float cj = C32[j];
-      rc += (cj > ci) || (cj == ci && j < i);
-    }
-    uint8_t act = 0;
-    if (rc < m) act = 1;
-    else if (!have_attn && rc < m + d) act = 2;
-    a.action[w0 + i] = act;
-  }
-  if (have_attn && d > 0) {
-    __syncthreads();
-    for (int i = tid; i < n_f; i += 1024) {
-      if (a.action[w0 + i] == 1) continue;
-      const float ai = A32[i];
-      int ra = 0;
-      for (int j = 0; j < n_f; ++j) {
-        if (a.action[w0 + j] == 1) continue;
-        const float aj = A32[j];
-        ra += (aj < ai) || (aj == ai && j < i);
+  // keys of the redundancy ranking: (C descending, window ascending)
+  for (int i = tid; i < n_pad; i += 1024) {
+    unsigned long long key = ~0ull;
+    if (i < n_f) {
+      const double S = a.sim[w0 + i];
+      float c32;
+      if (have_attn) {
+        const double ab = amax > 0.0 ? a.asum[w0 + i] / amax : 0.0;
+        // Eq. 13 in fp64 without contraction, then ONE rounding to fp32
+        c32 = (float)__dsub_rn(__dmul_rn(a.alpha, S), __dmul_rn(__dsub_rn(1.0, a.alpha), ab));
+      } else {
+        c32 = (float)S;
       }
-      if (ra < d) a.action[w0 + i] = 2;   // concurrent readers only test for "== 1"
+      key = ((unsigned long long)(~ordered_bits(c32)) << 32) | (unsigned)i;
+      a.action[w0 + i] = 0;
     }
+    s_keys[i] = key;
   }
   __syncthreads();
-
-  // stable compaction map over the sequence's tokens
-  const long long lo = sq.seq_off[b], hi = sq.seq_off[b + 1];
-  if (tid == 0) s_running = 0;
-  __syncthreads();
-  for (long long t0 = lo; t0 < hi; t0 += 1024) {
-    const long long t = t0 + tid;
-    int kd = -1;   // kind of the emitted row, -1 = nothing emitted
-    if (t < hi) {
-      const int v = a.vrank[t];
-      if (v < 0) kd = 0;
-      else {
-        const int w = v / a.W;
-        if (w >= n_f) kd = 1;
-        else {
-          const uint8_t act = a.action[w0 + w];
-          if (act == 0) kd = 1;
-          else if (act == 1 && v - w * a.W == 0) kd = 2;
+  if (m + d > 0) {
+    bitonic_sort_u64(s_keys, n_pad);
+    const int n_act = have_attn ? m : m + d;
+    for (int p = tid; p < n_act && p < n_f; p += 1024)
+      a.action[w0 + (int)(s_keys[p] & 0xffffffffu)] = p < m ? 1 : 2;
+    __syncthreads();
+    if (have_attn && d > 0) {
+      // drop ranking among the windows that were not merged: (A_bar ascending, window ascending)
+      for (int i = tid; i < n_pad; i += 1024) {
+        unsigned long long key = ~0ull;
+        if (i < n_f && a.action[w0 + i] == 0) {
+          const float a32 = (float)(amax > 0.0 ? a.asum[w0 + i] / amax : 0.0);
+          key = ((unsigned long long)ordered_bits(a32) << 32) | (unsigned)i;
         }
+        s_keys[i] = key;
       }
+      __syncthreads();
+      bitonic_sort_u64(s_keys, n_pad);
+      for (int p = tid; p < d && p < n_f - m; p += 1024)
+        a.action[w0 + (int)(s_keys[p] & 0xffffffffu)] = 2;
+      __syncthreads();
     }
-    const unsigned bal = __ballot_sync(0xffffffffu, kd >= 0);
-    if (lane == 0) s_warp[warp] = __popc(bal);
-    __syncthreads();
-    if (warp == 0) {
-      int c = s_warp[lane];
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, c, o);
-        if (lane >= o) c += n;
-      }
-      s_warp[lane] = c;
-    }
-    __syncthreads();
-    const int running = s_running;
-    if (kd >= 0) {
-      const long long pos = sq.out_off[b] + running + (warp ? s_warp[warp - 1] : 0) + __popc(bal & ((1u << lane) - 1u));
-      if (pos < sq.out_off[b + 1]) {
-        a.keep_idx_ws[pos] = (int32_t)t;
-        a.kind_ws[pos] = (uint8_t)kd;
-        if (a.keep_idx) a.keep_idx[pos] = (int32_t)t;
-        if (a.kind) a.kind[pos] = (uint8_t)kd;
-        if (a.is_visual_out) a.is_visual_out[pos] = kd != 0;
-      }
-    }
-    __syncthreads();
-    if (tid == 0) s_running = running + s_warp[31];
-    __syncthreads();
   }
-  if (tid == 0 && s_running != (int)(sq.out_off[b + 1] - sq.out_off[b])) atomicCAS(a.status, 0, DEV_INTERNAL);
+
+  // stable compaction map over the sequence's tokens: every thread owns a run of consecutive tokens
+  const long long lo = sq.seq_off[b], hi = sq.seq_off[b + 1];
+  const int per = (int)((hi - lo + 1023) / 1024);
+  const long long t_begin = lo + (long long)tid * per;
+  auto kind_of = [&](long long t) -> int {   // kind of the emitted row, -1 = nothing emitted
+    const int v = a.vrank[t];
+    if (v < 0) return 0;
+    const int w = v / a.W;
+    if (w >= n_f) return 1;
+    const uint8_t act = a.action[w0 + w];
+    if (act == 0) return 1;
+    return (act == 1 && v - w * a.W == 0) ? 2 : -1;
+  };
+  int cnt = 0;
+  for (int i = 0; i < per; ++i) {
+    const long long t = t_begin + i;
+    if (t < hi && kind_of(t) >= 0) ++cnt;
+  }
+  int incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int c = s_warp[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, c, o);
+      if (lane >= o) c += n;
+    }
+    s_warp[lane] = c;
+  }
+  __syncthreads();
+  long long pos = sq.out_off[b] + (warp ? s_warp[warp - 1] : 0) + (incl - cnt);
+  for (int i = 0; i < per; ++i) {
+    const long long t = t_begin + i;
+    if (t >= hi) break;
+    const int kd = kind_of(t);
+    if (kd < 0) continue;
+    if (pos < sq.out_off[b + 1]) {
+      a.keep_idx_ws[pos] = (int32_t)t;
+      a.kind_ws[pos] = (uint8_t)kd;
+      if (a.keep_idx) a.keep_idx[pos] = (int32_t)t;
+      if (a.kind) a.kind[pos] = (uint8_t)kd;
+      if (a.is_visual_out) a.is_visual_out[pos] = kd != 0;
+    }
+    ++pos;
+  }
+  if (tid == 0 && s_warp[31] != (int)(sq.out_off[b + 1] - sq.out_off[b])) atomicCAS(a.status, 0, DEV_INTERNAL);
 }
 
 // ------------------------------------------------------------------ gather / merge rows
@@ -495,7 +526,9 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
   if (((uintptr_t)x | (uintptr_t)x_out | (uintptr_t)probs) & 15) return FMMOE_ERR_INVALID_ARG;
   const PruneWs wp = plan_prune(T);
   if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < wp.total) return FMMOE_ERR_WORKSPACE;
-  const size_t sel_smem = (size_t)max_nf * 8;
+  size_t sel_pad = 2;
+  while ((int64_t)sel_pad < max_nf) sel_pad <<= 1;
+  const size_t sel_smem = sel_pad * 8;   // sort keys of the longest sequence's windows
   if (sel_smem > (size_t)h->max_smem_optin - 1024) return FMMOE_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);

@@ -1,22 +1,23 @@
 // Router: logits (Eq. 1), softmax (Eq. 2), modality-aware top-k (Eq. 3, with K_v
 // for vision tokens once the layer has reached l_v) and renormalised gates (Eq. 5),
-// fused in one kernel.  A CTA owns 32 tokens: the logits tile [32, E] is formed in
-// shared memory (bf16: mma.sync tensor-core tiles fed by a cp.async pipeline; fp32:
-// plain FMA), then each warp takes 8 tokens and runs the softmax / top-k / gate
-// step across the expert dimension with warp shuffles.  The kernel also adds the
-// selections to the per-expert histogram the permutation needs.
+// fused in one kernel per storage type.
+//   bf16: the logits tile [128 tokens, E] is a tcgen05 GEMM fed by TMA with its accumulator
+//         in tensor memory; one thread per token then reads its row back and runs the
+//         softmax / top-k / gate step on it.
+//   fp32: a CTA owns 32 tokens, forms their logits with plain FMA in shared memory (TF32
+//         would miss an fp32 tolerance), then each warp takes 8 tokens and runs the
+//         softmax / top-k / gate step across the expert dimension with warp shuffles.
+// Both kernels also add the selections to the per-expert histogram the permutation needs.
 #include <cuda_bf16.h>
 #include <float.h>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace fmmoe {
 
 constexpr int R_BM = 32;
 constexpr int R_THREADS = 128;
-constexpr int R_BK = 64;
-constexpr int R_LDS = R_BK + 8;   // bf16 elements per smem row (144 B: conflict-free ldmatrix)
-constexpr int R_STAGES = 3;
 
 struct RouteDev {
   const void* x; const void* w; const float* bias; const uint8_t* is_visual;
@@ -108,110 +109,249 @@ __device__ __forceinline__ void flush_hist(const int* hist, const RouteDev& a) {
       if (hist[e]) atomicAdd(&a.counts[e], hist[e]);
 }
 
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N)); }
+// ---------------------------------------------------------------------------------------
+// bf16 router on the tcgen05 tensor cores.  A CTA owns 128 tokens:
+//   warp 0    : TMA producer  (X tile 128x64 and the router matrix tile e_pad x 64 per stage)
+//   warp 1    : UMMA issuer   (128 x e_pad x 16 tcgen05.mma; the logits tile lives in TMEM)
+//   warps 2-5 : one thread per token row reads its logits back from TMEM in 32-column chunks
+//               and runs bias + softmax + top-k + gates on them (the chunks are re-read per
+//               pass instead of being held in registers: tensor memory is cheap to read).
+// The router matrix is read once per 128 tokens (from L2 after the first CTA), X once.
+// ---------------------------------------------------------------------------------------
+constexpr int RT_BM = 128;
+constexpr int RT_BK = 64;
+constexpr int RT_THREADS = 192;
+constexpr int RT_A_BYTES = RT_BM * RT_BK * 2;
+constexpr int RT_MAX_STAGES = 8;
 
-// bf16 router.  NT = n8-tiles per warp = e_pad / 32.
-template <int NT>
-__global__ void __launch_bounds__(R_THREADS) route_bf16_kernel(const RouteDev a) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int e_pad = NT * 32;
-  const int ldl = e_pad + 1;
-  __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);                    // [STAGES][R_BM][R_LDS]
-  __nv_bfloat16* Ws = Xs + R_STAGES * R_BM * R_LDS;                                   // [STAGES][e_pad][R_LDS]
-  float* Ls = reinterpret_cast<float*>(Ws + R_STAGES * e_pad * R_LDS);                // [R_BM][ldl]
-  int* hist = reinterpret_cast<int*>(Ls + R_BM * ldl);                                // [e_pad]
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const long long t0 = (long long)blockIdx.x * R_BM;
-  const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(a.x);
-  const __nv_bfloat16* W = static_cast<const __nv_bfloat16*>(a.w);
+__device__ __forceinline__ float route_logit(uint32_t raw, const float* bias_s, int e) { return __uint_as_float(raw) + bias_s[e]; }
 
-  // rows that are never loaded (tokens >= T, experts >= E) must read as zero
-  for (int i = tid; i < R_STAGES * (R_BM + e_pad) * R_LDS / 8; i += R_THREADS)
-    reinterpret_cast<uint4*>(smem_raw)[i] = make_uint4(0, 0, 0, 0);
-  for (int i = tid; i < e_pad; i += R_THREADS) hist[i] = 0;
-  __syncthreads();
-
-  const int kblocks = a.H / R_BK;
-  auto load_stage = [&](int st, int kb) {
-    const int k0 = kb * R_BK;
-    for (int c = tid; c < R_BM * (R_BK / 8); c += R_THREADS) {
-      const int r = c >> 3, cc = c & 7;
-      if (t0 + r < a.T) cp_async16(Xs + (st * R_BM + r) * R_LDS + cc * 8, X + (t0 + r) * a.H + k0 + cc * 8);
+template <int NCH>   // NCH = number of 32-column chunks that cover E
+__device__ __forceinline__ void route_tail_tmem(uint32_t taddr, const float* bias_s, int* hist, long long t,
+                                                const RouteDev& a) {
+  const bool tok_ok = t < a.T;
+  const int E = a.E;
+  const bool vec4 = (E & 3) == 0;
+  // pass 1: row maximum (and the logits themselves, if wanted)
+  float m = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) {
+    uint32_t v[32];
+    tmem_ld32(taddr + c * 32, v);
+    tmem_ld_wait();
+    float z[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const int e = c * 32 + j;
+      z[j] = e < E ? route_logit(v[j], bias_s, e) : -INFINITY;
+      m = fmaxf(m, z[j]);
     }
-    for (int c = tid; c < a.E * (R_BK / 8); c += R_THREADS) {
-      const int r = c >> 3, cc = c & 7;
-      cp_async16(Ws + (st * e_pad + r) * R_LDS + cc * 8, W + (long long)r * a.H + k0 + cc * 8);
-    }
-  };
-
-  float acc[2][NT][4];
+    if (a.logits && tok_ok) {
+      float* dst = a.logits + t * E + c * 32;
+      if (vec4) {
 #pragma unroll
-  for (int mi = 0; mi < 2; ++mi)
+        for (int j = 0; j < 32; j += 4)
+          if (c * 32 + j < E) *reinterpret_cast<float4*>(dst + j) = make_float4(z[j], z[j + 1], z[j + 2], z[j + 3]);
+      } else {
 #pragma unroll
-    for (int ni = 0; ni < NT; ++ni)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) acc[mi][ni][q] = 0.f;
-
-  for (int s = 0; s < R_STAGES - 1; ++s) {
-    if (s < kblocks) load_stage(s, s);
-    cp_async_commit();
-  }
-  for (int kb = 0; kb < kblocks; ++kb) {
-    cp_async_wait<R_STAGES - 2>();
-    __syncthreads();
-    if (kb + R_STAGES - 1 < kblocks) load_stage((kb + R_STAGES - 1) % R_STAGES, kb + R_STAGES - 1);
-    cp_async_commit();
-    const int st = kb % R_STAGES;
-    const __nv_bfloat16* xs = Xs + st * R_BM * R_LDS;
-    const __nv_bfloat16* ws = Ws + st * e_pad * R_LDS;
-#pragma unroll
-    for (int ks = 0; ks < R_BK / 16; ++ks) {
-      uint32_t af[2][4];
-#pragma unroll
-      for (int mi = 0; mi < 2; ++mi) {
-        const uint32_t addr = (uint32_t)__cvta_generic_to_shared(xs + (mi * 16 + (lane & 15)) * R_LDS + ks * 16 + (lane >> 4) * 8);
-        asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                     : "=r"(af[mi][0]), "=r"(af[mi][1]), "=r"(af[mi][2]), "=r"(af[mi][3]) : "r"(addr));
+        for (int j = 0; j < 32; ++j)
+          if (c * 32 + j < E) dst[j] = z[j];
       }
+    }
+  }
+  // pass 2: softmax denominator
+  float s = 0.f;
 #pragma unroll
-      for (int ni = 0; ni < NT; ++ni) {
-        const int n0 = warp * (NT * 8) + ni * 8;
-        uint32_t b0, b1;
-        const uint32_t addr = (uint32_t)__cvta_generic_to_shared(ws + (n0 + (lane & 7)) * R_LDS + ks * 16 + ((lane >> 3) & 1) * 8);
-        asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
+  for (int c = 0; c < NCH; ++c) {
+    uint32_t v[32];
+    tmem_ld32(taddr + c * 32, v);
+    tmem_ld_wait();
 #pragma unroll
-        for (int mi = 0; mi < 2; ++mi) {
-          asm volatile(
-              "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-              : "+f"(acc[mi][ni][0]), "+f"(acc[mi][ni][1]), "+f"(acc[mi][ni][2]), "+f"(acc[mi][ni][3])
-              : "r"(af[mi][0]), "r"(af[mi][1]), "r"(af[mi][2]), "r"(af[mi][3]), "r"(b0), "r"(b1));
+    for (int j = 0; j < 32; ++j) {
+      const int e = c * 32 + j;
+      if (e < E) s += __expf(route_logit(v[j], bias_s, e) - m);
+    }
+  }
+  // pass 3: probabilities (Eq. 2), only when the caller wants them (pruning layers)
+  if (a.probs) {
+    const float inv = 1.f / s;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      uint32_t v[32];
+      tmem_ld32(taddr + c * 32, v);
+      tmem_ld_wait();
+      float pr[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const int e = c * 32 + j;
+        pr[j] = e < E ? __expf(route_logit(v[j], bias_s, e) - m) * inv : 0.f;
+      }
+      if (tok_ok) {
+        float* dst = a.probs + t * E + c * 32;
+        if (vec4) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            if (c * 32 + j < E) *reinterpret_cast<float4*>(dst + j) = make_float4(pr[j], pr[j + 1], pr[j + 2], pr[j + 3]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c * 32 + j < E) dst[j] = pr[j];
         }
       }
     }
   }
-  cp_async_wait<0>();
-  // logits tile (+ bias) to shared memory
-  const int g = lane >> 2, tg = lane & 3;
+  // top-k (Eq. 3): k_t rounds of "largest logit not taken yet"; scanning upwards with a strict
+  // comparison gives equal logits to the lower expert index
+  const int k_t = tok_ok ? ((a.reduce_on && a.is_visual[t]) ? a.Kv : a.K) : 0;
+  uint32_t taken[NCH];
 #pragma unroll
-  for (int mi = 0; mi < 2; ++mi)
+  for (int c = 0; c < NCH; ++c) taken[c] = 0;
+  float denom = 0.f;
+  int32_t* oi = a.topk_idx + t * a.K;
+  float* ow = a.topk_w + t * a.K;
+  const int k_warp = __reduce_max_sync(0xffffffffu, k_t);   // tmem loads are warp-collective
+  for (int i = 0; i < k_warp; ++i) {
+    float best = -INFINITY;
+    int be = -1;
 #pragma unroll
-    for (int ni = 0; ni < NT; ++ni) {
-      const int col = warp * (NT * 8) + ni * 8 + 2 * tg;
-      const float b0 = (a.bias && col < a.E) ? a.bias[col] : 0.f;
-      const float b1 = (a.bias && col + 1 < a.E) ? a.bias[col + 1] : 0.f;
-      Ls[(mi * 16 + g) * ldl + col] = acc[mi][ni][0] + b0;
-      Ls[(mi * 16 + g) * ldl + col + 1] = acc[mi][ni][1] + b1;
-      Ls[(mi * 16 + g + 8) * ldl + col] = acc[mi][ni][2] + b0;
-      Ls[(mi * 16 + g + 8) * ldl + col + 1] = acc[mi][ni][3] + b1;
+    for (int c = 0; c < NCH; ++c) {
+      uint32_t v[32];
+      tmem_ld32(taddr + c * 32, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const int e = c * 32 + j;
+        const float z = route_logit(v[j], bias_s, e < E ? e : 0);
+        if (e < E && !((taken[c] >> j) & 1u) && (z > best || be < 0)) { best = z; be = e; }
+      }
     }
+    if (i < k_t) {
+#pragma unroll
+      for (int c = 0; c < NCH; ++c)
+        if (c == (be >> 5)) taken[c] |= 1u << (be & 31);
+      const float p = __expf(best - m);
+      denom += p;
+      oi[i] = be;
+      ow[i] = p;          // unnormalised; rescaled below
+      if (a.counts) atomicAdd(&hist[be], 1);
+    }
+  }
+  if (tok_ok) {
+    for (int i = 0; i < a.K; ++i) {
+      if (i < k_t) ow[i] = ow[i] / denom;     // Eq. 5
+      else { oi[i] = -1; ow[i] = 0.f; }
+      if (a.inv_row) a.inv_row[t * a.K + i] = -1;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(RT_THREADS, 1)
+route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const RouteDev a,
+                const int stages, const int tmem_cols, int* status) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  unsigned char* smem = smem_raw + ((1024 - (raw & 1023)) & 1023);
+  const int b_bytes = a.e_pad * RT_BK * 2;
+  const int stage_bytes = RT_A_BYTES + b_bytes;
+  float* bias_s = reinterpret_cast<float*>(smem + stages * stage_bytes);   // [256]
+  int* hist = reinterpret_cast<int*>(bias_s + FMMOE_MAX_EXPERTS);           // [256]
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(hist + FMMOE_MAX_EXPERTS);
+  uint64_t* empty_bar = full_bar + RT_MAX_STAGES;
+  uint64_t* tfull_bar = empty_bar + RT_MAX_STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfull_bar + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kblocks = a.H / RT_BK;
+
+  for (int e = threadIdx.x; e < FMMOE_MAX_EXPERTS; e += RT_THREADS) {
+    bias_s[e] = (a.bias && e < a.E) ? a.bias[e] : 0.f;
+    hist[e] = 0;
+  }
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < stages; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
+    mbar_init(tfull_bar, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, (uint32_t)tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
   __syncthreads();
-  route_tail<NT>(Ls, ldl, t0, a, hist);
-  flush_hist(hist, a);
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int row0 = blockIdx.x * RT_BM;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmW);
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = 0; kb < kblocks; ++kb) {
+        if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+        unsigned char* sA = smem + stage * stage_bytes;
+        mbar_arrive_expect_tx(&full_bar[stage], (uint32_t)stage_bytes);
+        tma_load_2d(sA, &tmX, &full_bar[stage], kb * RT_BK, row0);
+        tma_load_2d(sA + RT_A_BYTES, &tmW, &full_bar[stage], kb * RT_BK, 0);
+        if (++stage == stages) { stage = 0; phase ^= 1; }
+      }
+      if (!ok) { atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(RT_BM, a.e_pad);
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = 0; kb < kblocks; ++kb) {
+        if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sA = smem_u32(smem + stage * stage_bytes);
+        const uint64_t da = umma_desc_sw128(sA);
+        const uint64_t db = umma_desc_sw128(sA + RT_A_BYTES);
+#pragma unroll
+        for (int k = 0; k < RT_BK / 16; ++k) umma_bf16(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+        umma_commit(&empty_bar[stage]);
+        if (++stage == stages) { stage = 0; phase ^= 1; }
+      }
+      if (ok) umma_commit(tfull_bar);
+      else { atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+    }
+  } else {
+    const int q = warp & 3;
+    const long long t = (long long)row0 + q * 32 + lane;
+    if (mbar_wait(tfull_bar, 0, abort_flag)) {
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+      switch ((a.E + 31) / 32) {
+        case 1: route_tail_tmem<1>(taddr, bias_s, hist, t, a); break;
+        case 2: route_tail_tmem<2>(taddr, bias_s, hist, t, a); break;
+        case 3: route_tail_tmem<3>(taddr, bias_s, hist, t, a); break;
+        case 4: route_tail_tmem<4>(taddr, bias_s, hist, t, a); break;
+        case 5: route_tail_tmem<5>(taddr, bias_s, hist, t, a); break;
+        case 6: route_tail_tmem<6>(taddr, bias_s, hist, t, a); break;
+        case 7: route_tail_tmem<7>(taddr, bias_s, hist, t, a); break;
+        default: route_tail_tmem<8>(taddr, bias_s, hist, t, a); break;
+      }
+    } else {
+      atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1;
+    }
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) { }
+    __syncthreads();
+  }
+  if (a.counts)
+    for (int e = threadIdx.x; e < a.E; e += RT_THREADS)
+      if (hist[e]) atomicAdd(&a.counts[e], hist[e]);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
+  }
 }
 
 // fp32 router (no tensor cores: TF32 would miss the fp32 tolerance).  Thread (warp w,
@@ -272,18 +412,53 @@ __global__ void __launch_bounds__(R_THREADS) route_f32_kernel(const RouteDev a) 
   flush_hist(hist, a);
 }
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static bool route_map(fmmoe_handle* h, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {RT_BK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return reinterpret_cast<EncodeTiledFn>(h->encode_tiled)(
+             m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s) {
+  if (!h->encode_tiled) return FMMOE_ERR_CUDA;
+  d.e_pad = (d.E + 15) / 16 * 16;                       // UMMA N: a multiple of 16 for M = 128
+  const int stage_bytes = RT_A_BYTES + d.e_pad * RT_BK * 2;
+  int stages = (200 * 1024) / stage_bytes;
+  if (stages > RT_MAX_STAGES) stages = RT_MAX_STAGES;
+  const int kblocks = d.H / RT_BK;
+  if (stages > kblocks) stages = kblocks;
+  if (stages < 1) return FMMOE_ERR_UNSUPPORTED;
+  int tmem_cols = 32;
+  while (tmem_cols < (d.E + 31) / 32 * 32) tmem_cols *= 2;
+  const size_t smem = (size_t)stages * stage_bytes + FMMOE_MAX_EXPERTS * 8 + (2 * RT_MAX_STAGES + 1) * 8 + 16 + 1024;
+  CUtensorMap mx, mw;
+  if (!route_map(h, &mx, d.x, (uint64_t)d.T, (uint64_t)d.H, RT_BM)) return FMMOE_ERR_CUDA;
+  if (!route_map(h, &mw, d.w, (uint64_t)d.E, (uint64_t)d.H, (uint32_t)d.e_pad)) return FMMOE_ERR_CUDA;
+  FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const int grid = (int)((d.T + RT_BM - 1) / RT_BM);
+  {
+    ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
+    route_tc_kernel<<<grid, RT_THREADS, smem, s>>>(mx, mw, d, stages, tmem_cols, h->d_status);
+  }
+  FMMOE_CUDA_TRY(cudaGetLastError());
+  return FMMOE_OK;
+}
+
 template <int NT>
-static fmmoe_status launch_nt(fmmoe_handle* h, const RouteDev& d, int dtype, int grid, cudaStream_t s) {
+static fmmoe_status launch_nt(fmmoe_handle* h, const RouteDev& d, int grid, cudaStream_t s) {
   const int e_pad = NT * 32;
   const size_t tail = (size_t)R_BM * (e_pad + 1) * 4 + (size_t)e_pad * 4;
-  if (dtype == FMMOE_BF16) {
-    const size_t smem = (size_t)R_STAGES * (R_BM + e_pad) * R_LDS * 2 + tail;
-    FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_bf16_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
-    route_bf16_kernel<NT><<<grid, R_THREADS, smem, s>>>(d);
-  } else {
-    const size_t smem = (size_t)(R_BM + e_pad) * 33 * 4 + tail;
-    FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_f32_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const size_t smem = (size_t)(R_BM + e_pad) * 33 * 4 + tail;
+  FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_f32_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  {
     ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
     route_f32_kernel<NT><<<grid, R_THREADS, smem, s>>>(d);
   }
@@ -299,18 +474,22 @@ fmmoe_status launch_route(fmmoe_handle* h, const RouteArgs& a, cudaStream_t s) {
   d.e_pad = (a.E + 31) / 32 * 32;
   d.logits = a.logits; d.probs = a.probs; d.topk_idx = a.topk_idx; d.topk_w = a.topk_w;
   d.inv_row = a.inv_row; d.counts = a.counts;
-  const int grid = (int)((a.T + R_BM - 1) / R_BM);
   fmmoe_status st;
-  switch (d.e_pad / 32) {
-    case 1: st = launch_nt<1>(h, d, a.dtype, grid, s); break;
-    case 2: st = launch_nt<2>(h, d, a.dtype, grid, s); break;
-    case 3: st = launch_nt<3>(h, d, a.dtype, grid, s); break;
-    case 4: st = launch_nt<4>(h, d, a.dtype, grid, s); break;
-    case 5: st = launch_nt<5>(h, d, a.dtype, grid, s); break;
-    case 6: st = launch_nt<6>(h, d, a.dtype, grid, s); break;
-    case 7: st = launch_nt<7>(h, d, a.dtype, grid, s); break;
-    case 8: st = launch_nt<8>(h, d, a.dtype, grid, s); break;
-    default: return FMMOE_ERR_UNSUPPORTED;
+  if (a.dtype == FMMOE_BF16) {
+    st = launch_route_tc(h, d, s);
+  } else {
+    const int grid = (int)((a.T + R_BM - 1) / R_BM);
+    switch (d.e_pad / 32) {
+      case 1: st = launch_nt<1>(h, d, grid, s); break;
+      case 2: st = launch_nt<2>(h, d, grid, s); break;
+      case 3: st = launch_nt<3>(h, d, grid, s); break;
+      case 4: st = launch_nt<4>(h, d, grid, s); break;
+      case 5: st = launch_nt<5>(h, d, grid, s); break;
+      case 6: st = launch_nt<6>(h, d, grid, s); break;
+      case 7: st = launch_nt<7>(h, d, grid, s); break;
+      case 8: st = launch_nt<8>(h, d, grid, s); break;
+      default: return FMMOE_ERR_UNSUPPORTED;
+    }
   }
   if (st == FMMOE_OK) h->launches += 1;
   return st;
