@@ -2,8 +2,8 @@
 // for vision tokens once the layer has reached l_v) and renormalised gates (Eq. 5),
 // fused in one kernel per storage type.
 //   bf16: the logits tile [128 tokens, E] is a tcgen05 GEMM fed by TMA with its accumulator
-//         in tensor memory; one thread per token then reads its row back and runs the
-//         softmax / top-k / gate step on it.
+//         in tensor memory; the tile is then copied to shared memory and eight lanes per
+//         token run the softmax / top-k / gate step across the expert dimension.
 //   fp32: a CTA owns 32 tokens, forms their logits with plain FMA in shared memory (TF32
 //         would miss an fp32 tolerance), then each warp takes 8 tokens and runs the
 //         softmax / top-k / gate step across the expert dimension with warp shuffles.
@@ -110,150 +110,129 @@ __device__ __forceinline__ void flush_hist(const int* hist, const RouteDev& a) {
 }
 
 // ---------------------------------------------------------------------------------------
-// bf16 router on the tcgen05 tensor cores.  A CTA owns 128 tokens:
+// bf16 router on the tcgen05 tensor cores.  A CTA of 8 warps owns 128 tokens:
 //   warp 0    : TMA producer  (X tile 128x64 and the router matrix tile e_pad x 64 per stage)
 //   warp 1    : UMMA issuer   (128 x e_pad x 16 tcgen05.mma; the logits tile lives in TMEM)
-//   warps 2-5 : one thread per token row reads its logits back from TMEM in 32-column chunks
-//               and runs bias + softmax + top-k + gates on them (the chunks are re-read per
-//               pass instead of being held in registers: tensor memory is cheap to read).
+//   warps 4-7 : once the accumulator is complete, copy it (+ bias) from TMEM to shared memory,
+//               reusing the pipeline's stage buffers
+//   all warps : softmax / top-k / gates with 8 lanes per token (4 tokens per warp at a time):
+//               every lane holds E/8 logits of its token in registers, the row maximum, the
+//               sum and each top-k round are a local scan plus three shuffle steps across
+//               the expert dimension.
 // The router matrix is read once per 128 tokens (from L2 after the first CTA), X once.
 // ---------------------------------------------------------------------------------------
 constexpr int RT_BM = 128;
 constexpr int RT_BK = 64;
-constexpr int RT_THREADS = 192;
+constexpr int RT_THREADS = 256;
 constexpr int RT_A_BYTES = RT_BM * RT_BK * 2;
 constexpr int RT_MAX_STAGES = 8;
 
-__device__ __forceinline__ float route_logit(uint32_t raw, const float* bias_s, int e) { return __uint_as_float(raw) + bias_s[e]; }
+__device__ __forceinline__ float group8_max(float v) {
+#pragma unroll
+  for (int o = 4; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float group8_sum(float v) {
+#pragma unroll
+  for (int o = 4; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
 
-template <int NCH>   // NCH = number of 32-column chunks that cover E
-__device__ __forceinline__ void route_tail_tmem(uint32_t taddr, const float* bias_s, int* hist, long long t,
-                                                const RouteDev& a) {
-  const bool tok_ok = t < a.T;
+// Softmax / top-k / gates for the CTA's 128 tokens from the logits tile in shared memory.
+// NV = logits per lane (expert e = lane8 + 8 j), NV * 8 >= E.
+template <int NV>
+__device__ __forceinline__ void route_tail_group8(const float* Ls, int ldl, long long row0, int* hist, const RouteDev& a) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 3, l8 = lane & 7;
   const int E = a.E;
-  const bool vec4 = (E & 3) == 0;
-  // pass 1: row maximum (and the logits themselves, if wanted)
-  float m = -INFINITY;
+  for (int it = 0; it < RT_BM / 32; ++it) {
+    // rows of one warp are 8 apart: with an odd row pitch the four groups hit distinct banks
+    const int r = it * 32 + g * 8 + warp;
+    const long long t = row0 + r;
+    const bool tok_ok = t < a.T;
+    float z[NV];
 #pragma unroll
-  for (int c = 0; c < NCH; ++c) {
-    uint32_t v[32];
-    tmem_ld32(taddr + c * 32, v);
-    tmem_ld_wait();
-    float z[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const int e = c * 32 + j;
-      z[j] = e < E ? route_logit(v[j], bias_s, e) : -INFINITY;
-      m = fmaxf(m, z[j]);
+    for (int j = 0; j < NV; ++j) {
+      const int e = l8 + 8 * j;
+      z[j] = e < E ? Ls[r * ldl + e] : -INFINITY;
     }
     if (a.logits && tok_ok) {
-      float* dst = a.logits + t * E + c * 32;
-      if (vec4) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 4)
-          if (c * 32 + j < E) *reinterpret_cast<float4*>(dst + j) = make_float4(z[j], z[j + 1], z[j + 2], z[j + 3]);
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (c * 32 + j < E) dst[j] = z[j];
-      }
+      for (int j = 0; j < NV; ++j)
+        if (l8 + 8 * j < E) a.logits[t * E + l8 + 8 * j] = z[j];
     }
-  }
-  // pass 2: softmax denominator
-  float s = 0.f;
+    float m = z[0];
 #pragma unroll
-  for (int c = 0; c < NCH; ++c) {
-    uint32_t v[32];
-    tmem_ld32(taddr + c * 32, v);
-    tmem_ld_wait();
+    for (int j = 1; j < NV; ++j) m = fmaxf(m, z[j]);
+    m = group8_max(m);
+    float s = 0.f;
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const int e = c * 32 + j;
-      if (e < E) s += __expf(route_logit(v[j], bias_s, e) - m);
+    for (int j = 0; j < NV; ++j) s += __expf(z[j] - m);   // exp(-inf) = 0 for padded entries
+    s = group8_sum(s);
+    if (a.probs && tok_ok) {
+      const float inv = 1.f / s;
+#pragma unroll
+      for (int j = 0; j < NV; ++j)
+        if (l8 + 8 * j < E) a.probs[t * E + l8 + 8 * j] = __expf(z[j] - m) * inv;
     }
-  }
-  // pass 3: probabilities (Eq. 2), only when the caller wants them (pruning layers)
-  if (a.probs) {
-    const float inv = 1.f / s;
+    const int k_t = tok_ok ? ((a.reduce_on && a.is_visual[t]) ? a.Kv : a.K) : 0;
+    const int k_warp = __reduce_max_sync(0xffffffffu, k_t);
+    uint32_t taken = 0;
+    float denom = 0.f;
+    float sel_p[2] = {0.f, 0.f};
+    int sel_e[2] = {-1, -1};
+    for (int i = 0; i < k_warp; ++i) {
+      // two independent scan chains (even / odd j), merged; a strict comparison while walking
+      // upwards keeps the lower expert index among equal logits
+      float b0 = -INFINITY, b1 = -INFINITY;
+      int e0 = 0x7fffffff, e1 = 0x7fffffff;
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-      uint32_t v[32];
-      tmem_ld32(taddr + c * 32, v);
-      tmem_ld_wait();
-      float pr[32];
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const int e = c * 32 + j;
-        pr[j] = e < E ? __expf(route_logit(v[j], bias_s, e) - m) * inv : 0.f;
-      }
-      if (tok_ok) {
-        float* dst = a.probs + t * E + c * 32;
-        if (vec4) {
-#pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            if (c * 32 + j < E) *reinterpret_cast<float4*>(dst + j) = make_float4(pr[j], pr[j + 1], pr[j + 2], pr[j + 3]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c * 32 + j < E) dst[j] = pr[j];
+      for (int j = 0; j < NV; j += 2) {
+        if (l8 + 8 * j < E && !((taken >> j) & 1u) && (z[j] > b0 || e0 == 0x7fffffff)) { b0 = z[j]; e0 = l8 + 8 * j; }
+        if (j + 1 < NV && l8 + 8 * (j + 1) < E && !((taken >> (j + 1)) & 1u) && (z[j + 1] > b1 || e1 == 0x7fffffff)) {
+          b1 = z[j + 1]; e1 = l8 + 8 * (j + 1);
         }
       }
-    }
-  }
-  // top-k (Eq. 3): k_t rounds of "largest logit not taken yet"; scanning upwards with a strict
-  // comparison gives equal logits to the lower expert index
-  const int k_t = tok_ok ? ((a.reduce_on && a.is_visual[t]) ? a.Kv : a.K) : 0;
-  uint32_t taken[NCH];
+      float bv = b0; int be = e0;
+      if (e1 != 0x7fffffff && (be == 0x7fffffff || b1 > bv || (b1 == bv && e1 < be))) { bv = b1; be = e1; }
 #pragma unroll
-  for (int c = 0; c < NCH; ++c) taken[c] = 0;
-  float denom = 0.f;
-  int32_t* oi = a.topk_idx + t * a.K;
-  float* ow = a.topk_w + t * a.K;
-  const int k_warp = __reduce_max_sync(0xffffffffu, k_t);   // tmem loads are warp-collective
-  for (int i = 0; i < k_warp; ++i) {
-    float best = -INFINITY;
-    int be = -1;
-#pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-      uint32_t v[32];
-      tmem_ld32(taddr + c * 32, v);
-      tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const int e = c * 32 + j;
-        const float z = route_logit(v[j], bias_s, e < E ? e : 0);
-        if (e < E && !((taken[c] >> j) & 1u) && (z > best || be < 0)) { best = z; be = e; }
+      for (int o = 4; o; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oe = __shfl_xor_sync(0xffffffffu, be, o);
+        if (oe != 0x7fffffff && (be == 0x7fffffff || ov > bv || (ov == bv && oe < be))) { bv = ov; be = oe; }
+      }
+      if (i < k_t) {
+        if ((be & 7) == l8) taken |= 1u << (be >> 3);
+        const float p = __expf(bv - m);
+        denom += p;
+        if ((i & 7) == l8) { sel_p[i >> 3] = p; sel_e[i >> 3] = be; }
       }
     }
-    if (i < k_t) {
+    if (tok_ok) {
 #pragma unroll
-      for (int c = 0; c < NCH; ++c)
-        if (c == (be >> 5)) taken[c] |= 1u << (be & 31);
-      const float p = __expf(best - m);
-      denom += p;
-      oi[i] = be;
-      ow[i] = p;          // unnormalised; rescaled below
-      if (a.counts) atomicAdd(&hist[be], 1);
-    }
-  }
-  if (tok_ok) {
-    for (int i = 0; i < a.K; ++i) {
-      if (i < k_t) ow[i] = ow[i] / denom;     // Eq. 5
-      else { oi[i] = -1; ow[i] = 0.f; }
-      if (a.inv_row) a.inv_row[t * a.K + i] = -1;
+      for (int h = 0; h < 2; ++h) {
+        const int slot = l8 + 8 * h;
+        if (slot < a.K) {
+          const bool sel = slot < k_t;
+          a.topk_idx[t * a.K + slot] = sel ? sel_e[h] : -1;
+          a.topk_w[t * a.K + slot] = sel ? sel_p[h] / denom : 0.f;   // Eq. 5
+          if (a.inv_row) a.inv_row[t * a.K + slot] = -1;
+          if (sel && a.counts) atomicAdd(&hist[sel_e[h]], 1);
+        }
+      }
     }
   }
 }
 
 __global__ void __launch_bounds__(RT_THREADS, 1)
 route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const RouteDev a,
-                const int stages, const int tmem_cols, int* status) {
+                const int stages, const int tmem_cols, const int tile_bytes, int* status) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char* smem = smem_raw + ((1024 - (raw & 1023)) & 1023);
   const int b_bytes = a.e_pad * RT_BK * 2;
   const int stage_bytes = RT_A_BYTES + b_bytes;
-  float* bias_s = reinterpret_cast<float*>(smem + stages * stage_bytes);   // [256]
+  float* bias_s = reinterpret_cast<float*>(smem + tile_bytes);              // [256]
   int* hist = reinterpret_cast<int*>(bias_s + FMMOE_MAX_EXPERTS);           // [256]
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(hist + FMMOE_MAX_EXPERTS);
   uint64_t* empty_bar = full_bar + RT_MAX_STAGES;
@@ -262,6 +241,9 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.H / RT_BK;
+  const int nch = (a.E + 31) / 32;
+  const int ldl = nch * 32 + 1;                 // odd pitch of the logits tile in shared memory
+  float* Ls = reinterpret_cast<float*>(smem);   // [128][ldl], overlays the stage buffers after the GEMM
 
   for (int e = threadIdx.x; e < FMMOE_MAX_EXPERTS; e += RT_THREADS) {
     bias_s[e] = (a.bias && e < a.E) ? a.bias[e] : 0.f;
@@ -317,21 +299,19 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       if (ok) umma_commit(tfull_bar);
       else { atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
-  } else {
+  } else if (warp >= 4) {
+    // accumulator complete => every stage buffer has been consumed: reuse them for the logits
     const int q = warp & 3;
-    const long long t = (long long)row0 + q * 32 + lane;
     if (mbar_wait(tfull_bar, 0, abort_flag)) {
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
-      switch ((a.E + 31) / 32) {
-        case 1: route_tail_tmem<1>(taddr, bias_s, hist, t, a); break;
-        case 2: route_tail_tmem<2>(taddr, bias_s, hist, t, a); break;
-        case 3: route_tail_tmem<3>(taddr, bias_s, hist, t, a); break;
-        case 4: route_tail_tmem<4>(taddr, bias_s, hist, t, a); break;
-        case 5: route_tail_tmem<5>(taddr, bias_s, hist, t, a); break;
-        case 6: route_tail_tmem<6>(taddr, bias_s, hist, t, a); break;
-        case 7: route_tail_tmem<7>(taddr, bias_s, hist, t, a); break;
-        default: route_tail_tmem<8>(taddr, bias_s, hist, t, a); break;
+      float* dst = Ls + (q * 32 + lane) * ldl;
+      for (int c = 0; c < nch; ++c) {
+        uint32_t v[32];
+        tmem_ld32(taddr + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) dst[c * 32 + j] = __uint_as_float(v[j]) + bias_s[c * 32 + j];
       }
     } else {
       atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1;
@@ -344,10 +324,22 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const uint64_t t0 = global_timer_ns();
     while (global_timer_ns() - t0 < 200000ull) { }
     __syncthreads();
+  } else {
+    switch ((a.E + 31) / 32) {
+      case 1: route_tail_group8<4>(Ls, ldl, row0, hist, a); break;
+      case 2: route_tail_group8<8>(Ls, ldl, row0, hist, a); break;
+      case 3: route_tail_group8<12>(Ls, ldl, row0, hist, a); break;
+      case 4: route_tail_group8<16>(Ls, ldl, row0, hist, a); break;
+      case 5: route_tail_group8<20>(Ls, ldl, row0, hist, a); break;
+      case 6: route_tail_group8<24>(Ls, ldl, row0, hist, a); break;
+      case 7: route_tail_group8<28>(Ls, ldl, row0, hist, a); break;
+      default: route_tail_group8<32>(Ls, ldl, row0, hist, a); break;
+    }
+    __syncthreads();
+    if (a.counts)
+      for (int e = threadIdx.x; e < a.E; e += RT_THREADS)
+        if (hist[e]) atomicAdd(&a.counts[e], hist[e]);
   }
-  if (a.counts)
-    for (int e = threadIdx.x; e < a.E; e += RT_THREADS)
-      if (hist[e]) atomicAdd(&a.counts[e], hist[e]);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
@@ -438,7 +430,11 @@ static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s)
   if (stages < 1) return FMMOE_ERR_UNSUPPORTED;
   int tmem_cols = 32;
   while (tmem_cols < (d.E + 31) / 32 * 32) tmem_cols *= 2;
-  const size_t smem = (size_t)stages * stage_bytes + FMMOE_MAX_EXPERTS * 8 + (2 * RT_MAX_STAGES + 1) * 8 + 16 + 1024;
+  // the logits tile [128][32*ceil(E/32)+1] fp32 overlays the stage buffers once the GEMM is done
+  size_t tile_bytes = (size_t)stages * stage_bytes;
+  const size_t logit_bytes = (size_t)RT_BM * ((d.E + 31) / 32 * 32 + 1) * 4;
+  if (logit_bytes > tile_bytes) tile_bytes = (logit_bytes + 1023) / 1024 * 1024;
+  const size_t smem = tile_bytes + FMMOE_MAX_EXPERTS * 8 + (2 * RT_MAX_STAGES + 1) * 8 + 16 + 1024;
   CUtensorMap mx, mw;
   if (!route_map(h, &mx, d.x, (uint64_t)d.T, (uint64_t)d.H, RT_BM)) return FMMOE_ERR_CUDA;
   if (!route_map(h, &mw, d.w, (uint64_t)d.E, (uint64_t)d.H, (uint32_t)d.e_pad)) return FMMOE_ERR_CUDA;
@@ -446,7 +442,7 @@ static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s)
   const int grid = (int)((d.T + RT_BM - 1) / RT_BM);
   {
     ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
-    route_tc_kernel<<<grid, RT_THREADS, smem, s>>>(mx, mw, d, stages, tmem_cols, h->d_status);
+    route_tc_kernel<<<grid, RT_THREADS, smem, s>>>(mx, mw, d, stages, tmem_cols, (int)tile_bytes, h->d_status);
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   return FMMOE_OK;
