@@ -25,7 +25,7 @@ import numpy as np  # noqa: E402
 
 METRIC = "MoE-layer prefill tokens/s"
 UNIT = "tokens/s"
-WORKLOADS = ("C0", "C1", "C2", "C2x4", "C3")
+WORKLOADS = ("C0", "C1", "C2", "C2x4", "C3", "C4")
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
 # ncu captures summarised under profiles/ (null until a capture for that workload exists).
@@ -337,6 +337,197 @@ def run_ours(args):
     return 0
 
 
+# ------------------------------------------------------------------ the 24-layer stack (C4)
+def stack_describe(sc, n_layers):
+    lc = sc.layer
+    st = ", ".join(f"after layer {l}: to {int(pc.retain * 100)}% (W={pc.window}, gamma={pc.gamma})"
+                   for l, pc in sorted(sc.prune_after.items()))
+    return {"workload": f"C4: {n_layers} MoE layers of the C1 shape with residual adds (attention omitted), "
+                        f"{lc.batch} x ({lc.n_vis} visual + {lc.n_text} text) tokens, H={lc.hidden} E={lc.n_experts} "
+                        f"I={lc.inter} shared={lc.n_shared} K={lc.top_k}, K_v={lc.top_k_vis} from layer {sc.reduce_from}; "
+                        f"pruning {st}; attention-free score",
+            "tokens_per_step": lc.n_tokens,
+            "l2": f"inputs larger than L2: {n_layers} x {weight_bytes(lc) / 1e6:.0f} MB of distinct layer weights"}
+
+
+def stack_flops(lc, shapes):
+    """Activated MoE FLOPs of the stack (router + routed pairs + shared experts), per kernel class."""
+    H, E, I_, Ns, Is = lc.hidden, lc.n_experts, lc.inter, lc.n_shared, lc.shared_inter
+    g1 = sum(4 * H * I_ * P + 4 * H * Is * Ns * T for T, P in shapes)
+    g2 = sum(2 * H * I_ * P + 2 * H * Is * Ns * T for T, P in shapes)
+    rt = sum(2 * T * H * E for T, P in shapes)
+    return float(g1), float(g2), float(rt)
+
+
+def oracle_stack_sample(sc, n_layers_sample=2, n_tok=512):
+    """Bounded CPU sample for the stack: the first n_tok tokens of sequence 0 through the first layers."""
+    import torch
+    from paper_2511_17885_b200 import inputs as I
+    from oracle import fmmoe_oracle as O
+    lc = sc.layer
+    x, mask, seq_off, n_vis = I.make_tokens(lc)
+    idx = np.concatenate([np.arange(n_tok - 32), np.arange(lc.n_vis, lc.n_vis + 32)])
+    xs, ms = x[idx].astype(np.float64), mask[idx]
+    ws = []
+    for l in range(n_layers_sample):
+        w = I.stack_layer_weights_torch(sc, l, "cpu")
+        ws.append({k: (None if v is None else v.float().numpy()) for k, v in w.items()})
+    t0 = time.perf_counter()
+    for l in range(n_layers_sample):
+        r = O.moe_forward(xs, ms, ws[l], lc.top_k, lc.top_k_vis, l >= sc.reduce_from, add_residual=True)
+        xs = r["out"]
+    dt = time.perf_counter() - t0
+    return len(idx), n_layers_sample, dt
+
+
+def stack_cpu_baseline(sc, n_layers):
+    import torch
+    n_tok, nl, dt = oracle_stack_sample(sc)
+    # tokens/s through the whole stack, extrapolated from nl layers to n_layers
+    value = n_tok / (dt * n_layers / nl)
+    cores = len(os.sched_getaffinity(0))
+    try:
+        from threadpoolctl import threadpool_info
+        nt = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if nt:
+            cores = max(nt)
+    except Exception:
+        pass
+    sample = (f"{n_tok} tokens of sequence 0 through the first {nl} of {n_layers} layers (router, experts, combine, "
+              f"residual; fp64 numpy; no pruning stage falls in these layers), time scaled by {n_layers}/{nl}")
+    return {"value": value, "unit": UNIT, "cores": int(cores), "kind": "oracle", "sample": sample}
+
+
+def run_stack(args):
+    import torch
+    from paper_2511_17885_b200 import binding as B
+    from paper_2511_17885_b200 import dist as D
+    from paper_2511_17885_b200 import inputs as I
+    from paper_2511_17885_b200.workload import StackWorkload
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    rank, local, world = D.init("nccl") if int(os.environ.get("WORLD_SIZE", 1)) > 1 else (0, 0, 1)
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    sc = I.C4
+    n_layers = args.layers or sc.n_layers
+    peaks = load_peaks()
+    h = B.Handle(local)
+    wl = StackWorkload(sc, h, device=local, token_seed=D.token_seed_for_rank(sc.layer.seed, rank), n_layers=n_layers)
+    K, W = args.steps, max(args.warmup, 3)
+    for _ in range(W):
+        wl.step()
+    h.check_status("warm-up")
+    clocks = ClockSampler(local)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    D.barrier(); torch.cuda.synchronize()
+    clocks.start()
+    n0 = h.launch_count()
+    ev0.record()
+    for _ in range(K):
+        wl.step()
+    ev1.record()
+    clocks.sample_once()
+    torch.cuda.synchronize(); D.barrier()
+    launches = h.launch_count() - n0
+    h.check_status("timed region")
+    value, tmax = D.aggregate_throughput(wl.n_tokens * K, ev0.elapsed_time(ev1) * 1e-3, dev)
+    # instrumented pass
+    h.profile_reset(); h.profile_enable(True)
+    kp = min(K, 3)
+    for _ in range(kp):
+        wl.step()
+    torch.cuda.synchronize()
+    clocks.stop()
+    h.profile_enable(False)
+    prof = h.profile_read()
+    # end to end
+    for _ in range(2):
+        wl.step_host()
+    D.barrier(); torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(K):
+        wl.step_host()
+    e1.record()
+    torch.cuda.synchronize(); D.barrier()
+    e2e_value, _ = D.aggregate_throughput(wl.n_tokens * K, e0.elapsed_time(e1) * 1e-3, dev)
+    h.check_status("end-to-end region")
+
+    shapes = wl.layer_shapes()
+    g1, g2, rt = stack_flops(sc.layer, shapes)
+    dom = max(prof, key=lambda k: prof[k]["ms"])
+    per_launch_s = prof[dom]["ms"] * 1e-3 / max(prof[dom]["launches"], 1)
+    flops_per_launch = {"gemm1": g1, "gemm2": g2, "route": rt}.get(dom, 0.0) / n_layers
+    roof = {"bound": "tensor", "achieved": flops_per_launch / per_launch_s / 1e12, "peak": peaks["tf_sustained"],
+            "unit": "TFLOP/s", "kernel": dom, "us_per_launch": per_launch_s * 1e6, "algorithmic_flops": flops_per_launch,
+            "traffic": NCU_TRAFFIC_BYTES.get("C4", {}).get(dom), "peak_source": peaks["source"] + " (sustained bf16)"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    step_s = tmax / K
+    t_bound = max((g1 + g2 + rt) / (peaks["tf_sustained"] * 1e12), n_layers * weight_bytes(sc.layer) / (peaks["hbm_gbs"] * 1e9))
+    kernels = {k: {"us_per_step": v["ms"] * 1e3 / kp, "launches_per_step": v["launches"] / kp,
+                   "share": v["ms"] / max(sum(x["ms"] for x in prof.values()), 1e-12)} for k, v in prof.items() if v["launches"]}
+
+    # the unreduced, unpruned comparison run (K experts for every token, all tokens in every layer)
+    dense = None
+    if not args.no_dense:
+        del wl.x_out
+        wd = StackWorkload.__new__(StackWorkload)
+        wd.__dict__.update(wl.__dict__)
+        wd.dense, wd.reduce_from, wd.stages = True, n_layers + 1, []
+        wd.out_off, wd.out_vis = B.fmmoe_stack_output_layout([], n_layers, wl.seq_off, wl.n_vis)
+        wd.x_out = torch.empty((wd.out_off[-1], sc.layer.hidden), dtype=wl.x.dtype, device=dev)
+        wd.mask_out = torch.empty(wd.out_off[-1], dtype=torch.uint8, device=dev)
+        for _ in range(2):
+            wd.step()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        d0.record()
+        for _ in range(3):
+            wd.step()
+        d1.record()
+        torch.cuda.synchronize()
+        dg1, dg2, drt = stack_flops(sc.layer, wd.layer_shapes())
+        dense = {"ms_per_step": d0.elapsed_time(d1) / 3, "moe_flops": dg1 + dg2 + drt,
+                 "activated_flops_saved": 1.0 - (g1 + g2 + rt) / (dg1 + dg2 + drt)}
+        h.check_status("dense-k run")
+
+    cpu = stack_cpu_baseline(sc, n_layers) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+    if rank == 0:
+        conf = stack_describe(sc, n_layers)
+        conf.update({"parallelism": f"replicas x{world} (no collective)", "tokens_per_layer": [t for t, _ in shapes],
+                     "final_tokens": wl.out_off[-1]})
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": sc.layer.dtype, "data": "synthetic", "config": conf, "clocks": clocks.summary(),
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(),
+                        "d2h_bytes_per_step": wl.d2h_bytes()},
+                "gpu_launches": int(launches), "roofline": roof,
+                "step_roofline": {"frac": t_bound / step_s, "t_bound_us": t_bound * 1e6, "activated_flops": g1 + g2 + rt,
+                                  "peak_source": peaks["source"]},
+                "kernels": kernels, "dense_k_unpruned": dense, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    D.shutdown()
+    return 0
+
+
+def run_stack_reference(args):
+    if int(os.environ.get("RANK", 0)) != 0:
+        return 0
+    from paper_2511_17885_b200 import inputs as I
+    sc = I.C4
+    n_layers = args.layers or sc.n_layers
+    cb = stack_cpu_baseline(sc, n_layers)
+    line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sc.layer.n_tokens / cb["value"] * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": stack_describe(sc, n_layers), "cpu_baseline": cb,
+            "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -345,7 +536,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C1", choices=WORKLOADS)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="C4 only: run the first N layers of the stack")
+    ap.add_argument("--no-dense", action="store_true", help="C4 only: skip the unreduced, unpruned comparison run")
     args = ap.parse_args()
+    if args.workload == "C4":
+        sys.exit(run_stack_reference(args) if args.impl == "reference" else run_stack(args))
     sys.exit(run_reference(args) if args.impl == "reference" else run_ours(args))
 
 

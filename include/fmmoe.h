@@ -215,6 +215,43 @@ fmmoe_status fmmoe_prune_visual(fmmoe_handle *handle, const fmmoe_prune_params *
                                 int64_t *out_seq_off /* host [n_seq+1] */,
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* A stack of n_layers MoE layers of one shape with residual adds (x <- x + MoE_l(x)), the
+ * setting of Section 3.1's start layer and of the multi-stage pruning schedule (Section 3.2,
+ * Appendices A and D).  Attention and normalisation layers are not part of this library.
+ *   - Layer l (0-based) uses K_v experts for vision tokens iff l >= reduce_from (inclusive).
+ *   - A stage with after_layer = l prunes layer l's OUTPUT using layer l's routing
+ *     probabilities (computed on that layer's input); layers l+1.. see the shorter sequence.
+ *     Its `retain` is a fraction of each sequence's ORIGINAL vision-token count
+ *     (eta = floor(n_vis * retain)).  `attn` is the stage's attention-importance vector
+ *     (device, one entry per token of the sequence as it is at that layer) or NULL for the
+ *     attention-free score.  At most one stage per layer.
+ * layer_w: HOST array of n_layers weight structs (device pointers inside).  x / is_visual:
+ * the input tokens (not modified).  x_out [T', H], is_visual_out [T'] (may be NULL),
+ * out_seq_off (host, [n_seq+1]): the final sequence layout; T' and the offsets follow from
+ * fmmoe_stack_output_layout (host only, data-independent).  Flags: FMMOE_FLAG_DETERMINISTIC
+ * is honoured; the residual is always added and the reduction flag is set per layer.
+ * Everything is enqueued on cuda_stream without synchronising. */
+typedef struct {
+  int32_t after_layer;          /* prune after this layer, 0 .. n_layers-1                 */
+  int32_t reserved;
+  double  retain;               /* fraction of the original vision tokens to retain, 0..1 */
+  fmmoe_prune_params params;    /* W, gamma, alpha, modes                                  */
+  const float *attn;            /* device [T_at_that_layer] or NULL                        */
+} fmmoe_stack_stage;
+
+size_t fmmoe_stack_workspace_bytes(const fmmoe_layer_desc *desc, int64_t n_tokens, int32_t n_seq, uint32_t flags);
+fmmoe_status fmmoe_stack_output_layout(const fmmoe_stack_stage *stages, int32_t n_stages, int32_t n_layers,
+                                       const int64_t *seq_off /* host */, const int64_t *n_vis /* host */,
+                                       int32_t n_seq, int64_t *out_seq_off /* host [n_seq+1] */,
+                                       int64_t *out_n_vis /* host [n_seq] or NULL */);
+fmmoe_status fmmoe_stack_forward(fmmoe_handle *handle, const fmmoe_layer_desc *desc,
+                                 const fmmoe_weights *layer_w /* host [n_layers] */, int32_t n_layers,
+                                 int32_t reduce_from, const fmmoe_stack_stage *stages, int32_t n_stages,
+                                 const void *x, const uint8_t *is_visual, const int64_t *seq_off /* host */,
+                                 const int64_t *n_vis /* host */, int32_t n_seq, uint32_t flags,
+                                 void *x_out, uint8_t *is_visual_out, int64_t *out_seq_off /* host */,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* fmmoe_prune_visual without a caller-supplied workspace and without any allocation.
  * (The paper has no counterpart: this is a packaging variant of fmmoe_prune_visual above,
  * same arguments minus `workspace`/`workspace_bytes`, same kernels, same results.)

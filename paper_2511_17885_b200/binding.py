@@ -44,6 +44,11 @@ class PruneParams(C.Structure):
                 ("alpha", C.c_double), ("gamma", C.c_double)]
 
 
+class StackStage(C.Structure):
+    _fields_ = [("after_layer", C.c_int32), ("reserved", C.c_int32), ("retain", C.c_double),
+                ("params", PruneParams), ("attn", C.c_void_p)]
+
+
 class FmmoeError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -89,6 +94,14 @@ def lib() -> C.CDLL:
                                      C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), i32,
                                      vp, vp, vp, vp, C.POINTER(i64), vp, sz, vp]
     L.fmmoe_prune_visual.restype = C.c_int
+    L.fmmoe_stack_workspace_bytes.argtypes = [C.POINTER(LayerDesc), i64, i32, u32]
+    L.fmmoe_stack_workspace_bytes.restype = sz
+    L.fmmoe_stack_output_layout.argtypes = [C.POINTER(StackStage), i32, i32, C.POINTER(i64), C.POINTER(i64), i32,
+                                            C.POINTER(i64), C.POINTER(i64)]
+    L.fmmoe_stack_output_layout.restype = C.c_int
+    L.fmmoe_stack_forward.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), i32, i32, C.POINTER(StackStage), i32,
+                                      vp, vp, C.POINTER(i64), C.POINTER(i64), i32, u32, vp, vp, C.POINTER(i64), vp, sz, vp]
+    L.fmmoe_stack_forward.restype = C.c_int
     L.fmmoe_prune_visual_static.argtypes = [vp, C.POINTER(PruneParams), vp, i32, vp, vp, i32, i32, vp,
                                             C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), i32,
                                             vp, vp, vp, vp, C.POINTER(i64), vp]
@@ -134,6 +147,25 @@ def fmmoe_workspace_bytes(desc: LayerDesc, n_tokens: int, flags: int = 0) -> int
 
 def make_desc(hidden, n_experts, inter, n_shared, shared_inter, top_k, top_k_vis, dtype: torch.dtype) -> LayerDesc:
     return LayerDesc(hidden, n_experts, inter, n_shared, shared_inter, top_k, top_k_vis, _dtype_code(dtype))
+
+
+def make_stages(stages) -> "C.Array":
+    """[(after_layer, retain, PruneParams, attn tensor or None), ...] -> C array of fmmoe_stack_stage."""
+    arr = (StackStage * max(len(stages), 1))()
+    for i, (layer, retain, pp, attn) in enumerate(stages):
+        arr[i] = StackStage(int(layer), 0, float(retain), pp, attn.data_ptr() if attn is not None else None)
+    return arr
+
+
+def fmmoe_stack_output_layout(stages, n_layers: int, seq_off, n_vis):
+    """Host-only: (out_seq_off, out_n_vis) of a stack with these pruning stages."""
+    B = len(n_vis)
+    arr = make_stages(stages)
+    so = (C.c_int64 * (B + 1))(*[int(v) for v in seq_off])
+    nv = (C.c_int64 * max(B, 1))(*[int(v) for v in n_vis])
+    oo, ov = (C.c_int64 * (B + 1))(), (C.c_int64 * max(B, 1))()
+    _check(lib().fmmoe_stack_output_layout(arr, len(stages), n_layers, so, nv, B, oo, ov), "fmmoe_stack_output_layout")
+    return [int(v) for v in oo], [int(v) for v in ov][:B]
 
 
 def make_weights(w: Dict[str, Optional[torch.Tensor]]) -> Weights:
@@ -282,6 +314,32 @@ class Handle:
                                         _stream()), "fmmoe_prune_visual")
         return {"x_out": x_out, "is_visual_out": vis_out, "keep_idx": keep_idx, "kind": kind,
                 "out_seq_off": [int(v) for v in oo]}
+
+    def fmmoe_stack_forward(self, desc: LayerDesc, layer_weights, reduce_from: int, stages, x: torch.Tensor,
+                            is_visual: torch.Tensor, seq_off, n_vis, flags: int = 0,
+                            x_out: Optional[torch.Tensor] = None, is_visual_out: Optional[torch.Tensor] = None):
+        """n_layers x (x <- x + MoE(x)) with K_v from layer `reduce_from` on and pruning stages
+        [(after_layer, retain, PruneParams, attn or None), ...].  layer_weights: list of Weights structs.
+        Returns (x_out, is_visual_out, out_seq_off)."""
+        n_layers, B = len(layer_weights), len(n_vis)
+        T, H = x.shape
+        out_off, _ = fmmoe_stack_output_layout(stages, n_layers, seq_off, n_vis)
+        t_out = out_off[-1]
+        if x_out is None:
+            x_out = torch.empty((t_out, H), dtype=x.dtype, device=x.device)
+        if is_visual_out is None:
+            is_visual_out = torch.empty(t_out, dtype=torch.uint8, device=x.device)
+        warr = (Weights * n_layers)(*layer_weights)
+        sarr = make_stages(stages)
+        so = (C.c_int64 * (B + 1))(*[int(v) for v in seq_off])
+        nv = (C.c_int64 * max(B, 1))(*[int(v) for v in n_vis])
+        oo = (C.c_int64 * (B + 1))()
+        wsp, wsn = self._ws_args(int(lib().fmmoe_stack_workspace_bytes(C.byref(desc), T, B, flags)))
+        _check(lib().fmmoe_stack_forward(self._h, C.byref(desc), warr, n_layers, reduce_from, sarr, len(stages), _ptr(x),
+                                         _ptr(is_visual), so, nv, B, flags, _ptr(x_out), _ptr(is_visual_out), oo, wsp, wsn,
+                                         _stream()), "fmmoe_stack_forward")
+        assert [int(v) for v in oo] == out_off
+        return x_out, is_visual_out, out_off
 
     def fmmoe_prune_visual_static(self, p: PruneParams, probs: torch.Tensor, attn: Optional[torch.Tensor],
                                   x: torch.Tensor, is_visual: torch.Tensor, seq_off, n_vis, n_retain,

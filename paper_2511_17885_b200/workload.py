@@ -108,3 +108,78 @@ class LayerWorkload:
         off = self.route["expert_off"].cpu().numpy().astype(np.int64)
         cnt = np.diff(off)
         return int(off[-1]), int((cnt > 0).sum())
+
+
+class StackWorkload:
+    """The 24-layer stack: residual MoE layers of one shape, K_v from layer `reduce_from` on, pruning
+    stages after designated layers.  Weights are drawn on the device (distinct per layer).
+
+    step()      : tokens resident in HBM -> fmmoe_stack_forward
+    step_host() : tokens in pinned host memory -> H2D copy, fmmoe_stack_forward, D2H copy of the output
+    dense=True  : the unreduced, unpruned comparison run (K experts for every token, no stages)."""
+
+    def __init__(self, cfg: I.StackCfg, handle: B.Handle, device: int = 0, token_seed: Optional[int] = None,
+                 dense: bool = False, n_layers: Optional[int] = None):
+        self.cfg, self.h = cfg, handle
+        lc = cfg.layer
+        dev = f"cuda:{device}"
+        td = TDT[lc.dtype]
+        self.n_layers = cfg.n_layers if n_layers is None else n_layers
+        x, mask, seq_off, n_vis = I.make_tokens(lc, seed=token_seed)
+        self.seq_off, self.n_vis = seq_off, n_vis
+        self.x = torch.from_numpy(x).to(dev).to(td).contiguous()
+        self.mask = torch.from_numpy(mask).to(dev)
+        self.layers = [I.stack_layer_weights_torch(cfg, l, dev) for l in range(self.n_layers)]
+        self.wstructs = [B.make_weights(w) for w in self.layers]
+        self.desc = B.make_desc(lc.hidden, lc.n_experts, lc.inter, lc.n_shared, lc.shared_inter, lc.top_k,
+                                lc.top_k_vis, td)
+        self.dense = dense
+        self.reduce_from = self.n_layers + 1 if dense else cfg.reduce_from
+        self.stages = [] if dense else [(l, pc.retain, B.prune_params(pc.window, pc.gamma, pc.alpha), None)
+                                        for l, pc in sorted(cfg.prune_after.items()) if l < self.n_layers]
+        self.out_off, self.out_vis = B.fmmoe_stack_output_layout(self.stages, self.n_layers, seq_off, n_vis)
+        self.x_out = torch.empty((self.out_off[-1], lc.hidden), dtype=td, device=dev)
+        self.mask_out = torch.empty(self.out_off[-1], dtype=torch.uint8, device=dev)
+        self.x_host = torch.from_numpy(x).to(td).pin_memory()
+        self.mask_host = torch.from_numpy(mask).pin_memory()
+        self.out_host = torch.empty(self.x_out.shape, dtype=td).pin_memory()
+
+    @property
+    def n_tokens(self) -> int:
+        return self.cfg.layer.n_tokens
+
+    def step(self):
+        self.h.fmmoe_stack_forward(self.desc, self.wstructs, self.reduce_from, self.stages, self.x, self.mask,
+                                   self.seq_off, self.n_vis, 0, x_out=self.x_out, is_visual_out=self.mask_out)
+        return self.x_out
+
+    def step_host(self):
+        self.x.copy_(self.x_host, non_blocking=True)
+        self.mask.copy_(self.mask_host, non_blocking=True)
+        self.step()
+        self.out_host.copy_(self.x_out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return self.out_host
+
+    def h2d_bytes(self) -> int:
+        return self.x_host.numel() * self.x_host.element_size() + self.mask_host.numel()
+
+    def d2h_bytes(self) -> int:
+        return self.out_host.numel() * self.out_host.element_size()
+
+    def layer_shapes(self):
+        """Per layer (tokens, routed pairs): data-independent, from the kept counts of the stages."""
+        lc = self.cfg.layer
+        n_text = [int(self.seq_off[b + 1] - self.seq_off[b] - self.n_vis[b]) for b in range(len(self.n_vis))]
+        vis = [int(v) for v in self.n_vis]
+        out = []
+        stage_at = {l: (r, pp) for l, r, pp, _ in self.stages}
+        for l in range(self.n_layers):
+            kv = lc.top_k_vis if l >= self.reduce_from else lc.top_k
+            T = sum(vis) + sum(n_text)
+            out.append((T, sum(vis) * kv + sum(n_text) * lc.top_k))
+            if l in stage_at:
+                r, pp = stage_at[l]
+                vis = [B.fmmoe_prune_kept_count(vis[b], int(np.floor(int(self.n_vis[b]) * r + 1e-9)), pp)[0]
+                       for b in range(len(vis))]
+        return out
