@@ -43,10 +43,10 @@ bool plan_workspace(const fmmoe_layer_desc& d, int64_t T, uint32_t flags, WsPlan
   size_t o = 0;
   auto take = [&](size_t bytes) { const size_t at = o; o = align_up(o + bytes, 256); return at; };
   p->zero_off = 0;
-  p->counts_off = take(FMMOE_MAX_EXPERTS * 4);
   p->misc_off = take(8 * 4);
   p->acc_off = take(det ? 0 : Tz * H * 4);
   p->zero_bytes = o;
+  p->blk_cnt_off = take((size_t)d.n_experts * ((Tz + 31) / 32) * 4);
   p->topk_idx_off = take(P * 4);
   p->topk_w_off = take(P * 4);
   p->inv_row_off = take(P * 4);
@@ -67,7 +67,7 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 struct RoutePtrs {
   float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row;
-  int32_t* expert_off; int32_t* row_token; float* row_gate; int32_t* counts; int32_t* misc; MTile* mtiles;
+  int32_t* expert_off; int32_t* row_token; float* row_gate; int32_t* blk_cnt; int32_t* misc; MTile* mtiles;
 };
 
 static RoutePtrs bind_route(const WsPlan& pl, char* ws, const fmmoe_route_out* out) {
@@ -80,7 +80,7 @@ static RoutePtrs bind_route(const WsPlan& pl, char* ws, const fmmoe_route_out* o
   r.expert_off = (out && out->expert_off) ? out->expert_off : reinterpret_cast<int32_t*>(ws + pl.expert_off_off);
   r.row_token = (out && out->row_token) ? out->row_token : reinterpret_cast<int32_t*>(ws + pl.row_token_off);
   r.row_gate = reinterpret_cast<float*>(ws + pl.row_gate_off);
-  r.counts = reinterpret_cast<int32_t*>(ws + pl.counts_off);
+  r.blk_cnt = reinterpret_cast<int32_t*>(ws + pl.blk_cnt_off);
   r.misc = reinterpret_cast<int32_t*>(ws + pl.misc_off);
   r.mtiles = reinterpret_cast<MTile*>(ws + pl.mtiles_off);
   return r;
@@ -113,11 +113,13 @@ static fmmoe_status run_route(fmmoe_handle* h, const fmmoe_layer_desc& d, const 
   ra.T = T; ra.H = d.hidden; ra.E = d.n_experts; ra.K = d.top_k; ra.Kv = d.top_k_vis;
   ra.reduce_on = (flags & FMMOE_FLAG_REDUCE_ON) ? 1 : 0; ra.dtype = d.dtype;
   ra.logits = r.logits; ra.probs = r.probs; ra.topk_idx = r.topk_idx; ra.topk_w = r.topk_w;
-  ra.inv_row = r.inv_row; ra.counts = r.counts;
+  ra.inv_row = r.inv_row; ra.blk_cnt = r.blk_cnt;
   fmmoe_status st = launch_route(h, ra, s);
   if (st != FMMOE_OK || !need_permute) return st;
   PermuteArgs pa;
-  pa.topk_idx = r.topk_idx; pa.topk_w = r.topk_w; pa.counts = r.counts;
+  pa.topk_idx = r.topk_idx; pa.topk_w = r.topk_w; pa.blk_cnt = r.blk_cnt;
+  pa.blk_tokens = route_block_tokens(d.dtype);
+  pa.n_blk = (int)((T + pa.blk_tokens - 1) / pa.blk_tokens);
   pa.T = T; pa.K = d.top_k; pa.E = d.n_experts;
   pa.block_m = d.dtype == FMMOE_BF16 ? TC_BLOCK_M : F32_BLOCK_M;
   pa.expert_off = r.expert_off; pa.row_token = r.row_token; pa.row_gate = r.row_gate; pa.inv_row = r.inv_row;
@@ -214,7 +216,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_route(fmmoe
   if (T == 0) return FMMOE_OK;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);
-  FMMOE_CUDA_TRY(cudaMemsetAsync(ws + pl.counts_off, 0, pl.acc_off - pl.counts_off, s));
+  FMMOE_CUDA_TRY(cudaMemsetAsync(ws + pl.misc_off, 0, pl.acc_off - pl.misc_off, s));
   const RoutePtrs r = bind_route(pl, ws, out);
   const bool need_permute = out && (out->expert_off || out->row_token || out->inv_row);
   return run_route(h, *d, *w, x, is_visual, T, flags, r, need_permute, s);

@@ -81,6 +81,7 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 
 struct TileInfo {
   int seg, group_local, row0, rows, nb;
+  bool single;   // routed: the expert's rows fit this one M-tile
 };
 
 // Position `tile` of the interleaved order -> (segment, M-tile, N-block).
@@ -98,6 +99,7 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, int tile, i
     ti.nb = r - mt * p.seg[0].n_nblocks;
     const MTile m = p.mtiles[mt];
     ti.group_local = m.group; ti.row0 = m.row0; ti.rows = m.rows;
+    ti.single = m.pad != 0;
   } else {
     const int t2 = (int)sb;
     ti.seg = 1;
@@ -108,6 +110,7 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, int tile, i
     ti.row0 = mb * G_BM;
     const long long left = p.T - (long long)ti.row0;
     ti.rows = left < G_BM ? (int)left : G_BM;
+    ti.single = false;
   }
   return ti;
 }
@@ -161,7 +164,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
       tma_prefetch_desc(&tmA_r); tma_prefetch_desc(&tmB0_r); tma_prefetch_desc(&tmB1_r);
       if (p.shared_mtiles) { tma_prefetch_desc(&tmA_s); tma_prefetch_desc(&tmB0_s); tma_prefetch_desc(&tmB1_s); }
       const uint64_t pol_stream = l2_policy_evict_first();
-      const uint64_t pol_keep = l2_policy_evict_last();
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (uint32_t it = 0; ok; ++it) {
@@ -178,9 +180,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         const CUtensorMap* mA = ti.seg ? &tmA_s : &tmA_r;
         const CUtensorMap* mB0 = ti.seg ? &tmB0_s : &tmB0_r;
         const CUtensorMap* mB1 = ti.seg ? &tmB1_s : &tmB1_r;
-        // routed weights are read once per M-tile of their expert: let them leave L2 first;
-        // shared-expert weights are reused by every M-tile: default priority
-        const bool stream_b = ti.seg == 0;
+        // Weights of a routed expert whose rows fit one M-tile are read exactly once: let them
+        // leave L2 first.  Everything that is re-read (weights of multi-tile experts and of the
+        // shared experts, activation tiles) keeps the default priority: tiles that share data
+        // are adjacent in the order, so plain LRU keeps it resident for as long as it is needed.
+        const bool stream_b = ti.seg == 0 && ti.single;
         const int a_row = ti.row0 + ti.group_local * sg.a_group_stride;
         const int b_y0 = ti.group_local * sg.b_rows_per_group + ti.nb * (MODE == 0 ? 128 : 256);
         const int b_y1 = MODE == 0 ? b_y0 : b_y0 + 128;
@@ -188,7 +192,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
           if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           unsigned char* sA = smem + stage * G_STAGE_BYTES;
           mbar_arrive_expect_tx(&full_bar[stage], G_STAGE_BYTES);
-          tma_load_2d_hint(sA, mA, &full_bar[stage], kb * G_BK, a_row, pol_keep);
+          tma_load_2d(sA, mA, &full_bar[stage], kb * G_BK, a_row);
           if (stream_b) {
             tma_load_2d_hint(sA + G_A_BYTES, mB0, &full_bar[stage], kb * G_BK, b_y0, pol_stream);
             tma_load_2d_hint(sA + G_A_BYTES + G_B_BYTES / 2, mB1, &full_bar[stage], kb * G_BK, b_y1, pol_stream);

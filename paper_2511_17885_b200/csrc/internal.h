@@ -39,7 +39,7 @@ struct MTile {
   int32_t group;  // expert id
   int32_t row0;   // first row (in the grouped order)
   int32_t rows;   // valid rows in this tile (1..block_m)
-  int32_t pad;
+  int32_t pad;    // 1 if this is the only tile of its expert
 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -47,7 +47,7 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 // Workspace layout of fmmoe_route / fmmoe_moe_forward (byte offsets).
 struct WsPlan {
   size_t zero_off, zero_bytes;  // region cleared at the start of every call
-  size_t counts_off;            // int32 [FMMOE_MAX_EXPERTS] expert histogram
+  size_t blk_cnt_off;           // int32 [E][ceil(T/32)] per-block expert counts / offsets (not cleared)
   size_t misc_off;              // int32 [8]: [0] number of routed M-tiles, [1],[2] GEMM tile counters
   size_t acc_off;               // fp32 [T,H] combine accumulator (atomic mode)
   size_t topk_idx_off, topk_w_off, inv_row_off;
@@ -94,12 +94,16 @@ struct ProfScope {
 struct RouteArgs {
   const void* x; const void* router_w; const float* router_b; const uint8_t* is_visual;
   int64_t T; int H, E, K, Kv; int reduce_on; int dtype;
-  float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row; int32_t* counts;
+  float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row;
+  int32_t* blk_cnt;   // [E][n_blk]: per token block (route_block_tokens) and expert, the number of selections
 };
+// Tokens per router CTA (= granularity of blk_cnt and of the in-block ranks the router leaves in inv_row).
+static inline int route_block_tokens(int dtype) { return dtype == FMMOE_BF16 ? 128 : 32; }
 fmmoe_status launch_route(fmmoe_handle* h, const RouteArgs& a, cudaStream_t s);
 
 struct PermuteArgs {
-  const int32_t* topk_idx; const float* topk_w; const int32_t* counts;
+  const int32_t* topk_idx; const float* topk_w;
+  int32_t* blk_cnt; int n_blk; int blk_tokens;   // router's block counts (turned into offsets in place)
   int64_t T; int K, E; int block_m;
   int32_t* expert_off; int32_t* row_token; float* row_gate; int32_t* inv_row;
   MTile* mtiles; int32_t* n_mtiles;

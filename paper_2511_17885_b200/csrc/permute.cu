@@ -1,13 +1,14 @@
-// Permute-by-expert: from the per-expert histogram (filled by the router) to the
-// stable grouping of the routed (token, expert) pairs by expert.  The paper only
-// states that an unselected expert costs nothing (Section 3.1); the grouped order
-// used here is the unique stable one (rows of an expert ascend by token index), so
-// it is reproducible bit for bit: ranks come from ballots and scans, never from
-// the arrival order of atomics.
+// Permute-by-expert: the stable grouping of the routed (token, expert) pairs by expert.  The
+// paper only states that an unselected expert costs nothing (Section 3.1); the grouped order
+// used here is the unique stable one (rows of an expert ascend by token index), so it is
+// reproducible bit for bit: every rank comes from counts and scans, never from the arrival
+// order of atomics.
 //
-// One CTA per expert: it scans the histogram for its first row and its first
-// M-tile, then walks the tokens in order, 1024 at a time, and assigns consecutive
-// rows to those that selected the expert.
+// The router leaves, per block of tokens, the number of selections of every expert (blk_cnt)
+// and, per (token, slot), the token's rank among its block's tokens that chose that expert.
+//   scan_kernel    : per expert an exclusive scan of the block counts (in place), the scan of
+//                    the expert totals (expert_off) and the list of 128-row M-tiles
+//   scatter_kernel : row = expert_off[e] + block offset + in-block rank, for every pair
 #include <cuda_bf16.h>
 
 #include "internal.h"
@@ -17,89 +18,82 @@ namespace fmmoe {
 constexpr int P_THREADS = 1024;
 
 struct PermuteDev {
-  const int32_t* topk_idx; const float* topk_w; const int32_t* counts;
+  const int32_t* topk_idx; const float* topk_w;
+  int32_t* blk_cnt; int n_blk, blk_tokens;
   long long T; int K, E, block_m;
   int32_t* expert_off; int32_t* row_token; float* row_gate; int32_t* inv_row;
   MTile* mtiles; int32_t* n_mtiles;
 };
 
-__global__ void __launch_bounds__(P_THREADS) permute_kernel(const PermuteDev a) {
-  __shared__ int s_off, s_tile0, s_total_rows, s_total_tiles;
-  __shared__ int s_warp[P_THREADS / 32];
-  __shared__ int s_running;
-  const int e = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-  if (warp == 0) {   // prefix over the (<= 256) expert counts
-    int off = 0, tiles = 0, tot = 0, tot_tiles = 0;
-    for (int i = lane; i < a.E; i += 32) {
-      const int c = a.counts[i];
-      const int nt = (c + a.block_m - 1) / a.block_m;
-      if (i < e) { off += c; tiles += nt; }
-      tot += c; tot_tiles += nt;
-    }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) {
-      off += __shfl_xor_sync(0xffffffffu, off, o);
-      tiles += __shfl_xor_sync(0xffffffffu, tiles, o);
-      tot += __shfl_xor_sync(0xffffffffu, tot, o);
-      tot_tiles += __shfl_xor_sync(0xffffffffu, tot_tiles, o);
-    }
-    if (lane == 0) { s_off = off; s_tile0 = tiles; s_total_rows = tot; s_total_tiles = tot_tiles; s_running = 0; }
-  }
-  __syncthreads();
-  const int base = s_off;
-  const int cnt = a.counts[e];
-  if (tid == 0) {
-    if (a.expert_off) {
-      a.expert_off[e] = base;
-      if (e == a.E - 1) a.expert_off[a.E] = s_total_rows;
-    }
-    if (e == a.E - 1 && a.n_mtiles) a.n_mtiles[0] = s_total_tiles;
-  }
-  if (a.mtiles) {
-    const int nt = (cnt + a.block_m - 1) / a.block_m;
-    for (int i = tid; i < nt; i += P_THREADS) {
-      MTile m;
-      m.group = e; m.row0 = base + i * a.block_m;
-      m.rows = min(a.block_m, cnt - i * a.block_m); m.pad = 0;
-      a.mtiles[s_tile0 + i] = m;
-    }
-  }
-  if (cnt == 0) return;
-
-  for (long long t0 = 0; t0 < a.T; t0 += P_THREADS) {
-    const long long t = t0 + tid;
-    int slot = -1;
-    if (t < a.T) {
-      for (int s = 0; s < a.K; ++s)
-        if (a.topk_idx[t * a.K + s] == e) { slot = s; break; }
-    }
-    const unsigned bal = __ballot_sync(0xffffffffu, slot >= 0);
-    if (lane == 0) s_warp[warp] = __popc(bal);
-    __syncthreads();
-    if (warp == 0) {   // inclusive scan of the 32 warp counts
-      int v = s_warp[lane];
+__global__ void __launch_bounds__(P_THREADS) scan_kernel(const PermuteDev a) {
+  __shared__ int s_cnt[FMMOE_MAX_EXPERTS], s_off[FMMOE_MAX_EXPERTS + 1], s_tile0[FMMOE_MAX_EXPERTS + 1];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // per expert: exclusive scan over the token blocks, 32 blocks per step
+  for (int e = warp; e < a.E; e += P_THREADS / 32) {
+    int32_t* row = a.blk_cnt + (long long)e * a.n_blk;
+    int running = 0;
+    for (int b0 = 0; b0 < a.n_blk; b0 += 32) {
+      const int b = b0 + lane;
+      const int v = b < a.n_blk ? row[b] : 0;
+      int incl = v;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, v, o);
-        if (lane >= o) v += n;
+        const int n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
       }
-      s_warp[lane] = v;
+      if (b < a.n_blk) row[b] = running + incl - v;
+      running += __shfl_sync(0xffffffffu, incl, 31);
     }
-    __syncthreads();
-    const int running = s_running;
-    if (slot >= 0) {
-      const int pos = running + (warp ? s_warp[warp - 1] : 0) + __popc(bal & ((1u << lane) - 1u));
-      const int row = base + pos;
-      if (a.row_token) a.row_token[row] = (int)t;
-      if (a.row_gate) a.row_gate[row] = a.topk_w[t * a.K + slot];
-      if (a.inv_row) a.inv_row[t * a.K + slot] = row;
-    }
-    __syncthreads();
-    if (tid == 0) s_running = running + s_warp[31];
-    __syncthreads();
-    if (s_running >= cnt) break;   // all rows of this expert placed
+    if (lane == 0) s_cnt[e] = running;
   }
+  __syncthreads();
+  if (warp == 0) {   // scan over the (<= 256) expert totals: first row and first M-tile of each expert
+    int run_rows = 0, run_tiles = 0;
+    for (int e0 = 0; e0 < a.E; e0 += 32) {
+      const int e = e0 + lane;
+      const int c = e < a.E ? s_cnt[e] : 0;
+      const int nt = (c + a.block_m - 1) / a.block_m;
+      int ic = c, it = nt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n1 = __shfl_up_sync(0xffffffffu, ic, o);
+        const int n2 = __shfl_up_sync(0xffffffffu, it, o);
+        if (lane >= o) { ic += n1; it += n2; }
+      }
+      if (e < a.E) { s_off[e] = run_rows + ic - c; s_tile0[e] = run_tiles + it - nt; }
+      run_rows += __shfl_sync(0xffffffffu, ic, 31);
+      run_tiles += __shfl_sync(0xffffffffu, it, 31);
+    }
+    if (lane == 0) {
+      s_off[a.E] = run_rows; s_tile0[a.E] = run_tiles;
+      if (a.n_mtiles) a.n_mtiles[0] = run_tiles;
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e <= a.E; e += P_THREADS) a.expert_off[e] = s_off[e];
+  if (a.mtiles) {
+    for (int e = warp; e < a.E; e += P_THREADS / 32) {
+      const int cnt = s_cnt[e], base = s_off[e], nt = s_tile0[e + 1] - s_tile0[e];
+      for (int i = lane; i < nt; i += 32) {
+        MTile m;
+        m.group = e; m.row0 = base + i * a.block_m;
+        m.rows = min(a.block_m, cnt - i * a.block_m); m.pad = nt == 1;   // 1: the expert's only tile
+        a.mtiles[s_tile0[e] + i] = m;
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) scatter_kernel(const PermuteDev a) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.T * a.K) return;
+  const int e = a.topk_idx[i];
+  if (e < 0) return;                       // padded slot: inv_row already holds -1
+  const long long t = i / a.K;
+  const int row = a.expert_off[e] + a.blk_cnt[(long long)e * a.n_blk + (int)(t / a.blk_tokens)] + a.inv_row[i];
+  a.row_token[row] = (int32_t)t;
+  a.row_gate[row] = a.topk_w[i];
+  a.inv_row[i] = row;
 }
 
 // Copy the routed rows of X into expert-grouped order: xp[row] = x[row_token[row]].
@@ -119,15 +113,20 @@ __global__ void gather_rows_kernel(const uint4* __restrict__ x, const int32_t* _
 }
 
 fmmoe_status launch_permute(fmmoe_handle* h, const PermuteArgs& a, cudaStream_t s) {
-  if (a.E <= 0) return FMMOE_OK;
+  if (a.E <= 0 || a.T <= 0) return FMMOE_OK;
   PermuteDev d;
-  d.topk_idx = a.topk_idx; d.topk_w = a.topk_w; d.counts = a.counts;
+  d.topk_idx = a.topk_idx; d.topk_w = a.topk_w; d.blk_cnt = a.blk_cnt; d.n_blk = a.n_blk; d.blk_tokens = a.blk_tokens;
   d.T = a.T; d.K = a.K; d.E = a.E; d.block_m = a.block_m;
   d.expert_off = a.expert_off; d.row_token = a.row_token; d.row_gate = a.row_gate; d.inv_row = a.inv_row;
   d.mtiles = a.mtiles; d.n_mtiles = a.n_mtiles;
-  { ProfScope ps(h, FMMOE_KERNEL_PERMUTE, s); permute_kernel<<<a.E, P_THREADS, 0, s>>>(d); }
+  const long long pairs = a.T * a.K;
+  {
+    ProfScope ps(h, FMMOE_KERNEL_PERMUTE, s);
+    scan_kernel<<<1, P_THREADS, 0, s>>>(d);
+    scatter_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, s>>>(d);
+  }
   FMMOE_CUDA_TRY(cudaGetLastError());
-  h->launches += 1;
+  h->launches += 2;
   return FMMOE_OK;
 }
 

@@ -7,7 +7,10 @@
 //   fp32: a CTA owns 32 tokens, forms their logits with plain FMA in shared memory (TF32
 //         would miss an fp32 tolerance), then each warp takes 8 tokens and runs the
 //         softmax / top-k / gate step across the expert dimension with warp shuffles.
-// Both kernels also add the selections to the per-expert histogram the permutation needs.
+// Both kernels also start the permutation: a CTA records, per expert, which of its tokens
+// selected it (a bit mask in shared memory), from which it writes the block's expert counts
+// and, for every (token, slot), the rank of the token among the block's tokens that chose
+// the same expert.  Ranks come from bit counts, never from the arrival order of atomics.
 #include <cuda_bf16.h>
 #include <float.h>
 
@@ -22,7 +25,8 @@ constexpr int R_THREADS = 128;
 struct RouteDev {
   const void* x; const void* w; const float* bias; const uint8_t* is_visual;
   long long T; int H, E, K, Kv, reduce_on, e_pad;
-  float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row; int32_t* counts;
+  float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row;
+  int32_t* blk_cnt; int n_blk;   // [E][n_blk] selections of each token block per expert
 };
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -39,7 +43,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // Softmax / top-k / gates for the CTA's tokens, logits already in shared memory.
 // NTL = e_pad / 32 values per lane.
 template <int NTL>
-__device__ __forceinline__ void route_tail(const float* Ls, int ldl, long long t0, const RouteDev& a, int* hist) {
+__device__ __forceinline__ void route_tail(const float* Ls, int ldl, long long t0, const RouteDev& a, uint32_t* emask) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int r = warp; r < R_BM; r += R_THREADS / 32) {
     const long long t = t0 + r;
@@ -96,17 +100,37 @@ __device__ __forceinline__ void route_tail(const float* Ls, int ldl, long long t
       const bool sel = lane < k_t;
       a.topk_idx[t * a.K + lane] = sel ? my_idx : -1;
       a.topk_w[t * a.K + lane] = sel ? p / denom : 0.f;
-      if (a.inv_row) a.inv_row[t * a.K + lane] = -1;
-      if (sel && a.counts) atomicAdd(&hist[my_idx], 1);
+      if (sel) atomicOr(&emask[my_idx], 1u << r);   // one 32-bit word per expert: the block has 32 tokens
     }
   }
 }
 
-__device__ __forceinline__ void flush_hist(const int* hist, const RouteDev& a) {
+// After the block's selections are in `emask` ([E][WORDS] bit masks over the block's tokens):
+// write the block's per-expert counts and the in-block rank of every (token, slot).
+template <int WORDS>
+__device__ __forceinline__ void emit_block_ranks(const uint32_t* emask, long long t0, int blk, const RouteDev& a) {
   __syncthreads();
-  if (a.counts)
-    for (int e = threadIdx.x; e < a.E; e += R_THREADS)
-      if (hist[e]) atomicAdd(&a.counts[e], hist[e]);
+  for (int e = threadIdx.x; e < a.E; e += blockDim.x) {
+    int c = 0;
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w) c += __popc(emask[e * WORDS + w]);
+    a.blk_cnt[(long long)e * a.n_blk + blk] = c;
+  }
+  const int items = WORDS * 32 * a.K;
+  for (int it = threadIdx.x; it < items; it += blockDim.x) {
+    const int r = it / a.K;
+    const long long t = t0 + r;
+    if (t >= a.T) break;
+    const int e = __ldcg(a.topk_idx + t * a.K + (it - r * a.K));   // written by this CTA before the barrier
+    int rank = -1;
+    if (e >= 0) {
+      rank = __popc(emask[e * WORDS + (r >> 5)] & ((1u << (r & 31)) - 1u));
+#pragma unroll
+      for (int w = 0; w < WORDS; ++w)
+        if (w < (r >> 5)) rank += __popc(emask[e * WORDS + w]);
+    }
+    a.inv_row[t * a.K + (it - r * a.K)] = rank;
+  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -141,7 +165,7 @@ __device__ __forceinline__ float group8_sum(float v) {
 // Softmax / top-k / gates for the CTA's 128 tokens from the logits tile in shared memory.
 // NV = logits per lane (expert e = lane8 + 8 j), NV * 8 >= E.
 template <int NV>
-__device__ __forceinline__ void route_tail_group8(const float* Ls, int ldl, long long row0, int* hist, const RouteDev& a) {
+__device__ __forceinline__ void route_tail_group8(const float* Ls, int ldl, long long row0, uint32_t* emask, const RouteDev& a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 3, l8 = lane & 7;
   const int E = a.E;
@@ -216,8 +240,7 @@ __device__ __forceinline__ void route_tail_group8(const float* Ls, int ldl, long
           const bool sel = slot < k_t;
           a.topk_idx[t * a.K + slot] = sel ? sel_e[h] : -1;
           a.topk_w[t * a.K + slot] = sel ? sel_p[h] / denom : 0.f;   // Eq. 5
-          if (a.inv_row) a.inv_row[t * a.K + slot] = -1;
-          if (sel && a.counts) atomicAdd(&hist[sel_e[h]], 1);
+          if (sel) atomicOr(&emask[sel_e[h] * 4 + (r >> 5)], 1u << (r & 31));
         }
       }
     }
@@ -233,8 +256,8 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const int b_bytes = a.e_pad * RT_BK * 2;
   const int stage_bytes = RT_A_BYTES + b_bytes;
   float* bias_s = reinterpret_cast<float*>(smem + tile_bytes);              // [256]
-  int* hist = reinterpret_cast<int*>(bias_s + FMMOE_MAX_EXPERTS);           // [256]
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(hist + FMMOE_MAX_EXPERTS);
+  uint32_t* emask = reinterpret_cast<uint32_t*>(bias_s + FMMOE_MAX_EXPERTS);   // [256][4] token masks per expert
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(emask + FMMOE_MAX_EXPERTS * 4);
   uint64_t* empty_bar = full_bar + RT_MAX_STAGES;
   uint64_t* tfull_bar = empty_bar + RT_MAX_STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfull_bar + 1);
@@ -247,7 +270,8 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
   for (int e = threadIdx.x; e < FMMOE_MAX_EXPERTS; e += RT_THREADS) {
     bias_s[e] = (a.bias && e < a.E) ? a.bias[e] : 0.f;
-    hist[e] = 0;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) emask[e * 4 + w] = 0;
   }
   if (threadIdx.x == 0) {
     for (int i = 0; i < stages; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
@@ -326,19 +350,16 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     __syncthreads();
   } else {
     switch ((a.E + 31) / 32) {
-      case 1: route_tail_group8<4>(Ls, ldl, row0, hist, a); break;
-      case 2: route_tail_group8<8>(Ls, ldl, row0, hist, a); break;
-      case 3: route_tail_group8<12>(Ls, ldl, row0, hist, a); break;
-      case 4: route_tail_group8<16>(Ls, ldl, row0, hist, a); break;
-      case 5: route_tail_group8<20>(Ls, ldl, row0, hist, a); break;
-      case 6: route_tail_group8<24>(Ls, ldl, row0, hist, a); break;
-      case 7: route_tail_group8<28>(Ls, ldl, row0, hist, a); break;
-      default: route_tail_group8<32>(Ls, ldl, row0, hist, a); break;
+      case 1: route_tail_group8<4>(Ls, ldl, row0, emask, a); break;
+      case 2: route_tail_group8<8>(Ls, ldl, row0, emask, a); break;
+      case 3: route_tail_group8<12>(Ls, ldl, row0, emask, a); break;
+      case 4: route_tail_group8<16>(Ls, ldl, row0, emask, a); break;
+      case 5: route_tail_group8<20>(Ls, ldl, row0, emask, a); break;
+      case 6: route_tail_group8<24>(Ls, ldl, row0, emask, a); break;
+      case 7: route_tail_group8<28>(Ls, ldl, row0, emask, a); break;
+      default: route_tail_group8<32>(Ls, ldl, row0, emask, a); break;
     }
-    __syncthreads();
-    if (a.counts)
-      for (int e = threadIdx.x; e < a.E; e += RT_THREADS)
-        if (hist[e]) atomicAdd(&a.counts[e], hist[e]);
+    emit_block_ranks<4>(emask, row0, blockIdx.x, a);
   }
   if (warp == 1) {
     tc_fence_after();
@@ -357,12 +378,12 @@ __global__ void __launch_bounds__(R_THREADS) route_f32_kernel(const RouteDev a) 
   float* Xs = reinterpret_cast<float*>(smem_raw);   // [R_BM][BK+1]
   float* Ws = Xs + R_BM * (BK + 1);                 // [e_pad][BK+1]
   float* Ls = Ws + e_pad * (BK + 1);                // [R_BM][ldl]
-  int* hist = reinterpret_cast<int*>(Ls + R_BM * ldl);
+  uint32_t* emask = reinterpret_cast<uint32_t*>(Ls + R_BM * ldl);   // [e_pad] one word per expert (32 tokens)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const long long t0 = (long long)blockIdx.x * R_BM;
   const float* X = static_cast<const float*>(a.x);
   const float* W = static_cast<const float*>(a.w);
-  for (int i = tid; i < e_pad; i += R_THREADS) hist[i] = 0;
+  for (int i = tid; i < e_pad; i += R_THREADS) emask[i] = 0;
   float acc[R_BM / 4][NT];
 #pragma unroll
   for (int i = 0; i < R_BM / 4; ++i)
@@ -400,8 +421,8 @@ __global__ void __launch_bounds__(R_THREADS) route_f32_kernel(const RouteDev a) 
       Ls[(warp + 4 * i) * ldl + col] = acc[i][j] + ((a.bias && col < a.E) ? a.bias[col] : 0.f);
     }
   __syncthreads();
-  route_tail<NT>(Ls, ldl, t0, a, hist);
-  flush_hist(hist, a);
+  route_tail<NT>(Ls, ldl, t0, a, emask);
+  emit_block_ranks<1>(emask, t0, blockIdx.x, a);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -434,7 +455,7 @@ static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s)
   size_t tile_bytes = (size_t)stages * stage_bytes;
   const size_t logit_bytes = (size_t)RT_BM * ((d.E + 31) / 32 * 32 + 1) * 4;
   if (logit_bytes > tile_bytes) tile_bytes = (logit_bytes + 1023) / 1024 * 1024;
-  const size_t smem = tile_bytes + FMMOE_MAX_EXPERTS * 8 + (2 * RT_MAX_STAGES + 1) * 8 + 16 + 1024;
+  const size_t smem = tile_bytes + FMMOE_MAX_EXPERTS * 20 + (2 * RT_MAX_STAGES + 1) * 8 + 16 + 1024;
   CUtensorMap mx, mw;
   if (!route_map(h, &mx, d.x, (uint64_t)d.T, (uint64_t)d.H, RT_BM)) return FMMOE_ERR_CUDA;
   if (!route_map(h, &mw, d.w, (uint64_t)d.E, (uint64_t)d.H, (uint32_t)d.e_pad)) return FMMOE_ERR_CUDA;
@@ -469,7 +490,8 @@ fmmoe_status launch_route(fmmoe_handle* h, const RouteArgs& a, cudaStream_t s) {
   d.T = a.T; d.H = a.H; d.E = a.E; d.K = a.K; d.Kv = a.Kv; d.reduce_on = a.reduce_on;
   d.e_pad = (a.E + 31) / 32 * 32;
   d.logits = a.logits; d.probs = a.probs; d.topk_idx = a.topk_idx; d.topk_w = a.topk_w;
-  d.inv_row = a.inv_row; d.counts = a.counts;
+  d.inv_row = a.inv_row; d.blk_cnt = a.blk_cnt;
+  d.n_blk = (int)((a.T + route_block_tokens(a.dtype) - 1) / route_block_tokens(a.dtype));
   fmmoe_status st;
   if (a.dtype == FMMOE_BF16) {
     st = launch_route_tc(h, d, s);
