@@ -46,7 +46,7 @@ bool plan_workspace(const fmmoe_layer_desc& d, int64_t T, uint32_t flags, WsPlan
   p->misc_off = take(8 * 4);
   p->acc_off = take(det ? 0 : Tz * H * 4);
   p->zero_bytes = o;
-  p->blk_cnt_off = take((size_t)d.n_experts * ((Tz + 31) / 32) * 4);
+  p->blk_cnt_off = take((size_t)d.n_experts * ((Tz + 31) / 32 + 4) * 4);
   p->topk_idx_off = take(P * 4);
   p->topk_w_off = take(P * 4);
   p->inv_row_off = take(P * 4);
@@ -118,8 +118,8 @@ static fmmoe_status run_route(fmmoe_handle* h, const fmmoe_layer_desc& d, const 
   if (st != FMMOE_OK || !need_permute) return st;
   PermuteArgs pa;
   pa.topk_idx = r.topk_idx; pa.topk_w = r.topk_w; pa.blk_cnt = r.blk_cnt;
-  pa.blk_tokens = route_block_tokens(d.dtype);
-  pa.n_blk = (int)((T + pa.blk_tokens - 1) / pa.blk_tokens);
+  pa.blk_tokens = route_block_tokens(d.dtype, T, d.hidden);
+  pa.n_blk = route_num_blocks(d.dtype, T, d.hidden);
   pa.T = T; pa.K = d.top_k; pa.E = d.n_experts;
   pa.block_m = d.dtype == FMMOE_BF16 ? TC_BLOCK_M : F32_BLOCK_M;
   pa.expert_off = r.expert_off; pa.row_token = r.row_token; pa.row_gate = r.row_gate; pa.inv_row = r.inv_row;

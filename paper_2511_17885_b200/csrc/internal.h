@@ -97,8 +97,23 @@ struct RouteArgs {
   float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row;
   int32_t* blk_cnt;   // [E][n_blk]: per token block (route_block_tokens) and expert, the number of selections
 };
+// bf16 router: number of CTAs (a cluster) that share one 128-token tile by splitting the
+// contraction.  Few tiles => split, so that more SMs stream X.
+static inline int route_split(int64_t T, int H) {
+  const int64_t tiles = (T + 127) / 128;
+  const int kblocks = H / 64;
+  if (tiles * 4 <= 160 && kblocks % 4 == 0) return 4;
+  if (tiles * 2 <= 160 && kblocks % 2 == 0) return 2;
+  return 1;
+}
 // Tokens per router CTA (= granularity of blk_cnt and of the in-block ranks the router leaves in inv_row).
-static inline int route_block_tokens(int dtype) { return dtype == FMMOE_BF16 ? 128 : 32; }
+static inline int route_block_tokens(int dtype, int64_t T, int H) {
+  return dtype == FMMOE_BF16 ? 128 / route_split(T, H) : 32;
+}
+// Number of router CTAs = number of token blocks (the last tile's blocks may lie past T: they are empty).
+static inline int route_num_blocks(int dtype, int64_t T, int H) {
+  return dtype == FMMOE_BF16 ? (int)((T + 127) / 128) * route_split(T, H) : (int)((T + 31) / 32);
+}
 fmmoe_status launch_route(fmmoe_handle* h, const RouteArgs& a, cudaStream_t s);
 
 struct PermuteArgs {

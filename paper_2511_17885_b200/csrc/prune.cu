@@ -181,21 +181,26 @@ __device__ __forceinline__ uint32_t ordered_bits(float f) {
 
 // Ascending bitonic sort of n (a power of two) 64-bit keys in shared memory by the whole CTA.
 // Keys are unique (the window index is part of them), so the result does not depend on the
-// network's comparison order.
+// network's comparison order.  One thread per compare-exchange pair; pair p of warp w only ever
+// touches elements 64w .. 64w+63 while the partner distance j is <= 32, so those steps need a
+// warp barrier only.
 __device__ __forceinline__ void bitonic_sort_u64(unsigned long long* keys, int n) {
+  const int half = n >> 1;
   for (int k = 2; k <= n; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int idx = threadIdx.x; idx < n; idx += blockDim.x) {
-        const int ixj = idx ^ j;
-        if (ixj > idx) {
-          const unsigned long long x = keys[idx], y = keys[ixj];
-          const bool up = (idx & k) == 0;
-          if ((x > y) == up) { keys[idx] = y; keys[ixj] = x; }
-        }
+      for (int p = threadIdx.x; p < half; p += blockDim.x) {
+        const int lo = ((p & ~(j - 1)) << 1) | (p & (j - 1));
+        const int hi = lo | j;
+        const unsigned long long x = keys[lo], y = keys[hi];
+        const bool up = (lo & k) == 0;
+        if ((x > y) == up) { keys[lo] = y; keys[hi] = x; }
       }
-      __syncthreads();
+      if (j > 32 || half > (int)blockDim.x) __syncthreads();
+      else __syncwarp();
     }
+    if (k >= 64) __syncthreads();   // the next merge starts with partners in other warps' ranges
   }
+  __syncthreads();
 }
 
 // One CTA per sequence.  Eq. 12-13 (one rounding to fp32), then the merge set (Eq. 15) and the

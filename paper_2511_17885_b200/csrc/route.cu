@@ -139,6 +139,9 @@ __device__ __forceinline__ void emit_block_ranks(const uint32_t* emask, long lon
 //   warp 1    : UMMA issuer   (128 x e_pad x 16 tcgen05.mma; the logits tile lives in TMEM)
 //   warps 4-7 : once the accumulator is complete, copy it (+ bias) from TMEM to shared memory,
 //               reusing the pipeline's stage buffers
+//   cluster   : with few token tiles the contraction is split over a cluster of 2 or 4 CTAs
+//               (more SMs pulling X); every CTA then owns 128/split rows of the tile and adds
+//               the partial tiles of its peers, in rank order, through distributed shared memory
 //   all warps : softmax / top-k / gates with 8 lanes per token (4 tokens per warp at a time):
 //               every lane holds E/8 logits of its token in registers, the row maximum, the
 //               sum and each top-k round are a local scan plus three shuffle steps across
@@ -162,23 +165,35 @@ __device__ __forceinline__ float group8_sum(float v) {
   return v;
 }
 
-// Softmax / top-k / gates for the CTA's 128 tokens from the logits tile in shared memory.
+// Softmax / top-k / gates for rows [row_lo, row_lo + n_rows) of the tile (n_rows a multiple of
+// 32).  The logits of a row are the sum, in rank order, of the `split` partial tiles held in the
+// shared memory of the cluster's CTAs (ls_addr[q] = address of rank q's tile), plus the bias.
 // NV = logits per lane (expert e = lane8 + 8 j), NV * 8 >= E.
 template <int NV>
-__device__ __forceinline__ void route_tail_group8(const float* Ls, int ldl, long long row0, uint32_t* emask, const RouteDev& a) {
+__device__ __forceinline__ void route_tail_group8(const uint32_t* ls_addr, int split, int ldl, const float* bias_s,
+                                                  long long row0, int row_lo, int n_rows, uint32_t* emask, int words,
+                                                  const RouteDev& a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 3, l8 = lane & 7;
   const int E = a.E;
-  for (int it = 0; it < RT_BM / 32; ++it) {
+  for (int it = 0; it < n_rows / 32; ++it) {
     // rows of one warp are 8 apart: with an odd row pitch the four groups hit distinct banks
-    const int r = it * 32 + g * 8 + warp;
+    const int rl = it * 32 + g * 8 + warp;   // row inside this CTA's share
+    const int r = row_lo + rl;               // row inside the tile
     const long long t = row0 + r;
     const bool tok_ok = t < a.T;
     float z[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
       const int e = l8 + 8 * j;
-      z[j] = e < E ? Ls[r * ldl + e] : -INFINITY;
+      float v = -INFINITY;
+      if (e < E) {
+        const uint32_t off = (uint32_t)(r * ldl + e) * 4u;
+        v = ld_cluster_f32(ls_addr[0] + off);
+        for (int q = 1; q < split; ++q) v += ld_cluster_f32(ls_addr[q] + off);
+        v += bias_s[e];
+      }
+      z[j] = v;
     }
     if (a.logits && tok_ok) {
 #pragma unroll
@@ -240,7 +255,7 @@ __device__ __forceinline__ void route_tail_group8(const float* Ls, int ldl, long
           const bool sel = slot < k_t;
           a.topk_idx[t * a.K + slot] = sel ? sel_e[h] : -1;
           a.topk_w[t * a.K + slot] = sel ? sel_p[h] / denom : 0.f;   // Eq. 5
-          if (sel) atomicOr(&emask[sel_e[h] * 4 + (r >> 5)], 1u << (r & 31));
+          if (sel) atomicOr(&emask[sel_e[h] * words + (rl >> 5)], 1u << (rl & 31));
         }
       }
     }
@@ -249,7 +264,7 @@ __device__ __forceinline__ void route_tail_group8(const float* Ls, int ldl, long
 
 __global__ void __launch_bounds__(RT_THREADS, 1)
 route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const RouteDev a,
-                const int stages, const int tmem_cols, const int tile_bytes, int* status) {
+                const int stages, const int tmem_cols, const int tile_bytes, const int split, int* status) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char* smem = smem_raw + ((1024 - (raw & 1023)) & 1023);
@@ -263,7 +278,9 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfull_bar + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kblocks = a.H / RT_BK;
+  const int krank = (int)cluster_ctarank();            // this CTA's slice of the contraction
+  const int kblocks = a.H / RT_BK / split;
+  const int kb0 = krank * kblocks;
   const int nch = (a.E + 31) / 32;
   const int ldl = nch * 32 + 1;                 // odd pitch of the logits tile in shared memory
   float* Ls = reinterpret_cast<float*>(smem);   // [128][ldl], overlays the stage buffers after the GEMM
@@ -287,7 +304,7 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int row0 = blockIdx.x * RT_BM;
+  const int row0 = (blockIdx.x / split) * RT_BM;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -298,8 +315,8 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { ok = false; break; }
         unsigned char* sA = smem + stage * stage_bytes;
         mbar_arrive_expect_tx(&full_bar[stage], (uint32_t)stage_bytes);
-        tma_load_2d(sA, &tmX, &full_bar[stage], kb * RT_BK, row0);
-        tma_load_2d(sA + RT_A_BYTES, &tmW, &full_bar[stage], kb * RT_BK, 0);
+        tma_load_2d(sA, &tmX, &full_bar[stage], (kb0 + kb) * RT_BK, row0);
+        tma_load_2d(sA + RT_A_BYTES, &tmW, &full_bar[stage], (kb0 + kb) * RT_BK, 0);
         if (++stage == stages) { stage = 0; phase ^= 1; }
       }
       if (!ok) { atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1; }
@@ -335,7 +352,7 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         tmem_ld32(taddr + c * 32, v);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) dst[c * 32 + j] = __uint_as_float(v[j]) + bias_s[c * 32 + j];
+        for (int j = 0; j < 32; ++j) dst[c * 32 + j] = __uint_as_float(v[j]);   // this CTA's partial sums
       }
     } else {
       atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1;
@@ -344,23 +361,37 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   __syncwarp();
   tc_fence_before();
   __syncthreads();
-  if (*abort_flag) {
+  const bool failed = *abort_flag != 0;
+  if (failed) {
     const uint64_t t0 = global_timer_ns();
     while (global_timer_ns() - t0 < 200000ull) { }
     __syncthreads();
-  } else {
-    switch ((a.E + 31) / 32) {
-      case 1: route_tail_group8<4>(Ls, ldl, row0, emask, a); break;
-      case 2: route_tail_group8<8>(Ls, ldl, row0, emask, a); break;
-      case 3: route_tail_group8<12>(Ls, ldl, row0, emask, a); break;
-      case 4: route_tail_group8<16>(Ls, ldl, row0, emask, a); break;
-      case 5: route_tail_group8<20>(Ls, ldl, row0, emask, a); break;
-      case 6: route_tail_group8<24>(Ls, ldl, row0, emask, a); break;
-      case 7: route_tail_group8<28>(Ls, ldl, row0, emask, a); break;
-      default: route_tail_group8<32>(Ls, ldl, row0, emask, a); break;
-    }
-    emit_block_ranks<4>(emask, row0, blockIdx.x, a);
   }
+  // Every CTA of the cluster now holds its partial logits tile in shared memory.  Both cluster
+  // barriers are executed unconditionally (a CTA that gave up still arrives), so no peer can
+  // be left waiting.
+  cluster_sync_all();
+  if (!failed) {
+    uint32_t ls_addr[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) ls_addr[q] = cluster_map_shared(smem_u32(Ls), q < split ? q : 0);
+    const int n_rows = RT_BM / split, row_lo = krank * n_rows, words = n_rows / 32;
+    switch ((a.E + 31) / 32) {
+      case 1: route_tail_group8<4>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
+      case 2: route_tail_group8<8>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
+      case 3: route_tail_group8<12>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
+      case 4: route_tail_group8<16>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
+      case 5: route_tail_group8<20>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
+      case 6: route_tail_group8<24>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
+      case 7: route_tail_group8<28>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
+      default: route_tail_group8<32>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
+    }
+    // the token block of this CTA: rows [row_lo, row_lo + n_rows) of the tile
+    if (split == 1) emit_block_ranks<4>(emask, (long long)row0, blockIdx.x, a);
+    else if (split == 2) emit_block_ranks<2>(emask, (long long)row0 + row_lo, blockIdx.x, a);
+    else emit_block_ranks<1>(emask, (long long)row0 + row_lo, blockIdx.x, a);
+  }
+  cluster_sync_all();   // peers may still be reading this CTA's tile until here
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
@@ -446,7 +477,8 @@ static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s)
   const int stage_bytes = RT_A_BYTES + d.e_pad * RT_BK * 2;
   int stages = (200 * 1024) / stage_bytes;
   if (stages > RT_MAX_STAGES) stages = RT_MAX_STAGES;
-  const int kblocks = d.H / RT_BK;
+  const int split = route_split(d.T, d.H);
+  const int kblocks = d.H / RT_BK / split;
   if (stages > kblocks) stages = kblocks;
   if (stages < 1) return FMMOE_ERR_UNSUPPORTED;
   int tmem_cols = 32;
@@ -460,10 +492,19 @@ static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s)
   if (!route_map(h, &mx, d.x, (uint64_t)d.T, (uint64_t)d.H, RT_BM)) return FMMOE_ERR_CUDA;
   if (!route_map(h, &mw, d.w, (uint64_t)d.E, (uint64_t)d.H, (uint32_t)d.e_pad)) return FMMOE_ERR_CUDA;
   FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  const int grid = (int)((d.T + RT_BM - 1) / RT_BM);
+  const int tiles = (int)((d.T + RT_BM - 1) / RT_BM);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(tiles * split), 1, 1);
+  cfg.blockDim = dim3(RT_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)split; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
   {
     ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
-    route_tc_kernel<<<grid, RT_THREADS, smem, s>>>(mx, mw, d, stages, tmem_cols, (int)tile_bytes, h->d_status);
+    FMMOE_CUDA_TRY(cudaLaunchKernelEx(&cfg, route_tc_kernel, mx, mw, d, stages, tmem_cols, (int)tile_bytes, split, h->d_status));
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   return FMMOE_OK;
@@ -491,7 +532,7 @@ fmmoe_status launch_route(fmmoe_handle* h, const RouteArgs& a, cudaStream_t s) {
   d.e_pad = (a.E + 31) / 32 * 32;
   d.logits = a.logits; d.probs = a.probs; d.topk_idx = a.topk_idx; d.topk_w = a.topk_w;
   d.inv_row = a.inv_row; d.blk_cnt = a.blk_cnt;
-  d.n_blk = (int)((a.T + route_block_tokens(a.dtype) - 1) / route_block_tokens(a.dtype));
+  d.n_blk = route_num_blocks(a.dtype, a.T, a.H);
   fmmoe_status st;
   if (a.dtype == FMMOE_BF16) {
     st = launch_route_tc(h, d, s);
