@@ -165,35 +165,31 @@ __device__ __forceinline__ float group8_sum(float v) {
   return v;
 }
 
-// Softmax / top-k / gates for rows [row_lo, row_lo + n_rows) of the tile (n_rows a multiple of
-// 32).  The logits of a row are the sum, in rank order, of the `split` partial tiles held in the
-// shared memory of the cluster's CTAs (ls_addr[q] = address of rank q's tile), plus the bias.
+__device__ __forceinline__ int group8_min_int(int v) {
+#pragma unroll
+  for (int o = 4; o; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Softmax / top-k / gates for n_rows (a multiple of 32) token rows whose logits (bias included)
+// sit in shared memory, row pitch ldl (odd).  Eight lanes per token, four tokens per warp.
 // NV = logits per lane (expert e = lane8 + 8 j), NV * 8 >= E.
 template <int NV>
-__device__ __forceinline__ void route_tail_group8(const uint32_t* ls_addr, int split, int ldl, const float* bias_s,
-                                                  long long row0, int row_lo, int n_rows, uint32_t* emask, int words,
-                                                  const RouteDev& a) {
+__device__ __forceinline__ void route_tail_group8(const float* Lr, int ldl, long long t_first, int n_rows, uint32_t* emask,
+                                                  int words, const RouteDev& a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 3, l8 = lane & 7;
   const int E = a.E;
   for (int it = 0; it < n_rows / 32; ++it) {
     // rows of one warp are 8 apart: with an odd row pitch the four groups hit distinct banks
-    const int rl = it * 32 + g * 8 + warp;   // row inside this CTA's share
-    const int r = row_lo + rl;               // row inside the tile
-    const long long t = row0 + r;
+    const int rl = it * 32 + g * 8 + warp;
+    const long long t = t_first + rl;
     const bool tok_ok = t < a.T;
     float z[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
       const int e = l8 + 8 * j;
-      float v = -INFINITY;
-      if (e < E) {
-        const uint32_t off = (uint32_t)(r * ldl + e) * 4u;
-        v = ld_cluster_f32(ls_addr[0] + off);
-        for (int q = 1; q < split; ++q) v += ld_cluster_f32(ls_addr[q] + off);
-        v += bias_s[e];
-      }
-      z[j] = v;
+      z[j] = e < E ? Lr[rl * ldl + e] : -INFINITY;
     }
     if (a.logits && tok_ok) {
 #pragma unroll
@@ -216,32 +212,25 @@ __device__ __forceinline__ void route_tail_group8(const uint32_t* ls_addr, int s
     }
     const int k_t = tok_ok ? ((a.reduce_on && a.is_visual[t]) ? a.Kv : a.K) : 0;
     const int k_warp = __reduce_max_sync(0xffffffffu, k_t);
-    uint32_t taken = 0;
     float denom = 0.f;
     float sel_p[2] = {0.f, 0.f};
     int sel_e[2] = {-1, -1};
     for (int i = 0; i < k_warp; ++i) {
-      // two independent scan chains (even / odd j), merged; a strict comparison while walking
-      // upwards keeps the lower expert index among equal logits
-      float b0 = -INFINITY, b1 = -INFINITY;
-      int e0 = 0x7fffffff, e1 = 0x7fffffff;
+      // largest remaining logit of the token, then the lowest expert index that holds it
+      // (a taken entry is overwritten with -inf; real logits are finite)
+      float bv = z[0];
 #pragma unroll
-      for (int j = 0; j < NV; j += 2) {
-        if (l8 + 8 * j < E && !((taken >> j) & 1u) && (z[j] > b0 || e0 == 0x7fffffff)) { b0 = z[j]; e0 = l8 + 8 * j; }
-        if (j + 1 < NV && l8 + 8 * (j + 1) < E && !((taken >> (j + 1)) & 1u) && (z[j + 1] > b1 || e1 == 0x7fffffff)) {
-          b1 = z[j + 1]; e1 = l8 + 8 * (j + 1);
-        }
-      }
-      float bv = b0; int be = e0;
-      if (e1 != 0x7fffffff && (be == 0x7fffffff || b1 > bv || (b1 == bv && e1 < be))) { bv = b1; be = e1; }
+      for (int j = 1; j < NV; ++j) bv = fmaxf(bv, z[j]);
+      bv = group8_max(bv);
+      int be = 0x7fffffff;
 #pragma unroll
-      for (int o = 4; o; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oe = __shfl_xor_sync(0xffffffffu, be, o);
-        if (oe != 0x7fffffff && (be == 0x7fffffff || ov > bv || (ov == bv && oe < be))) { bv = ov; be = oe; }
-      }
+      for (int j = NV - 1; j >= 0; --j)
+        if (z[j] == bv) be = l8 + 8 * j;
+      be = group8_min_int(be);
       if (i < k_t) {
-        if ((be & 7) == l8) taken |= 1u << (be >> 3);
+#pragma unroll
+        for (int j = 0; j < NV; ++j)
+          if (l8 + 8 * j == be) z[j] = -INFINITY;
         const float p = __expf(bv - m);
         denom += p;
         if ((i & 7) == l8) { sel_p[i >> 3] = p; sel_e[i >> 3] = be; }
@@ -372,19 +361,48 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   // be left waiting.
   cluster_sync_all();
   if (!failed) {
-    uint32_t ls_addr[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) ls_addr[q] = cluster_map_shared(smem_u32(Ls), q < split ? q : 0);
     const int n_rows = RT_BM / split, row_lo = krank * n_rows, words = n_rows / 32;
+    // This CTA's rows of the logits tile = sum over the cluster's partial tiles, in rank order,
+    // plus the bias.  The rows are one contiguous, 16-byte aligned run of every CTA's tile
+    // (32 rows * pitch * 4 bytes), read from the peers with 16-byte distributed-shared-memory
+    // loads and written to Lr (row pitch ldl, after the tile).
+    // (a single-CTA cluster owns the whole tile and adds the bias in place)
+    float* Lr = split == 1 ? Ls : reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(Ls + RT_BM * ldl) + 15) & ~uintptr_t(15));
+    {
+      uint32_t peer[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) peer[q] = cluster_map_shared(smem_u32(Ls + row_lo * ldl), q < split ? q : 0);
+      const int n4 = n_rows * ldl / 4;
+      for (int i = threadIdx.x; i < n4; i += RT_THREADS) {
+        float4 acc4 = ld_cluster_v4f32(peer[0] + i * 16);
+#pragma unroll
+        for (int q = 1; q < 4; ++q) {
+          if (q < split) {
+            const float4 v = ld_cluster_v4f32(peer[q] + i * 16);
+            acc4.x += v.x; acc4.y += v.y; acc4.z += v.z; acc4.w += v.w;
+          }
+        }
+        // bias by column: element index -> column
+        const int e0 = (i * 4) % ldl;
+        float vals[4] = {acc4.x, acc4.y, acc4.z, acc4.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          int e = e0 + c; if (e >= ldl) e -= ldl;
+          Lr[i * 4 + c] = vals[c] + (e < FMMOE_MAX_EXPERTS ? bias_s[e] : 0.f);
+        }
+      }
+    }
+    __syncthreads();
+    const long long t_first = (long long)row0 + row_lo;
     switch ((a.E + 31) / 32) {
-      case 1: route_tail_group8<4>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
-      case 2: route_tail_group8<8>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
-      case 3: route_tail_group8<12>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
-      case 4: route_tail_group8<16>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
-      case 5: route_tail_group8<20>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
-      case 6: route_tail_group8<24>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
-      case 7: route_tail_group8<28>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
-      default: route_tail_group8<32>(ls_addr, split, ldl, bias_s, row0, row_lo, n_rows, emask, words, a); break;
+      case 1: route_tail_group8<4>(Lr, ldl, t_first, n_rows, emask, words, a); break;
+      case 2: route_tail_group8<8>(Lr, ldl, t_first, n_rows, emask, words, a); break;
+      case 3: route_tail_group8<12>(Lr, ldl, t_first, n_rows, emask, words, a); break;
+      case 4: route_tail_group8<16>(Lr, ldl, t_first, n_rows, emask, words, a); break;
+      case 5: route_tail_group8<20>(Lr, ldl, t_first, n_rows, emask, words, a); break;
+      case 6: route_tail_group8<24>(Lr, ldl, t_first, n_rows, emask, words, a); break;
+      case 7: route_tail_group8<28>(Lr, ldl, t_first, n_rows, emask, words, a); break;
+      default: route_tail_group8<32>(Lr, ldl, t_first, n_rows, emask, words, a); break;
     }
     // the token block of this CTA: rows [row_lo, row_lo + n_rows) of the tile
     if (split == 1) emit_block_ranks<4>(emask, (long long)row0, blockIdx.x, a);
@@ -485,7 +503,8 @@ static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s)
   while (tmem_cols < (d.E + 31) / 32 * 32) tmem_cols *= 2;
   // the logits tile [128][32*ceil(E/32)+1] fp32 overlays the stage buffers once the GEMM is done
   size_t tile_bytes = (size_t)stages * stage_bytes;
-  const size_t logit_bytes = (size_t)RT_BM * ((d.E + 31) / 32 * 32 + 1) * 4;
+  const size_t ldl_bytes = (size_t)((d.E + 31) / 32 * 32 + 1) * 4;
+  const size_t logit_bytes = RT_BM * ldl_bytes + (split > 1 ? (RT_BM / split) * ldl_bytes + 16 : 0);   // partial tile (+ this CTA's summed rows)
   if (logit_bytes > tile_bytes) tile_bytes = (logit_bytes + 1023) / 1024 * 1024;
   const size_t smem = tile_bytes + FMMOE_MAX_EXPERTS * 20 + (2 * RT_MAX_STAGES + 1) * 8 + 16 + 1024;
   CUtensorMap mx, mw;
