@@ -107,13 +107,13 @@ static fmmoe_status check_common(fmmoe_handle* h, const fmmoe_layer_desc* d, con
 
 static fmmoe_status run_route(fmmoe_handle* h, const fmmoe_layer_desc& d, const fmmoe_weights& w, const void* x,
                               const uint8_t* is_visual, int64_t T, uint32_t flags, const RoutePtrs& r,
-                              bool need_permute, cudaStream_t s) {
+                              bool need_permute, float* acc_zero, cudaStream_t s) {
   RouteArgs ra;
   ra.x = x; ra.router_w = w.router_w; ra.router_b = w.router_b; ra.is_visual = is_visual;
   ra.T = T; ra.H = d.hidden; ra.E = d.n_experts; ra.K = d.top_k; ra.Kv = d.top_k_vis;
   ra.reduce_on = (flags & FMMOE_FLAG_REDUCE_ON) ? 1 : 0; ra.dtype = d.dtype;
   ra.logits = r.logits; ra.probs = r.probs; ra.topk_idx = r.topk_idx; ra.topk_w = r.topk_w;
-  ra.inv_row = r.inv_row; ra.blk_cnt = r.blk_cnt;
+  ra.inv_row = r.inv_row; ra.blk_cnt = r.blk_cnt; ra.acc_zero = acc_zero; ra.misc_zero = r.misc;
   fmmoe_status st = launch_route(h, ra, s);
   if (st != FMMOE_OK || !need_permute) return st;
   PermuteArgs pa;
@@ -216,10 +216,9 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_route(fmmoe
   if (T == 0) return FMMOE_OK;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);
-  FMMOE_CUDA_TRY(cudaMemsetAsync(ws + pl.misc_off, 0, pl.acc_off - pl.misc_off, s));
   const RoutePtrs r = bind_route(pl, ws, out);
   const bool need_permute = out && (out->expert_off || out->row_token || out->inv_row);
-  return run_route(h, *d, *w, x, is_visual, T, flags, r, need_permute, s);
+  return run_route(h, *d, *w, x, is_visual, T, flags, r, need_permute, nullptr, s);
 }
 
 extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward(fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w,
@@ -236,9 +235,9 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);
   const bool det = flags & FMMOE_FLAG_DETERMINISTIC;
-  FMMOE_CUDA_TRY(cudaMemsetAsync(ws + pl.zero_off, 0, pl.zero_bytes, s));
   const RoutePtrs r = bind_route(pl, ws, route);
-  st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, s);
+  // the router clears the scheduler words and (atomic mode) the fp32 accumulator it owns rows of
+  st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, det ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s);
   if (st != FMMOE_OK) return st;
 
   FfnArgs fa = {};

@@ -6,6 +6,7 @@
 #include <cuda_bf16.h>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace fmmoe {
 
@@ -37,6 +38,8 @@ template <> struct Vec4<__nv_bfloat16> {
 
 template <typename T>
 __global__ void finalize_kernel(const FinalizeDev a) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int hv = a.H / 4;
   const long long n = a.T * hv;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
@@ -79,8 +82,8 @@ fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_
   if (blocks > cap) blocks = cap;
   {
     ProfScope ps(h, FMMOE_KERNEL_FINALIZE, s);
-    if (a.dtype == FMMOE_BF16) finalize_kernel<__nv_bfloat16><<<(int)blocks, threads, 0, s>>>(d);
-    else finalize_kernel<float><<<(int)blocks, threads, 0, s>>>(d);
+    if (a.dtype == FMMOE_BF16) FMMOE_CUDA_TRY(launch_pdl(finalize_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(threads), 0, s, 1, d));
+    else FMMOE_CUDA_TRY(launch_pdl(finalize_kernel<float>, dim3((unsigned)blocks), dim3(threads), 0, s, 1, d));
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 1;

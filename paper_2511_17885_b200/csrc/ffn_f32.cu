@@ -3,6 +3,7 @@
 // same two GEMMs and the same combine as the tensor-core path, tiles of 32 rows x
 // 64 columns, 256 threads, 2 x 4 outputs per thread.
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace fmmoe {
 
@@ -31,6 +32,8 @@ __global__ void __launch_bounds__(F_THREADS) ffn_f32_kernel(const F32Params p) {
   __shared__ float B0s[F_BN][F_BK + 1];
   __shared__ float B1s[MODE == 0 ? F_BN : 1][F_BK + 1];
   __shared__ long long s_arow[F_BM];   // source row of A for each tile row, -1 if none
+  pdl_launch_dependents();
+  pdl_wait();
   const bool routed = p.mtiles != nullptr;
   int group, row0, rows;
   if (routed) {
@@ -124,14 +127,14 @@ fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   p.b0 = static_cast<const float*>(a.w->w_gate); p.b1 = static_cast<const float*>(a.w->w_up);
   p.out = static_cast<float*>(a.act);
   if (a.max_mtiles > 0) {
-    { ProfScope prof_(h, FMMOE_KERNEL_GEMM1, s); ffn_f32_kernel<0><<<dim3(a.max_mtiles, (I + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(p); }
+    { ProfScope prof_(h, FMMOE_KERNEL_GEMM1, s); FMMOE_CUDA_TRY(launch_pdl(ffn_f32_kernel<0>, dim3(a.max_mtiles, (I + F_BN - 1) / F_BN), dim3(F_THREADS), 0, s, 1, p)); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     // routed GEMM-2
     F32Params q = p;
     q.K = I; q.N = H; q.a = static_cast<const float*>(a.act);
     q.b0 = static_cast<const float*>(a.w->w_down); q.b1 = nullptr;
     q.out = a.y; q.acc = a.acc; q.deterministic = a.deterministic;
-    { ProfScope prof_(h, FMMOE_KERNEL_GEMM2, s); ffn_f32_kernel<1><<<dim3(a.max_mtiles, (H + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(q); }
+    { ProfScope prof_(h, FMMOE_KERNEL_GEMM2, s); FMMOE_CUDA_TRY(launch_pdl(ffn_f32_kernel<1>, dim3(a.max_mtiles, (H + F_BN - 1) / F_BN), dim3(F_THREADS), 0, s, 1, q)); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     h->launches += 2;
   }
@@ -140,13 +143,13 @@ fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
     ps.mt_per_shared = mtps; ps.T = a.T; ps.K = H; ps.N = Is; ps.a = static_cast<const float*>(a.x);
     ps.b0 = static_cast<const float*>(a.w->ws_gate); ps.b1 = static_cast<const float*>(a.w->ws_up);
     ps.out = static_cast<float*>(a.act_sh);
-    { ProfScope prof_(h, FMMOE_KERNEL_GEMM1, s); ffn_f32_kernel<0><<<dim3(Ns * mtps, (Is + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(ps); }
+    { ProfScope prof_(h, FMMOE_KERNEL_GEMM1, s); FMMOE_CUDA_TRY(launch_pdl(ffn_f32_kernel<0>, dim3(Ns * mtps, (Is + F_BN - 1) / F_BN), dim3(F_THREADS), 0, s, 1, ps)); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     F32Params qs = ps;
     qs.K = Is; qs.N = H; qs.a = static_cast<const float*>(a.act_sh);
     qs.b0 = static_cast<const float*>(a.w->ws_down); qs.b1 = nullptr;
     qs.out = a.ysh; qs.acc = a.acc; qs.deterministic = a.deterministic;
-    { ProfScope prof_(h, FMMOE_KERNEL_GEMM2, s); ffn_f32_kernel<1><<<dim3(Ns * mtps, (H + F_BN - 1) / F_BN), F_THREADS, 0, s>>>(qs); }
+    { ProfScope prof_(h, FMMOE_KERNEL_GEMM2, s); FMMOE_CUDA_TRY(launch_pdl(ffn_f32_kernel<1>, dim3(Ns * mtps, (H + F_BN - 1) / F_BN), dim3(F_THREADS), 0, s, 1, qs)); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     h->launches += 2;
   }

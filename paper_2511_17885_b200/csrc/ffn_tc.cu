@@ -138,6 +138,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_launch_dependents();
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < G_STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
@@ -155,6 +156,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // barriers, tensor memory and descriptors are set up; everything below reads what earlier
+  // kernels of the stream wrote
+  pdl_wait();
   const int n_mt_r = p.n_mtiles ? *p.n_mtiles : 0;
   const int total_tiles = n_mt_r * p.seg[0].n_nblocks + p.shared_mtiles * p.seg[1].n_nblocks;
 
@@ -425,9 +429,9 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
     h->tc_attr_set = true;
   }
   const int grid = h->sm_count;
-  { ProfScope ps(h, FMMOE_KERNEL_GEMM1, s); ffn_tc_kernel<0><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(A1r, A1s, G1r, U1r, G1s, U1s, p1); }
+  { ProfScope ps(h, FMMOE_KERNEL_GEMM1, s); FMMOE_CUDA_TRY(launch_pdl(ffn_tc_kernel<0>, dim3(grid), dim3(G_THREADS), G_SMEM_BYTES, s, 1, A1r, A1s, G1r, U1r, G1s, U1s, p1)); }
   FMMOE_CUDA_TRY(cudaGetLastError());
-  { ProfScope ps(h, FMMOE_KERNEL_GEMM2, s); ffn_tc_kernel<1><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(A2r, A2s, D2r, D2r, D2s, D2s, p2); }
+  { ProfScope ps(h, FMMOE_KERNEL_GEMM2, s); FMMOE_CUDA_TRY(launch_pdl(ffn_tc_kernel<1>, dim3(grid), dim3(G_THREADS), G_SMEM_BYTES, s, 1, A2r, A2s, D2r, D2r, D2s, D2s, p2)); }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 2;
   return FMMOE_OK;

@@ -5,6 +5,7 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <utility>
 #include <vector>
 
 #include "../../include/fmmoe.h"
@@ -90,12 +91,35 @@ struct ProfScope {
     if (_e != cudaSuccess) return FMMOE_ERR_CUDA;    \
   } while (0)
 
+// Launch with programmatic dependent launch allowed (the kernel calls pdl_wait() before it touches
+// data of earlier kernels), optionally as clusters of `cluster_x` CTAs.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                     unsigned cluster_x, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster_x; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr; cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- launchers (each returns after enqueueing; *launches is incremented per kernel) ----
 struct RouteArgs {
   const void* x; const void* router_w; const float* router_b; const uint8_t* is_visual;
   int64_t T; int H, E, K, Kv; int reduce_on; int dtype;
   float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row;
   int32_t* blk_cnt;   // [E][n_blk]: per token block (route_block_tokens) and expert, the number of selections
+  float* acc_zero;    // [T,H] fp32 combine accumulator to clear (each CTA its own tokens' rows), or NULL
+  int32_t* misc_zero; // int32 [8] scheduler words to clear, or NULL
 };
 // bf16 router: number of CTAs (a cluster) that share one 128-token tile by splitting the
 // contraction.  Few tiles => split, so that more SMs stream X.

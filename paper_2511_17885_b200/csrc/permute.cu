@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace fmmoe {
 
@@ -28,6 +29,8 @@ struct PermuteDev {
 __global__ void __launch_bounds__(P_THREADS) scan_kernel(const PermuteDev a) {
   __shared__ int s_cnt[FMMOE_MAX_EXPERTS], s_off[FMMOE_MAX_EXPERTS + 1], s_tile0[FMMOE_MAX_EXPERTS + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
+  pdl_wait();
   // per expert: exclusive scan over the token blocks, 32 blocks per step
   for (int e = warp; e < a.E; e += P_THREADS / 32) {
     int32_t* row = a.blk_cnt + (long long)e * a.n_blk;
@@ -85,6 +88,8 @@ __global__ void __launch_bounds__(P_THREADS) scan_kernel(const PermuteDev a) {
 }
 
 __global__ void __launch_bounds__(256) scatter_kernel(const PermuteDev a) {
+  pdl_launch_dependents();
+  pdl_wait();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= a.T * a.K) return;
   const int e = a.topk_idx[i];
@@ -101,6 +106,8 @@ __global__ void __launch_bounds__(256) scatter_kernel(const PermuteDev a) {
 __global__ void gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ row_token,
                                    const int32_t* __restrict__ expert_off, int E, long long p_max, int row_vec,
                                    uint4* __restrict__ xp) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int P = expert_off[E];
   const int warps = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -122,8 +129,8 @@ fmmoe_status launch_permute(fmmoe_handle* h, const PermuteArgs& a, cudaStream_t 
   const long long pairs = a.T * a.K;
   {
     ProfScope ps(h, FMMOE_KERNEL_PERMUTE, s);
-    scan_kernel<<<1, P_THREADS, 0, s>>>(d);
-    scatter_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, s>>>(d);
+    FMMOE_CUDA_TRY(launch_pdl(scan_kernel, dim3(1), dim3(P_THREADS), 0, s, 1, d));
+    FMMOE_CUDA_TRY(launch_pdl(scatter_kernel, dim3((unsigned)((pairs + 255) / 256)), dim3(256), 0, s, 1, d));
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 2;
@@ -140,8 +147,8 @@ fmmoe_status launch_gather_rows(fmmoe_handle* h, const void* x, const int32_t* r
   if (blocks > cap) blocks = cap;
   {
     ProfScope ps(h, FMMOE_KERNEL_GATHER, s);
-    gather_rows_kernel<<<(int)blocks, threads, 0, s>>>(static_cast<const uint4*>(x), row_token, expert_off, E, p_max,
-                                                       row_vec, static_cast<uint4*>(xp));
+    FMMOE_CUDA_TRY(launch_pdl(gather_rows_kernel, dim3((unsigned)blocks), dim3(threads), 0, s, 1, static_cast<const uint4*>(x), row_token,
+                              expert_off, E, (long long)p_max, row_vec, static_cast<uint4*>(xp)));
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 1;

@@ -15,6 +15,7 @@
 #include <pthread.h>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace fmmoe {
 
@@ -50,6 +51,8 @@ __global__ void __launch_bounds__(1024) vis_index_kernel(const PruneDev a, const
   __shared__ int s_warp[32];
   __shared__ int s_running;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
+  pdl_wait();
   const long long lo = sq.seq_off[b], hi = sq.seq_off[b + 1];
   if (tid == 0) s_running = 0;
   __syncthreads();
@@ -151,6 +154,8 @@ __device__ __forceinline__ void score_window(const PruneDev& a, const int32_t* m
 __global__ void __launch_bounds__(256) window_score_kernel(const PruneDev a, const PruneSeqs sq) {
   const int lane = threadIdx.x & 31;
   const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  pdl_launch_dependents();
+  pdl_wait();
   if (gw >= sq.win_off[sq.n_seq]) return;
   int b = 0;
   while (b + 1 < sq.n_seq && gw >= sq.win_off[b + 1]) ++b;
@@ -210,6 +215,8 @@ __global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const Pr
   __shared__ double s_red[32];
   __shared__ int s_warp[32];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
+  pdl_wait();
   const int n_f = sq.n_vis[b] / a.W;
   const int w0 = sq.win_off[b];
   const int m = sq.m[b], d = sq.d[b];
@@ -365,6 +372,8 @@ __global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const Pr
   __shared__ float s_red[8][MAXW + 1];
   __shared__ float s_scale;
   const long long row = row_base + blockIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   if (blockIdx.x >= n_rows) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const T* X = static_cast<const T*>(a.x);
@@ -573,24 +582,24 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
     for (int i = 0; i <= nb; ++i) rel.win_off[i] -= win_base;
     PruneDev al = a;
     al.sim = a.sim + win_base; al.asum = a.asum + win_base; al.action = a.action + win_base;
-    { ProfScope ps(h, FMMOE_KERNEL_PRUNE_INDEX, s); vis_index_kernel<<<nb, 1024, 0, s>>>(al, rel); }
+    { ProfScope ps(h, FMMOE_KERNEL_PRUNE_INDEX, s); FMMOE_CUDA_TRY(launch_pdl(vis_index_kernel, dim3(nb), dim3(1024), 0, s, 1, al, rel)); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     h->launches += 1;
     if (n_win > 0) {
-      { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SCORE, s); window_score_kernel<<<(n_win + 7) / 8, 256, 0, s>>>(al, rel); }
+      { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SCORE, s); FMMOE_CUDA_TRY(launch_pdl(window_score_kernel, dim3((n_win + 7) / 8), dim3(256), 0, s, 1, al, rel)); }
       FMMOE_CUDA_TRY(cudaGetLastError());
       h->launches += 1;
     }
-    { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SELECT, s); select_kernel<<<nb, 1024, sel_smem, s>>>(al, rel); }
+    { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SELECT, s); FMMOE_CUDA_TRY(launch_pdl(select_kernel, dim3(nb), dim3(1024), sel_smem, s, 1, al, rel)); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     h->launches += 1;
     const long long rows = rel.out_off[nb] - rel.out_off[0];
     if (rows > 0) {
       ProfScope ps(h, FMMOE_KERNEL_PRUNE_COMPACT, s);
       if (dtype == FMMOE_BF16)
-        compact_kernel<__nv_bfloat16><<<(unsigned)rows, 256, 0, s>>>(al, rel, rel.out_off[0], rows);
+        FMMOE_CUDA_TRY(launch_pdl(compact_kernel<__nv_bfloat16>, dim3((unsigned)rows), dim3(256), 0, s, 1, al, rel, (long long)rel.out_off[0], (long long)rows));
       else
-        compact_kernel<float><<<(unsigned)rows, 256, 0, s>>>(al, rel, rel.out_off[0], rows);
+        FMMOE_CUDA_TRY(launch_pdl(compact_kernel<float>, dim3((unsigned)rows), dim3(256), 0, s, 1, al, rel, (long long)rel.out_off[0], (long long)rows));
       FMMOE_CUDA_TRY(cudaGetLastError());
       h->launches += 1;
     }

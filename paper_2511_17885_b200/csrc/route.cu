@@ -27,6 +27,7 @@ struct RouteDev {
   long long T; int H, E, K, Kv, reduce_on, e_pad;
   float* logits; float* probs; int32_t* topk_idx; float* topk_w; int32_t* inv_row;
   int32_t* blk_cnt; int n_blk;   // [E][n_blk] selections of each token block per expert
+  float* acc_zero; int32_t* misc_zero;   // combine accumulator [T,H] / scheduler words to clear (or NULL)
 };
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -274,11 +275,7 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const int ldl = nch * 32 + 1;                 // odd pitch of the logits tile in shared memory
   float* Ls = reinterpret_cast<float*>(smem);   // [128][ldl], overlays the stage buffers after the GEMM
 
-  for (int e = threadIdx.x; e < FMMOE_MAX_EXPERTS; e += RT_THREADS) {
-    bias_s[e] = (a.bias && e < a.E) ? a.bias[e] : 0.f;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) emask[e * 4 + w] = 0;
-  }
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
     for (int i = 0; i < stages; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
     mbar_init(tfull_bar, 1);
@@ -288,6 +285,12 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   if (warp == 1) {
     tmem_alloc(tmem_slot, (uint32_t)tmem_cols);
     tmem_relinquish();
+  }
+  pdl_wait();   // from here on: global memory that earlier kernels of the stream may have written
+  for (int e = threadIdx.x; e < FMMOE_MAX_EXPERTS; e += RT_THREADS) {
+    bias_s[e] = (a.bias && e < a.E) ? a.bias[e] : 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) emask[e * 4 + w] = 0;
   }
   tc_fence_before();
   __syncthreads();
@@ -329,7 +332,23 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       if (ok) umma_commit(tfull_bar);
       else { atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
-  } else if (warp >= 4) {
+  } else if (warp < 4) {
+    // warps 2-3 have nothing to do until the tail: clear this CTA's rows of the layer's fp32
+    // combine accumulator (and, once, the tile schedulers' counters) while the GEMM streams
+    if (a.misc_zero && blockIdx.x == 0 && threadIdx.x == 64)
+      for (int i = 1; i < 8; ++i) a.misc_zero[i] = 0;
+    if (a.acc_zero) {
+      const int n_rows = RT_BM / split;
+      const long long t_lo = (long long)row0 + krank * n_rows;
+      long long t_hi = t_lo + n_rows;
+      if (t_hi > a.T) t_hi = a.T;
+      if (t_lo < t_hi) {
+        float4* dst = reinterpret_cast<float4*>(a.acc_zero + t_lo * a.H);
+        const long long n4 = (t_hi - t_lo) * a.H / 4;
+        for (long long i = threadIdx.x - 64; i < n4; i += 64) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+  } else {
     // accumulator complete => every stage buffer has been consumed: reuse them for the logits
     const int q = warp & 3;
     if (mbar_wait(tfull_bar, 0, abort_flag)) {
@@ -430,6 +449,16 @@ __global__ void __launch_bounds__(R_THREADS) route_f32_kernel(const RouteDev a) 
   uint32_t* emask = reinterpret_cast<uint32_t*>(Ls + R_BM * ldl);   // [e_pad] one word per expert (32 tokens)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const long long t0 = (long long)blockIdx.x * R_BM;
+  pdl_launch_dependents();
+  pdl_wait();
+  if (a.misc_zero && blockIdx.x == 0 && tid == 0)
+    for (int i = 1; i < 8; ++i) a.misc_zero[i] = 0;
+  if (a.acc_zero) {   // clear this block's rows of the combine accumulator
+    long long t_hi = t0 + R_BM;
+    if (t_hi > a.T) t_hi = a.T;
+    const long long n = (t_hi - t0) * a.H;
+    for (long long i = tid; i < n; i += R_THREADS) a.acc_zero[t0 * a.H + i] = 0.f;
+  }
   const float* X = static_cast<const float*>(a.x);
   const float* W = static_cast<const float*>(a.w);
   for (int i = tid; i < e_pad; i += R_THREADS) emask[i] = 0;
@@ -512,18 +541,10 @@ static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s)
   if (!route_map(h, &mw, d.w, (uint64_t)d.E, (uint64_t)d.H, (uint32_t)d.e_pad)) return FMMOE_ERR_CUDA;
   FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const int tiles = (int)((d.T + RT_BM - 1) / RT_BM);
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(tiles * split), 1, 1);
-  cfg.blockDim = dim3(RT_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)split; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
   {
     ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
-    FMMOE_CUDA_TRY(cudaLaunchKernelEx(&cfg, route_tc_kernel, mx, mw, d, stages, tmem_cols, (int)tile_bytes, split, h->d_status));
+    FMMOE_CUDA_TRY(launch_pdl(route_tc_kernel, dim3((unsigned)(tiles * split)), dim3(RT_THREADS), smem, s, (unsigned)split, mx, mw, d,
+                              stages, tmem_cols, (int)tile_bytes, split, h->d_status));
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   return FMMOE_OK;
@@ -537,7 +558,7 @@ static fmmoe_status launch_nt(fmmoe_handle* h, const RouteDev& d, int grid, cuda
   FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_f32_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
-    route_f32_kernel<NT><<<grid, R_THREADS, smem, s>>>(d);
+    FMMOE_CUDA_TRY(launch_pdl(route_f32_kernel<NT>, dim3(grid), dim3(R_THREADS), smem, s, 1, d));
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   return FMMOE_OK;
@@ -550,7 +571,7 @@ fmmoe_status launch_route(fmmoe_handle* h, const RouteArgs& a, cudaStream_t s) {
   d.T = a.T; d.H = a.H; d.E = a.E; d.K = a.K; d.Kv = a.Kv; d.reduce_on = a.reduce_on;
   d.e_pad = (a.E + 31) / 32 * 32;
   d.logits = a.logits; d.probs = a.probs; d.topk_idx = a.topk_idx; d.topk_w = a.topk_w;
-  d.inv_row = a.inv_row; d.blk_cnt = a.blk_cnt;
+  d.inv_row = a.inv_row; d.blk_cnt = a.blk_cnt; d.acc_zero = a.acc_zero; d.misc_zero = a.misc_zero;
   d.n_blk = route_num_blocks(a.dtype, a.T, a.H);
   fmmoe_status st;
   if (a.dtype == FMMOE_BF16) {
