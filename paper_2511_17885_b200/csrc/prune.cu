@@ -208,10 +208,35 @@ __device__ __forceinline__ void bitonic_sort_u64(unsigned long long* keys, int n
   __syncthreads();
 }
 
+// Ascending bitonic sort of up to 1024 keys, ONE key per thread of a 1024-thread CTA (threads
+// past the data hold the maximum key).  Partners less than 32 apart exchange by shuffle, the
+// others through `xch` (1024 keys of shared memory).  Returns the key of position threadIdx.x.
+__device__ __forceinline__ unsigned long long bitonic_sort_1024_regs(unsigned long long key, int n, unsigned long long* xch) {
+  const int tid = threadIdx.x;
+  for (int k = 2; k <= n; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      unsigned long long other;
+      if (j < 32) {
+        other = __shfl_xor_sync(0xffffffffu, key, j);
+      } else {
+        xch[tid] = key;
+        __syncthreads();
+        other = xch[tid ^ j];
+        __syncthreads();
+      }
+      const bool up = (tid & k) == 0;          // this block of k keys sorts ascending
+      const bool lower = (tid & j) == 0;       // this thread keeps the smaller of the pair if ascending
+      const bool take_min = up == lower;
+      key = take_min ? (key < other ? key : other) : (key > other ? key : other);
+    }
+  }
+  return key;
+}
+
 // One CTA per sequence.  Eq. 12-13 (one rounding to fp32), then the merge set (Eq. 15) and the
 // drop set by SORTING (score, window index) keys: position p of the sorted order is rank p.
 __global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const PruneSeqs sq) {
-  extern __shared__ unsigned long long s_keys[];   // [n_pad]
+  extern __shared__ unsigned long long s_keys[];   // [max(n_pad, 1024)] keys, then [n_pad] action bytes
   __shared__ double s_red[32];
   __shared__ int s_warp[32];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -223,6 +248,8 @@ __global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const Pr
   const bool have_attn = a.attn != nullptr;
   int n_pad = 2;
   while (n_pad < n_f) n_pad <<= 1;
+  const bool in_regs = n_pad <= 1024;
+  uint8_t* s_action = reinterpret_cast<uint8_t*>(s_keys + (n_pad > 1024 ? n_pad : 1024));   // [n_pad]
 
   // Eq. 12: divide by the largest window sum (0 if all sums are 0)
   double amax = 0.0;
@@ -235,45 +262,51 @@ __global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const Pr
     amax = s_red[0];
     for (int i = 1; i < 32; ++i) amax = fmax(amax, s_red[i]);
   }
-  // keys of the redundancy ranking: (C descending, window ascending)
-  for (int i = tid; i < n_pad; i += 1024) {
-    unsigned long long key = ~0ull;
-    if (i < n_f) {
-      const double S = a.sim[w0 + i];
-      float c32;
-      if (have_attn) {
-        const double ab = amax > 0.0 ? a.asum[w0 + i] / amax : 0.0;
-        // Eq. 13 in fp64 without contraction, then ONE rounding to fp32
-        c32 = (float)__dsub_rn(__dmul_rn(a.alpha, S), __dmul_rn(__dsub_rn(1.0, a.alpha), ab));
-      } else {
-        c32 = (float)S;
-      }
-      key = ((unsigned long long)(~ordered_bits(c32)) << 32) | (unsigned)i;
-      a.action[w0 + i] = 0;
+  // key of the redundancy ranking: (C descending, window ascending); Eq. 13 in fp64 without
+  // contraction, then ONE rounding to fp32
+  auto c_key = [&](int i) -> unsigned long long {
+    if (i >= n_f) return ~0ull;
+    const double S = a.sim[w0 + i];
+    float c32;
+    if (have_attn) {
+      const double ab = amax > 0.0 ? a.asum[w0 + i] / amax : 0.0;
+      c32 = (float)__dsub_rn(__dmul_rn(a.alpha, S), __dmul_rn(__dsub_rn(1.0, a.alpha), ab));
+    } else {
+      c32 = (float)S;
     }
-    s_keys[i] = key;
-  }
+    return ((unsigned long long)(~ordered_bits(c32)) << 32) | (unsigned)i;
+  };
+  // key of the drop ranking among the windows that were not merged: (A_bar ascending, window ascending)
+  auto a_key = [&](int i) -> unsigned long long {
+    if (i >= n_f || s_action[i] != 0) return ~0ull;
+    const float a32 = (float)(amax > 0.0 ? a.asum[w0 + i] / amax : 0.0);
+    return ((unsigned long long)ordered_bits(a32) << 32) | (unsigned)i;
+  };
+  for (int i = tid; i < n_pad; i += 1024) s_action[i] = 0;
   __syncthreads();
   if (m + d > 0) {
-    bitonic_sort_u64(s_keys, n_pad);
     const int n_act = have_attn ? m : m + d;
-    for (int p = tid; p < n_act && p < n_f; p += 1024)
-      a.action[w0 + (int)(s_keys[p] & 0xffffffffu)] = p < m ? 1 : 2;
-    __syncthreads();
-    if (have_attn && d > 0) {
-      // drop ranking among the windows that were not merged: (A_bar ascending, window ascending)
-      for (int i = tid; i < n_pad; i += 1024) {
-        unsigned long long key = ~0ull;
-        if (i < n_f && a.action[w0 + i] == 0) {
-          const float a32 = (float)(amax > 0.0 ? a.asum[w0 + i] / amax : 0.0);
-          key = ((unsigned long long)ordered_bits(a32) << 32) | (unsigned)i;
-        }
-        s_keys[i] = key;
-      }
+    if (in_regs) {
+      const unsigned long long k = bitonic_sort_1024_regs(c_key(tid), n_pad, s_keys);
+      if (tid < n_act && tid < n_f) s_action[(int)(k & 0xffffffffu)] = tid < m ? 1 : 2;
+    } else {
+      for (int i = tid; i < n_pad; i += 1024) s_keys[i] = c_key(i);
       __syncthreads();
       bitonic_sort_u64(s_keys, n_pad);
-      for (int p = tid; p < d && p < n_f - m; p += 1024)
-        a.action[w0 + (int)(s_keys[p] & 0xffffffffu)] = 2;
+      for (int p = tid; p < n_act && p < n_f; p += 1024) s_action[(int)(s_keys[p] & 0xffffffffu)] = p < m ? 1 : 2;
+    }
+    __syncthreads();
+    if (have_attn && d > 0) {
+      if (in_regs) {
+        const unsigned long long k = bitonic_sort_1024_regs(a_key(tid), n_pad, s_keys);
+        __syncthreads();
+        if (tid < d && tid < n_f - m) s_action[(int)(k & 0xffffffffu)] = 2;
+      } else {
+        for (int i = tid; i < n_pad; i += 1024) s_keys[i] = a_key(i);
+        __syncthreads();
+        bitonic_sort_u64(s_keys, n_pad);
+        for (int p = tid; p < d && p < n_f - m; p += 1024) s_action[(int)(s_keys[p] & 0xffffffffu)] = 2;
+      }
       __syncthreads();
     }
   }
@@ -282,19 +315,30 @@ __global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const Pr
   const long long lo = sq.seq_off[b], hi = sq.seq_off[b + 1];
   const int per = (int)((hi - lo + 1023) / 1024);
   const long long t_begin = lo + (long long)tid * per;
-  auto kind_of = [&](long long t) -> int {   // kind of the emitted row, -1 = nothing emitted
-    const int v = a.vrank[t];
+  auto kind_of = [&](int v) -> int {   // kind of the emitted row for a token of vision rank v, -1 = nothing emitted
     if (v < 0) return 0;
     const int w = v / a.W;
     if (w >= n_f) return 1;
-    const uint8_t act = a.action[w0 + w];
+    const uint8_t act = s_action[w];
     if (act == 0) return 1;
     return (act == 1 && v - w * a.W == 0) ? 2 : -1;
   };
-  int cnt = 0;
-  for (int i = 0; i < per; ++i) {
+  constexpr int CACHE = 8;             // kinds of the first tokens of the run stay in registers
+  int kinds[CACHE];
+#pragma unroll
+  for (int i = 0; i < CACHE; ++i) {
     const long long t = t_begin + i;
-    if (t < hi && kind_of(t) >= 0) ++cnt;
+    kinds[i] = (i < per && t < hi) ? a.vrank[t] : -2;      // independent loads first
+  }
+  int cnt = 0;
+#pragma unroll
+  for (int i = 0; i < CACHE; ++i) {
+    kinds[i] = kinds[i] == -2 ? -1 : kind_of(kinds[i]);
+    cnt += kinds[i] >= 0;
+  }
+  for (int i = CACHE; i < per; ++i) {
+    const long long t = t_begin + i;
+    if (t < hi && kind_of(a.vrank[t]) >= 0) ++cnt;
   }
   int incl = cnt;
 #pragma unroll
@@ -315,11 +359,7 @@ __global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const Pr
   }
   __syncthreads();
   long long pos = sq.out_off[b] + (warp ? s_warp[warp - 1] : 0) + (incl - cnt);
-  for (int i = 0; i < per; ++i) {
-    const long long t = t_begin + i;
-    if (t >= hi) break;
-    const int kd = kind_of(t);
-    if (kd < 0) continue;
+  auto emit = [&](long long t, int kd) {
     if (pos < sq.out_off[b + 1]) {
       a.keep_idx_ws[pos] = (int32_t)t;
       a.kind_ws[pos] = (uint8_t)kd;
@@ -328,6 +368,15 @@ __global__ void __launch_bounds__(1024) select_kernel(const PruneDev a, const Pr
       if (a.is_visual_out) a.is_visual_out[pos] = kd != 0;
     }
     ++pos;
+  };
+#pragma unroll
+  for (int i = 0; i < CACHE; ++i)
+    if (kinds[i] >= 0) emit(t_begin + i, kinds[i]);
+  for (int i = CACHE; i < per; ++i) {
+    const long long t = t_begin + i;
+    if (t >= hi) break;
+    const int kd = kind_of(a.vrank[t]);
+    if (kd >= 0) emit(t, kd);
   }
   if (tid == 0 && s_warp[31] != (int)(sq.out_off[b + 1] - sq.out_off[b])) atomicCAS(a.status, 0, DEV_INTERNAL);
 }
@@ -542,7 +591,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
   if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < wp.total) return FMMOE_ERR_WORKSPACE;
   size_t sel_pad = 2;
   while ((int64_t)sel_pad < max_nf) sel_pad <<= 1;
-  const size_t sel_smem = sel_pad * 8;   // sort keys of the longest sequence's windows
+  const size_t sel_smem = (sel_pad > 1024 ? sel_pad : 1024) * 8 + sel_pad;   // sort keys + action bytes of the longest sequence
   if (sel_smem > (size_t)h->max_smem_optin - 1024) return FMMOE_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);

@@ -332,9 +332,9 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       if (ok) umma_commit(tfull_bar);
       else { atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
-  } else if (warp < 4) {
-    // warps 2-3 have nothing to do until the tail: clear this CTA's rows of the layer's fp32
-    // combine accumulator (and, once, the tile schedulers' counters) while the GEMM streams
+  } else {
+    // warps 2-7 have nothing to do while the GEMM streams: clear this CTA's rows of the layer's
+    // fp32 combine accumulator (and, once, the tile schedulers' counters)
     if (a.misc_zero && blockIdx.x == 0 && threadIdx.x == 64)
       for (int i = 1; i < 8; ++i) a.misc_zero[i] = 0;
     if (a.acc_zero) {
@@ -345,10 +345,11 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       if (t_lo < t_hi) {
         float4* dst = reinterpret_cast<float4*>(a.acc_zero + t_lo * a.H);
         const long long n4 = (t_hi - t_lo) * a.H / 4;
-        for (long long i = threadIdx.x - 64; i < n4; i += 64) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (long long i = threadIdx.x - 64; i < n4; i += RT_THREADS - 64) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
-  } else {
+  }
+  if (warp >= 4) {
     // accumulator complete => every stage buffer has been consumed: reuse them for the logits
     const int q = warp & 3;
     if (mbar_wait(tfull_bar, 0, abort_flag)) {
