@@ -418,6 +418,9 @@ def run_stack(args):
     for _ in range(W):
         wl.step()
     h.check_status("warm-up")
+    if not bool(torch.isfinite(wl.x_out.float()).all()):
+        raise SystemExit("bench.py: the stack's output is not finite")
+    out_std = float(wl.x_out.float().std())
     clocks = ClockSampler(local)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     D.barrier(); torch.cuda.synchronize()
@@ -496,7 +499,9 @@ def run_stack(args):
     if rank == 0:
         conf = stack_describe(sc, n_layers)
         conf.update({"parallelism": f"replicas x{world} (no collective)", "tokens_per_layer": [t for t, _ in shapes],
-                     "final_tokens": wl.out_off[-1]})
+                     "final_tokens": wl.out_off[-1], "output_std": out_std,
+                     "weights": "N(0, 0.02^2); down-projections N(0, (0.02/sqrt(2*layers))^2) so that the norm-free "
+                                "residual stack stays at unit scale"})
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
                 "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": sc.layer.dtype, "data": "synthetic", "config": conf, "clocks": clocks.summary(),

@@ -2,6 +2,7 @@
 // sequence of one MoE layer (Section 3.1):
 //   clear -> route (Eq. 1-3, 5 + histogram) -> permute-by-expert -> [gather rows]
 //   -> GEMM-1 + SwiGLU -> GEMM-2 + combine (Eq. 4) -> finalize.
+#include <stdlib.h>
 #include <string.h>
 
 #include "internal.h"
@@ -161,6 +162,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
   h->launches = 0;
   h->d_status = nullptr; h->h_status = nullptr; h->encode_tiled = nullptr;
   h->tc_attr_set = false; h->profiling = false; h->ev_used = 0;
+  { const char* dbg = getenv("FMMOE_DEBUG_SYNC"); h->debug_sync = dbg && dbg[0] == '1'; h->debug_seq = 0; }
   if (cudaMalloc(&h->d_status, 256) != cudaSuccess || cudaMemset(h->d_status, 0, 256) != cudaSuccess ||
       cudaMallocHost(&h->h_status, 256) != cudaSuccess) {
     if (h->d_status) cudaFree(h->d_status);

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <stdio.h>
 
 #include <utility>
 #include <vector>
@@ -21,6 +22,8 @@ struct fmmoe_handle {
   bool tc_attr_set;     // dynamic shared memory opt-in done for the tensor-core kernels
   // optional kernel timeline
   bool profiling;
+  bool debug_sync;      // FMMOE_DEBUG_SYNC=1: synchronise after every kernel and report the first CUDA error on stderr
+  int64_t debug_seq;    // kernels launched so far in debug mode
   std::vector<cudaEvent_t> ev_pool;
   size_t ev_used;
   struct ProfRec { int id; size_t start, stop; };
@@ -66,8 +69,8 @@ bool plan_workspace(const fmmoe_layer_desc& d, int64_t T, uint32_t flags, WsPlan
 
 // Brackets one kernel launch with events when the handle's timeline is on.
 struct ProfScope {
-  fmmoe_handle* h; cudaStream_t s; size_t rec; bool on;
-  ProfScope(fmmoe_handle* h_, int id, cudaStream_t s_) : h(h_), s(s_), rec(0), on(h_->profiling) {
+  fmmoe_handle* h; cudaStream_t s; size_t rec; bool on; int kid;
+  ProfScope(fmmoe_handle* h_, int id, cudaStream_t s_) : h(h_), s(s_), rec(0), on(h_->profiling), kid(id) {
     if (!on) return;
     while (h->ev_pool.size() < h->ev_used + 2) {
       cudaEvent_t e;
@@ -82,6 +85,15 @@ struct ProfScope {
   }
   ~ProfScope() {
     if (on) cudaEventRecord(h->ev_pool[h->prof[rec].stop], s);
+    if (h->debug_sync) {
+      ++h->debug_seq;
+      cudaError_t e = cudaStreamSynchronize(s);
+      if (e == cudaSuccess) e = cudaGetLastError();
+      if (e != cudaSuccess) {
+        fprintf(stderr, "fmmoe: kernel class %d (launch scope #%lld) failed: %s\n", kid, (long long)h->debug_seq, cudaGetErrorString(e));
+        h->debug_sync = false;   // report the first failure only
+      }
+    }
   }
 };
 

@@ -93,9 +93,10 @@ __global__ void __launch_bounds__(256) scatter_kernel(const PermuteDev a) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= a.T * a.K) return;
   const int e = a.topk_idx[i];
-  if (e < 0) return;                       // padded slot: inv_row already holds -1
+  if (e < 0 || e >= a.E) return;           // padded slot: inv_row already holds -1
   const long long t = i / a.K;
   const int row = a.expert_off[e] + a.blk_cnt[(long long)e * a.n_blk + (int)(t / a.blk_tokens)] + a.inv_row[i];
+  if (row < 0 || row >= a.expert_off[a.E]) return;   // cannot happen for a consistent routing record
   a.row_token[row] = (int32_t)t;
   a.row_gate[row] = a.topk_w[i];
   a.inv_row[i] = row;

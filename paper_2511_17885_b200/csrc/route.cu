@@ -60,6 +60,12 @@ __device__ __forceinline__ void route_tail(const float* Ls, int ldl, long long t
       for (int j = 0; j < NTL; ++j)
         if (lane + 32 * j < a.E) a.logits[t * a.E + lane + 32 * j] = v[j];
     }
+    // The shuffle reductions below need a total order: non-finite logits (overflowed activations
+    // upstream) are clamped and NaN counts as the lowest value, so that all lanes agree on every
+    // round's winner and each selected index is a valid, distinct expert.  Finite inputs are untouched.
+#pragma unroll
+    for (int j = 0; j < NTL; ++j)
+      if (lane + 32 * j < a.E) v[j] = fminf(fmaxf(v[j], -FLT_MAX), FLT_MAX);
     float m = v[0];
 #pragma unroll
     for (int j = 1; j < NTL; ++j) m = fmaxf(m, v[j]);
@@ -101,7 +107,7 @@ __device__ __forceinline__ void route_tail(const float* Ls, int ldl, long long t
       const bool sel = lane < k_t;
       a.topk_idx[t * a.K + lane] = sel ? my_idx : -1;
       a.topk_w[t * a.K + lane] = sel ? p / denom : 0.f;
-      if (sel) atomicOr(&emask[my_idx], 1u << r);   // one 32-bit word per expert: the block has 32 tokens
+      if (sel && (unsigned)my_idx < (unsigned)a.E) atomicOr(&emask[my_idx], 1u << r);   // one 32-bit word per expert: the block has 32 tokens
     }
   }
 }
@@ -124,7 +130,7 @@ __device__ __forceinline__ void emit_block_ranks(const uint32_t* emask, long lon
     if (t >= a.T) break;
     const int e = __ldcg(a.topk_idx + t * a.K + (it - r * a.K));   // written by this CTA before the barrier
     int rank = -1;
-    if (e >= 0) {
+    if (e >= 0 && e < a.E) {
       rank = __popc(emask[e * WORDS + (r >> 5)] & ((1u << (r & 31)) - 1u));
 #pragma unroll
       for (int w = 0; w < WORDS; ++w)
@@ -197,6 +203,13 @@ __device__ __forceinline__ void route_tail_group8(const float* Lr, int ldl, long
       for (int j = 0; j < NV; ++j)
         if (l8 + 8 * j < E) a.logits[t * E + l8 + 8 * j] = z[j];
     }
+    // The selection below marks a taken entry with -inf and looks experts up by value, so it needs
+    // finite logits: non-finite ones (overflowed activations upstream) are clamped, NaN counts as the
+    // lowest value.  Finite inputs are untouched; whatever the input, every selected index is a
+    // valid, distinct expert.
+#pragma unroll
+    for (int j = 0; j < NV; ++j)
+      if (l8 + 8 * j < E) z[j] = fminf(fmaxf(z[j], -FLT_MAX), FLT_MAX);
     float m = z[0];
 #pragma unroll
     for (int j = 1; j < NV; ++j) m = fmaxf(m, z[j]);
@@ -245,7 +258,7 @@ __device__ __forceinline__ void route_tail_group8(const float* Lr, int ldl, long
           const bool sel = slot < k_t;
           a.topk_idx[t * a.K + slot] = sel ? sel_e[h] : -1;
           a.topk_w[t * a.K + slot] = sel ? sel_p[h] / denom : 0.f;   // Eq. 5
-          if (sel) atomicOr(&emask[sel_e[h] * words + (rl >> 5)], 1u << (rl & 31));
+          if (sel && (unsigned)sel_e[h] < (unsigned)E) atomicOr(&emask[sel_e[h] * words + (rl >> 5)], 1u << (rl & 31));
         }
       }
     }

@@ -261,14 +261,18 @@ def stack_layer_weights_torch(cfg: StackCfg, layer: int, device: str):
         t.normal_(0.0, std, generator=g)
         return t.to(dt)
 
+    # Residual-branch scaling: without normalisation layers (the stack has none) a residual stack whose
+    # down-projections have the same std as the other weights grows quadratically per layer and
+    # overflows bf16 by layer ~9; std / sqrt(2 * n_layers) keeps the activations at unit scale.
+    down_std = 0.02 / float(np.sqrt(2.0 * cfg.n_layers))
     w = {"router_w": draw((E, H)),
          "router_b": torch.empty(E, device=device, dtype=torch.float32).normal_(0.0, lc.router_bias_std, generator=g)
          if lc.router_bias_std > 0 else None,
-         "w_gate": draw((E, I, H)), "w_up": draw((E, I, H)), "w_down": draw((E, H, I)),
+         "w_gate": draw((E, I, H)), "w_up": draw((E, I, H)), "w_down": draw((E, H, I), down_std),
          "ws_gate": None, "ws_up": None, "ws_down": None}
     if lc.n_shared:
         Is = lc.shared_inter
         w["ws_gate"] = draw((lc.n_shared, Is, H))
         w["ws_up"] = draw((lc.n_shared, Is, H))
-        w["ws_down"] = draw((lc.n_shared, H, Is))
+        w["ws_down"] = draw((lc.n_shared, H, Is), down_std)
     return w

@@ -1,0 +1,171 @@
+"""GPU parity at the full workload sizes, in the launch configuration the benchmark times.
+
+C1 (DeepSeekMoE-style, 2,432 tokens), C2 (Qwen3-MoE-style, 3,584 tokens) and its batch of four,
+C3 (pruning sweep at 75/50/25 % followed by the layer on the kept tokens) and C4 (24 layers,
+8 x 2,432 tokens, K_v = 3 from layer 3, pruning after layers 3 and 12).  Integer results (expert
+selections on the kernel's own fp32 logits, permutation, keep-sets) are compared bit-exactly over
+ALL tokens; layer outputs on sampled tokens the oracle evaluates one by one (every expert a token
+selected, in fp64), within the bf16 tolerance of 2e-2 (max over rows of |y - ref|_inf / |ref|_inf)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fmmoe_oracle as O
+from paper_2511_17885_b200 import binding as B
+from paper_2511_17885_b200 import inputs as I
+from paper_2511_17885_b200.workload import LayerWorkload
+from gpu_util import handle, host, row_rel_err
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+def oracle_rows(x, mask, w, K, Kv, reduce_on, logits32, rows, add_residual=False):
+    """Oracle layer output for the sampled token rows only (routing from the kernel's fp32 logits)."""
+    r = O.route(x[rows], w["router_w"], w.get("router_b"), mask[rows], K, Kv, reduce_on, logits32=logits32[rows])
+    out = O.moe_combine(x[rows], r["topk_idx"], r["topk_w"], w, add_residual)
+    return r, out
+
+
+def check_layer_workload(cfg, n_samples=96, seed=0):
+    h = handle()
+    wl = LayerWorkload(cfg, h, device=0, prune=None, keep_host=True)
+    T, E, K = cfg.n_tokens, cfg.n_experts, cfg.top_k
+    wl.route = {"logits": torch.empty(T, E, dtype=torch.float32, device="cuda"),
+                "probs": torch.empty(T, E, dtype=torch.float32, device="cuda"),
+                "topk_idx": torch.empty(T, K, dtype=torch.int32, device="cuda"),
+                "topk_w": torch.empty(T, K, dtype=torch.float32, device="cuda"),
+                "expert_off": torch.empty(E + 1, dtype=torch.int32, device="cuda"),
+                "row_token": torch.empty(T * K, dtype=torch.int32, device="cuda"),
+                "inv_row": torch.empty(T, K, dtype=torch.int32, device="cuda")}
+    wl.step()
+    h.check_status()
+    x, mask, w = wl.host["x"], wl.host["mask"], wl.host["w"]
+    g = {k: host(v) for k, v in wl.route.items()}
+    # every token: selection (on the kernel's logits), gates, permutation
+    full = O.route(x, w["router_w"], w.get("router_b"), mask, K, cfg.top_k_vis, True, logits32=g["logits"])
+    assert np.array_equal(g["topk_idx"], full["topk_idx"])
+    assert np.abs(g["topk_w"] - full["topk_w"]).max() < 2e-5
+    assert np.abs(g["probs"] - full["probs"]).max() < 2e-5
+    scale = np.abs(full["logits"]).max()
+    assert np.abs(g["logits"] - full["logits"]).max() / scale < 2e-5
+    off, row_token, inv = O.permutation(full["topk_idx"], E)
+    assert np.array_equal(g["expert_off"], off)
+    assert np.array_equal(g["row_token"][:off[-1]], row_token)
+    assert np.array_equal(g["inv_row"], inv)
+    k_t = (full["topk_idx"] >= 0).sum(1)
+    assert set(k_t[mask == 1].tolist()) == {cfg.top_k_vis} and set(k_t[mask == 0].tolist()) == {K}
+    # sampled tokens: layer output
+    rows = np.sort(np.random.default_rng(seed).choice(T, n_samples, replace=False))
+    _, ref = oracle_rows(x, mask, w, K, cfg.top_k_vis, True, g["logits"], rows)
+    err = row_rel_err(host(wl.out)[rows], ref)
+    assert err < TOL, err
+    return wl, g
+
+
+def test_c1_full():
+    wl, g = check_layer_workload(I.C1)
+    assert int(g["expert_off"][-1]) == 2304 * 3 + 128 * 6
+
+
+def test_c2_full_and_batch_of_four():
+    check_layer_workload(I.C2)
+    wl, g = check_layer_workload(I.C2X4, n_samples=64)
+    assert int(g["expert_off"][-1]) == 4 * (3328 * 4 + 256 * 8)
+
+
+def test_c3_sweep_keep_sets_and_downstream_forward():
+    cfg = I.C3
+    h = handle()
+    wl = LayerWorkload(cfg, h, device=0, prune=None, keep_host=True)
+    T, E, K = cfg.n_tokens, cfg.n_experts, cfg.top_k
+    wl.route["logits"] = torch.empty(T, E, dtype=torch.float32, device="cuda")
+    wl.step()
+    x, mask, w = wl.host["x"], wl.host["mask"], wl.host["w"]
+    probs = host(wl.route["probs"])
+    kept_expected = {0.75: 2500, 0.5: 1666, 0.25: 836}
+    for pc in cfg.prune:
+        n_ret = I.retain_counts(wl.n_vis, pc.retain)
+        pr = h.fmmoe_prune_visual(B.prune_params(pc.window, pc.gamma, pc.alpha), wl.route["probs"], None, wl.x, wl.mask,
+                                  wl.seq_off, wl.n_vis, n_ret)
+        h.check_status()
+        ref = O.prune_visual(x, mask, probs, None, wl.seq_off, n_ret, pc.window, pc.alpha, pc.gamma)
+        assert np.array_equal(host(pr["keep_idx"]), ref["keep_idx"])           # bit-exact keep-set
+        assert np.array_equal(host(pr["kind"]), ref["kind"])
+        assert int(host(pr["is_visual_out"]).sum()) == kept_expected[pc.retain]
+        assert row_rel_err(host(pr["x_out"]), ref["x_out"]) < TOL
+        # downstream layer on the kept tokens + 256 text tokens
+        xk, mk = pr["x_out"], pr["is_visual_out"]
+        Tk = xk.shape[0]
+        route = {"logits": torch.empty(Tk, E, dtype=torch.float32, device="cuda"),
+                 "topk_idx": torch.empty(Tk, K, dtype=torch.int32, device="cuda")}
+        out = h.fmmoe_moe_forward(wl.desc, wl.ws, xk, mk, B.FLAG_REDUCE_ON, route=route)
+        h.check_status()
+        xk_h, mk_h, lg = host(xk), host(mk), host(route["logits"])
+        full = O.route(xk_h, w["router_w"], None, mk_h, K, cfg.top_k_vis, True, logits32=lg)
+        assert np.array_equal(host(route["topk_idx"]), full["topk_idx"])
+        rows = np.sort(np.random.default_rng(5).choice(Tk, 48, replace=False))
+        _, refo = oracle_rows(xk_h, mk_h, w, K, cfg.top_k_vis, True, lg, rows)
+        assert row_rel_err(host(out)[rows], refo) < TOL
+
+
+def test_c4_stack_full():
+    """24 layers at full size: the stack driver against the same sequence of single-layer calls (bit for
+    bit with the fixed-order combine), keep-sets of both stages bit-exact against the oracle, and sampled
+    layer outputs teacher-forced against the oracle at the first layer, both pruning layers and the last."""
+    sc = I.C4
+    lc = sc.layer
+    h = handle()
+    dev = "cuda:0"
+    td = torch.bfloat16
+    x, mask, seq_off, n_vis = I.make_tokens(lc)
+    xd = torch.from_numpy(x).to(dev).to(td).contiguous()
+    md = torch.from_numpy(mask).to(dev)
+    layers = [I.stack_layer_weights_torch(sc, l, dev) for l in range(sc.n_layers)]
+    wstructs = [B.make_weights(w) for w in layers]
+    desc = B.make_desc(lc.hidden, lc.n_experts, lc.inter, lc.n_shared, lc.shared_inter, lc.top_k, lc.top_k_vis, td)
+    stages = [(l, pc.retain, B.prune_params(pc.window, pc.gamma, pc.alpha), None) for l, pc in sorted(sc.prune_after.items())]
+    y, vis_out, out_off = h.fmmoe_stack_forward(desc, wstructs, sc.reduce_from, stages, xd, md, seq_off, n_vis,
+                                                B.FLAG_DETERMINISTIC)
+    h.check_status("stack")
+    assert out_off[-1] == 8 * (577 + 128)
+    assert bool(torch.isfinite(y.float()).all())
+    E, K = lc.n_experts, lc.top_k
+    checked = {0, 3, 12, sc.n_layers - 1}
+    cur_x, cur_m, cur_off, cur_vis = xd, md, list(seq_off), [int(v) for v in n_vis]
+    rng = np.random.default_rng(9)
+    for l in range(sc.n_layers):
+        T = cur_x.shape[0]
+        reduce_on = l >= sc.reduce_from
+        lf = B.FLAG_DETERMINISTIC | B.FLAG_RESIDUAL | (B.FLAG_REDUCE_ON if reduce_on else 0)
+        route = {"probs": torch.empty(T, E, dtype=torch.float32, device=dev)}
+        if l in checked:
+            route["logits"] = torch.empty(T, E, dtype=torch.float32, device=dev)
+            route["topk_idx"] = torch.empty(T, K, dtype=torch.int32, device=dev)
+        out = h.fmmoe_moe_forward(desc, wstructs[l], cur_x, cur_m, lf, route=route)
+        if l in checked:
+            wh = {k: (None if v is None else v.float().cpu().numpy()) for k, v in layers[l].items()}
+            xh, mh, lg = host(cur_x), host(cur_m), host(route["logits"])
+            full = O.route(xh, wh["router_w"], wh["router_b"], mh, K, lc.top_k_vis, reduce_on, logits32=lg)
+            assert np.array_equal(host(route["topk_idx"]), full["topk_idx"]), f"layer {l}: selection"
+            rows = np.sort(rng.choice(T, 32, replace=False))
+            _, ref = oracle_rows(xh, mh, wh, K, lc.top_k_vis, reduce_on, lg, rows, add_residual=True)
+            assert row_rel_err(host(out)[rows], ref) < TOL, f"layer {l}: output"
+        if l in sc.prune_after:
+            pc = sc.prune_after[l]
+            eta = I.retain_counts(n_vis, pc.retain)
+            pr = h.fmmoe_prune_visual(B.prune_params(pc.window, pc.gamma, pc.alpha), route["probs"], None, out, cur_m,
+                                      cur_off, cur_vis, eta)
+            ref = O.prune_visual(host(out), host(cur_m), host(route["probs"]), None, cur_off, eta, pc.window, pc.alpha,
+                                 pc.gamma)
+            assert np.array_equal(host(pr["keep_idx"]), ref["keep_idx"]), f"layer {l}: keep-set"
+            assert np.array_equal(host(pr["kind"]), ref["kind"])
+            n_text = [cur_off[b + 1] - cur_off[b] - cur_vis[b] for b in range(len(cur_vis))]
+            cur_off = pr["out_seq_off"]
+            cur_vis = [cur_off[b + 1] - cur_off[b] - n_text[b] for b in range(len(n_text))]
+            cur_x, cur_m = pr["x_out"], pr["is_visual_out"]
+        else:
+            cur_x = out
+    h.check_status("layerwise")
+    assert cur_off == out_off
+    assert torch.equal(cur_x, y) and torch.equal(cur_m, vis_out)

@@ -121,3 +121,31 @@ def test_route_empty_and_invalid():
         h.fmmoe_route(un, w, torch.zeros(4, 72, dtype=torch.bfloat16, device="cuda"),
                       torch.zeros(4, dtype=torch.uint8, device="cuda"), 1)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_route_non_finite_activations_still_give_valid_distinct_experts(dtype):
+    """Overflowed activations upstream (inf / nan rows) must not turn into out-of-range expert indices:
+    the router clamps non-finite logits before it selects, so every token gets k distinct experts in
+    [0, E) and the permutation stays consistent."""
+    r = np.random.default_rng(8)
+    T, H, E, K, Kv = 300, 128, 24, 4, 2
+    x = I.round_to_storage(r.standard_normal((T, H)), dtype)
+    x[5] = np.inf; x[17] = np.nan; x[40, ::2] = -np.inf; x[41] = 3e38
+    w = I.round_to_storage(0.05 * r.standard_normal((E, H)), dtype)
+    mask = (r.random(T) < 0.5).astype(np.uint8)
+    td = TDT[dtype]
+    desc = B.make_desc(H, E, 64, 0, 64, K, Kv, td)
+    ws = B.make_weights({"router_w": dev(w, td)})
+    out = handle().fmmoe_route(desc, ws, dev(x, td), dev(mask), B.FLAG_REDUCE_ON)
+    handle().check_status()
+    idx = host(out["topk_idx"])
+    for t in range(T):
+        k = Kv if mask[t] else K
+        sel = idx[t, :k]
+        assert (sel >= 0).all() and (sel < E).all() and len(set(sel.tolist())) == k, (t, sel)
+        assert (idx[t, k:] == -1).all()
+    off, row_token, inv = O.permutation(idx, E)
+    assert np.array_equal(host(out["expert_off"]), off)
+    assert np.array_equal(host(out["row_token"])[:off[-1]], row_token)
+    assert np.array_equal(host(out["inv_row"]), inv)
