@@ -337,6 +337,36 @@ def prune_visual(x, is_visual, probs, attn, seq_off, n_retain, window, alpha, ga
             "out_seq_off": out_off, "per_seq": outs}
 
 
+def attention_importance(q_last: np.ndarray, k: np.ndarray, seq_off: Sequence[int],
+                         scale: Optional[float] = None) -> np.ndarray:
+    """Eq. 7: A_hat = A[:, -1] of the head-averaged attention matrix, i.e. for each sequence the
+    attention weights FROM its last token (the last text token of [T_v, T_t]) TO every token of the
+    sequence, softmax over the sequence per head, then the mean over heads.  Returned for every
+    token; the pruning stage reads the vision entries (Eq. 11).
+
+    q_last [n_seq, n_heads, d]: the last tokens' queries; k [T, n_kv_heads, d]: the keys.
+    READING: head h uses kv head h // (n_heads / n_kv_heads) (grouped-query attention, as in the
+    paper's backbones); the last token sees the whole sequence, so the causal mask plays no role;
+    scale defaults to 1/sqrt(d)."""
+    q = np.asarray(q_last, F64)
+    kk = np.asarray(k, F64)
+    n_seq, n_heads, d = q.shape
+    T, n_kv, _ = kk.shape
+    group = n_heads // n_kv
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    out = np.zeros(T, F64)
+    for b in range(n_seq):
+        lo, hi = int(seq_off[b]), int(seq_off[b + 1])
+        if hi == lo:
+            continue
+        for h in range(n_heads):
+            z = scale * (kk[lo:hi, h // group, :] @ q[b, h])
+            e = np.exp(z - z.max())
+            out[lo:hi] += e / e.sum()
+    return out / n_heads
+
+
 # ----------------------------------------------------------------------------
 # Appendix D / E: closed forms
 # ----------------------------------------------------------------------------

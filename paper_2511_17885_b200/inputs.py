@@ -230,6 +230,25 @@ def retain_counts(n_vis: np.ndarray, retain: float) -> np.ndarray:
     return np.floor(np.asarray(n_vis, dtype=np.float64) * retain + 1e-9).astype(np.int64)
 
 
+# Appendix A: per-model pruning hyper-parameters, keyed by the OVERALL retention of the three-stage schedule.
+PAPER_SCHEDULES = {
+    "internvl3.5": {"layers": (5, 8, 12), "window": 5,
+                    0.75: dict(alpha=0.5, gamma=0.025), 0.50: dict(alpha=0.6, gamma=0.05), 0.25: dict(alpha=1.0, gamma=0.1)},
+    "deepseek-vl2": {"layers": (2, 5, 8), "window": 3,
+                     0.75: dict(alpha=0.3, gamma=0.05), 0.50: dict(alpha=0.9, gamma=0.05), 0.25: dict(alpha=0.7, gamma=0.2)},
+}
+
+
+def paper_schedule(model: str, overall_retain: float) -> Dict[int, PruneCfg]:
+    """The paper's three-stage schedule (Appendix A and D): pruning after three designated layers with the
+    same per-stage ratio beta = r^(1/3), so that stage t keeps beta^t of the ORIGINAL vision tokens."""
+    sc = PAPER_SCHEDULES[model]
+    hp = sc[overall_retain]
+    beta = overall_retain ** (1.0 / 3.0)
+    return {layer: PruneCfg(window=sc["window"], gamma=hp["gamma"], alpha=hp["alpha"], retain=beta ** (t + 1))
+            for t, layer in enumerate(sc["layers"])}
+
+
 def interleaved_mask(n_tokens: int, rng: np.random.Generator, p_vis: float = 0.7) -> np.ndarray:
     """A modality mask with text and vision runs interleaved (edge-case tests)."""
     m = np.zeros(n_tokens, dtype=np.uint8)

@@ -41,3 +41,12 @@ def test_vision_is_smooth_text_is_not():
 def test_attention_importance_normalised():
     a = I.make_attention_importance(I.C2)
     assert a.dtype == np.float32 and abs(a[:I.C2.n_vis].sum() - 1) < 1e-4 and (a[I.C2.n_vis:] == 0).all()
+
+
+def test_paper_three_stage_schedule():
+    sch = I.paper_schedule("internvl3.5", 0.5)
+    assert sorted(sch) == [5, 8, 12] and all(pc.window == 5 and pc.gamma == 0.05 and pc.alpha == 0.6 for pc in sch.values())
+    assert abs(sch[12].retain - 0.5) < 1e-12 and abs(sch[5].retain - 0.5 ** (1 / 3)) < 1e-12      # beta ~ 0.79
+    assert abs(round(sch[5].retain, 2) - 0.79) < 1e-9
+    d = I.paper_schedule("deepseek-vl2", 0.25)
+    assert sorted(d) == [2, 5, 8] and d[2].window == 3 and d[2].gamma == 0.2 and abs(round(d[2].retain, 2) - 0.63) < 1e-9

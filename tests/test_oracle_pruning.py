@@ -266,3 +266,64 @@ def test_stack_pruning_takes_effect_after_the_layer_and_reduce_from_is_inclusive
     p = O.prune_visual(b["out"], vis, b["probs"], None, off, [10], 2, 1.0, 0.1)
     c = O.moe_forward(p["x_out"], p["is_visual_out"], ws[2], 2, 1, True, add_residual=True)
     assert np.allclose(y, c["out"], atol=1e-12)
+
+
+# ---------------------------------------------------------------------------- Eq. 7
+def _full_causal_attention(Q, K, scale):
+    """Textbook attention probabilities of ONE head: softmax(mask(Q K^T * scale)), pure Python loops."""
+    L = Q.shape[0]
+    A = np.zeros((L, L))
+    for i in range(L):
+        z = [scale * sum(Q[i, c] * K[j, c] for c in range(Q.shape[1])) for j in range(i + 1)]
+        m = max(z)
+        e = [math.exp(v - m) for v in z]
+        tot = sum(e)
+        for j in range(i + 1):
+            A[i, j] = e[j] / tot
+    return A
+
+
+def test_attention_importance_is_the_last_row_of_head_averaged_causal_attention():
+    r = np.random.default_rng(0)
+    lens, n_heads, n_kv, d = [7, 4], 4, 2, 6
+    T = sum(lens)
+    seq_off = np.concatenate([[0], np.cumsum(lens)])
+    K = r.standard_normal((T, n_kv, d))
+    Qfull = r.standard_normal((T, n_heads, d))                 # queries of every token; only the last ones matter
+    q_last = np.stack([Qfull[seq_off[b + 1] - 1] for b in range(len(lens))])
+    got = O.attention_importance(q_last, K, seq_off)
+    want = np.zeros(T)
+    for b in range(len(lens)):
+        lo, hi = seq_off[b], seq_off[b + 1]
+        Abar = sum(_full_causal_attention(Qfull[lo:hi, h], K[lo:hi, h // (n_heads // n_kv)], 1 / math.sqrt(d))
+                   for h in range(n_heads)) / n_heads                                           # head-averaged A
+        want[lo:hi] = Abar[-1, :]                                                               # A[:, -1] of Eq. 7
+    assert np.allclose(got, want, atol=1e-14)
+
+
+def test_attention_importance_invariants():
+    r = np.random.default_rng(1)
+    lens = [9, 5, 12]
+    seq_off = np.concatenate([[0], np.cumsum(lens)])
+    T = sum(lens)
+    K = r.standard_normal((T, 2, 8)); q = r.standard_normal((3, 6, 8))
+    a = O.attention_importance(q, K, seq_off)
+    for b in range(3):
+        assert abs(a[seq_off[b]:seq_off[b + 1]].sum() - 1.0) < 1e-14          # a distribution per sequence
+    assert (a > 0).all()
+    # identical keys (or a zero query): uniform attention
+    Ku = np.tile(K[:1], (T, 1, 1))
+    au = O.attention_importance(q, Ku, seq_off)
+    for b in range(3):
+        assert np.allclose(au[seq_off[b]:seq_off[b + 1]], 1.0 / lens[b])
+    assert np.allclose(O.attention_importance(np.zeros_like(q), K, seq_off), au)
+    # a key aligned with every head's query and a huge scale: all the weight on that token
+    K2 = K.copy(); q2 = np.ones((3, 6, 8)); K2[:] = -np.ones(8); K2[4] = np.ones(8)
+    a2 = O.attention_importance(q2, K2, seq_off, scale=50.0)
+    assert abs(a2[4] - 1.0) < 1e-12 and a2[:4].max() < 1e-12
+    # grouped-query attention == multi-head attention on the expanded keys
+    Kx = np.repeat(K, 3, axis=1)
+    assert np.allclose(O.attention_importance(q, Kx, seq_off), a, atol=1e-15)
+    # a sequence's result does not depend on its neighbours
+    alone = O.attention_importance(q[1:2], K[seq_off[1]:seq_off[2]], [0, lens[1]])
+    assert np.allclose(alone, a[seq_off[1]:seq_off[2]], atol=1e-15)
