@@ -160,7 +160,7 @@ fmmoe_status fmmoe_moe_forward_host(fmmoe_handle *handle, const fmmoe_layer_desc
 enum {
   FMMOE_KERNEL_ROUTE = 0, FMMOE_KERNEL_PERMUTE = 1, FMMOE_KERNEL_GATHER = 2, FMMOE_KERNEL_GEMM1 = 3,
   FMMOE_KERNEL_GEMM2 = 4, FMMOE_KERNEL_FINALIZE = 5, FMMOE_KERNEL_PRUNE_INDEX = 6, FMMOE_KERNEL_PRUNE_SCORE = 7,
-  FMMOE_KERNEL_PRUNE_SELECT = 8, FMMOE_KERNEL_PRUNE_COMPACT = 9, FMMOE_KERNEL_COUNT = 10
+  FMMOE_KERNEL_PRUNE_SELECT = 8, FMMOE_KERNEL_PRUNE_COMPACT = 9, FMMOE_KERNEL_ATTN = 10, FMMOE_KERNEL_COUNT = 11
 };
 fmmoe_status fmmoe_profile_enable(fmmoe_handle *handle, int enable);
 fmmoe_status fmmoe_profile_reset(fmmoe_handle *handle);
@@ -214,6 +214,23 @@ fmmoe_status fmmoe_prune_visual(fmmoe_handle *handle, const fmmoe_prune_params *
                                 void *x_out, uint8_t *is_visual_out, int32_t *keep_idx, uint8_t *kind,
                                 int64_t *out_seq_off /* host [n_seq+1] */,
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Section 3.2.1, Eq. 7: cross-modal attention importance.  For every sequence, the attention
+ * weights of its LAST token (the last text token of [T_v, T_t]) to all tokens of the sequence,
+ * averaged over the attention heads:
+ *   attn_out[t] = (1 / n_heads) * sum_h softmax_over_the_sequence(scale * q_last[b, h] . k[., kv(h)])[t]
+ * with kv(h) = h / (n_heads / n_kv_heads) (grouped-query attention; n_kv_heads == n_heads is the
+ * plain multi-head case).  The last token attends to the whole sequence, so no mask is needed.
+ * fmmoe_prune_visual reads the entries at vision tokens (Eq. 11).  The attention layer itself is
+ * the caller's: q_last [n_seq, n_heads, head_dim] are that layer's queries of the last tokens,
+ * k [T, n_kv_heads, head_dim] its keys (as used in its own attention, e.g. after rotary
+ * embedding), both `dtype`, device.  attn_out: [T] fp32, device.  The mean over heads is taken in
+ * head order (reproducible).  head_dim any positive size; n_heads / n_kv_heads <= 16. */
+size_t fmmoe_attention_workspace_bytes(int64_t n_tokens, int32_t n_seq, int32_t n_heads);
+fmmoe_status fmmoe_attention_importance(fmmoe_handle *handle, const void *q_last, const void *k, int32_t dtype,
+                                        int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                        const int64_t *seq_off /* host [n_seq+1] */, int32_t n_seq,
+                                        float *attn_out, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* A stack of n_layers MoE layers of one shape with residual adds (x <- x + MoE_l(x)), the
  * setting of Section 3.1's start layer and of the multi-stage pruning schedule (Section 3.2,

@@ -94,6 +94,9 @@ def lib() -> C.CDLL:
                                      C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), i32,
                                      vp, vp, vp, vp, C.POINTER(i64), vp, sz, vp]
     L.fmmoe_prune_visual.restype = C.c_int
+    L.fmmoe_attention_workspace_bytes.argtypes = [i64, i32, i32]; L.fmmoe_attention_workspace_bytes.restype = sz
+    L.fmmoe_attention_importance.argtypes = [vp, vp, vp, i32, i32, i32, i32, C.c_float, C.POINTER(i64), i32, vp, vp, sz, vp]
+    L.fmmoe_attention_importance.restype = C.c_int
     L.fmmoe_stack_workspace_bytes.argtypes = [C.POINTER(LayerDesc), i64, i32, u32]
     L.fmmoe_stack_workspace_bytes.restype = sz
     L.fmmoe_stack_output_layout.argtypes = [C.POINTER(StackStage), i32, i32, C.POINTER(i64), C.POINTER(i64), i32,
@@ -221,7 +224,7 @@ class Handle:
         return int(lib().fmmoe_launch_count(self._h))
 
     KERNELS = ("route", "permute", "gather", "gemm1", "gemm2", "finalize", "prune_index", "prune_score",
-               "prune_select", "prune_compact")
+               "prune_select", "prune_compact", "attn")
 
     def profile_enable(self, on: bool = True):
         _check(lib().fmmoe_profile_enable(self._h, 1 if on else 0), "fmmoe_profile_enable")
@@ -314,6 +317,23 @@ class Handle:
                                         _stream()), "fmmoe_prune_visual")
         return {"x_out": x_out, "is_visual_out": vis_out, "keep_idx": keep_idx, "kind": kind,
                 "out_seq_off": [int(v) for v in oo]}
+
+    def fmmoe_attention_importance(self, q_last: torch.Tensor, k: torch.Tensor, seq_off, scale: Optional[float] = None,
+                                   out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Eq. 7: head-averaged attention of each sequence's last token to all its tokens.
+        q_last [n_seq, n_heads, d], k [T, n_kv_heads, d] -> attn [T] fp32."""
+        n_seq, n_heads, d = q_last.shape
+        T, n_kv, _ = k.shape
+        if scale is None:
+            scale = 1.0 / float(d) ** 0.5
+        if out is None:
+            out = torch.empty(T, dtype=torch.float32, device=k.device)
+        so = (C.c_int64 * (n_seq + 1))(*[int(v) for v in seq_off])
+        wsp, wsn = self._ws_args(int(lib().fmmoe_attention_workspace_bytes(T, n_seq, n_heads)))
+        _check(lib().fmmoe_attention_importance(self._h, _ptr(q_last), _ptr(k), _dtype_code(k.dtype), n_heads, n_kv, d,
+                                                C.c_float(scale), so, n_seq, _ptr(out), wsp, wsn, _stream()),
+               "fmmoe_attention_importance")
+        return out
 
     def fmmoe_stack_forward(self, desc: LayerDesc, layer_weights, reduce_from: int, stages, x: torch.Tensor,
                             is_visual: torch.Tensor, seq_off, n_vis, flags: int = 0,

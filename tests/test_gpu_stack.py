@@ -151,3 +151,55 @@ def test_stack_invalid_arguments():
     with pytest.raises(B.FmmoeError):      # two stages on one layer
         h.fmmoe_stack_forward(desc, [w, w], 0, [(0, 0.5, B.prune_params(3, 0.05), None),
                                                 (0, 0.3, B.prune_params(3, 0.05), None)], x, m, [0, 10], [10])
+
+
+def test_stack_paper_three_stage_schedule_with_attention():
+    """The paper's schedule (pruning after layers 2, 5, 8, W = 3, per-stage ratio r^(1/3), Appendix A hyper-
+    parameters for 50 %) with attention-guided scoring: C = alpha S - (1 - alpha) A_bar, drop by smallest A_bar.
+    Stack driver == layer-by-layer calls, keep-sets bit-exact against the oracle at every stage."""
+    dtype, td = "bf16", torch.bfloat16
+    n_layers, H, E, I_, K, Kv = 10, 128, 16, 64, 4, 2
+    sched = I.paper_schedule("deepseek-vl2", 0.5)
+    ws_host = make_stack(dtype, n_layers, H, E, I_, 1, 64, seed=70)
+    x, mask, seq_off, n_vis = tokens(dtype, [420, 333], H, seed=71)
+    desc = B.make_desc(H, E, I_, 1, 64, K, Kv, td)
+    wdev = [upload_weights(w, dtype) for w in ws_host]
+    wstructs = [B.make_weights(w) for w in wdev]
+    h = handle()
+    r = np.random.default_rng(72)
+    # the attention-importance vector of a stage has one entry per token of the sequence AS IT IS at that layer
+    stages, attn_dev, done = [], {}, []
+    for layer, pc in sorted(sched.items()):
+        off_here, _ = B.fmmoe_stack_output_layout(done, layer + 1, seq_off, n_vis)
+        a = dev(r.random(off_here[-1]).astype(np.float32))
+        attn_dev[layer] = a
+        st = (layer, pc.retain, B.prune_params(pc.window, pc.gamma, pc.alpha), a)
+        stages.append(st); done.append(st)
+    xd, md = dev(x, td), dev(mask)
+    flags = B.FLAG_DETERMINISTIC
+    y, vis_out, out_off = h.fmmoe_stack_forward(desc, wstructs, 1, stages, xd, md, seq_off, n_vis, flags)
+    h.check_status("stack")
+    cur_x, cur_m, cur_off, cur_vis = xd, md, list(seq_off), [int(v) for v in n_vis]
+    for l in range(n_layers):
+        T = cur_x.shape[0]
+        lf = flags | B.FLAG_RESIDUAL | (B.FLAG_REDUCE_ON if l >= 1 else 0)
+        route = {"probs": torch.empty(T, E, dtype=torch.float32, device="cuda")}
+        out = h.fmmoe_moe_forward(desc, wstructs[l], cur_x, cur_m, lf, route=route)
+        if l in sched:
+            pc = sched[l]
+            eta = I.retain_counts(n_vis, pc.retain)
+            pr = h.fmmoe_prune_visual(B.prune_params(pc.window, pc.gamma, pc.alpha), route["probs"], attn_dev[l], out,
+                                      cur_m, cur_off, cur_vis, eta)
+            ref = O.prune_visual(host(out), host(cur_m), host(route["probs"]), host(attn_dev[l]), cur_off, eta, pc.window,
+                                 pc.alpha, pc.gamma)
+            assert np.array_equal(host(pr["keep_idx"]), ref["keep_idx"]), f"stage after layer {l}"
+            assert np.array_equal(host(pr["kind"]), ref["kind"])
+            n_text = [cur_off[b + 1] - cur_off[b] - cur_vis[b] for b in range(len(cur_vis))]
+            cur_off = pr["out_seq_off"]
+            cur_vis = [cur_off[b + 1] - cur_off[b] - n_text[b] for b in range(len(n_text))]
+            cur_x, cur_m = pr["x_out"], pr["is_visual_out"]
+        else:
+            cur_x = out
+    assert cur_off == out_off and torch.equal(cur_x, y) and torch.equal(cur_m, vis_out)
+    kept = sum(cur_vis)
+    assert sum(int(v) for v in n_vis) * 0.5 <= kept < sum(int(v) for v in n_vis) * 0.5 + 2 * 3 * 3
