@@ -1,7 +1,8 @@
 // C-ABI entry points: handle, workspace planning, argument validation, and the launch
 // sequence of one MoE layer (Section 3.1):
-//   clear -> route (Eq. 1-3, 5 + histogram) -> permute-by-expert -> [gather rows]
-//   -> GEMM-1 + SwiGLU -> GEMM-2 + combine (Eq. 4) -> finalize.
+//   route (Eq. 1-3, 5; block counts and in-block ranks) -> permute-by-expert (scan, scatter)
+//   -> [copy of the routed rows into expert order, small batches] -> GEMM-1 (+ row gather by
+//   token, large batches) + SwiGLU -> GEMM-2 + combine (Eq. 4) -> finalize.
 #include <stdlib.h>
 #include <string.h>
 
@@ -253,8 +254,11 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward
   fa.ysh = det ? reinterpret_cast<float*>(ws + pl.ysh_off) : nullptr;
   fa.deterministic = det; fa.d_status = h->d_status;
   if (d->dtype == FMMOE_BF16) {
-    st = launch_gather_rows(h, x, r.row_token, r.expert_off, d->n_experts, pl.p_max, d->hidden, 2, fa.xp, s);
-    if (st != FMMOE_OK) return st;
+    fa.gather_in_gemm = gather_rows_in_gemm(T) ? 1 : 0;
+    if (!fa.gather_in_gemm) {
+      st = launch_gather_rows(h, x, r.row_token, r.expert_off, d->n_experts, pl.p_max, d->hidden, 2, fa.xp, s);
+      if (st != FMMOE_OK) return st;
+    }
     st = launch_ffn_tc(h, fa, s);
   } else {
     st = launch_ffn_f32(h, fa, s);

@@ -8,6 +8,10 @@
 // Both run in one persistent, warp-specialised kernel template:
 //   warp 0    : tile scheduler + TMA producer (A tile 128x64 + two B boxes 128x64 per stage,
 //               128B swizzle, L2 eviction hints)
+//   warps 6-9 : GEMM-1 at large batch only: gather the rows of a routed M-tile straight from x by
+//               token with cp.async into the same swizzled layout, so that no expert-ordered copy
+//               of x is written and read back (at small batch that copy plus plain TMA boxes is
+//               faster: the kernel is then launched without these warps)
 //   warp 1    : UMMA issuer   (one thread; 128x256x16 tcgen05.mma, accumulators in TMEM)
 //   warps 2-5 : epilogue      (tcgen05.ld -> registers -> shared-memory transpose -> coalesced
 //               global stores / reductions), overlapped with the next tile's main loop
@@ -40,7 +44,9 @@ constexpr int G_SCHED = 4;         // slots of the tile-id ring
 constexpr int G_A_BYTES = G_BM * G_BK * 2;          // 16 KB
 constexpr int G_B_BYTES = 2 * 128 * G_BK * 2;       // 32 KB (two 128-row boxes)
 constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;
-constexpr int G_THREADS = 192;
+constexpr int G_THREADS = 192;          // scheduler/producer warp, issuer warp, four epilogue warps
+constexpr int G_LOADERS = 128;          // GEMM-1 only: four more warps that gather the routed rows of x
+constexpr int G_THREADS_G1 = G_THREADS + G_LOADERS;
 constexpr int G_TMEM_COLS = 512;
 constexpr int G_EPI_LD = 33;                                 // padded row of the epilogue transpose buffer
 constexpr int G_EPI_BYTES = 4 * 32 * G_EPI_LD * 4;           // one 32x32 fp32 block per epilogue warp
@@ -67,11 +73,13 @@ struct GemmParams {
   Segment seg[2];
   // epilogue
   __nv_bfloat16* act[2];      // MODE 0: activation outputs (routed, shared)
-  const int32_t* row_token;   // MODE 1
+  const __nv_bfloat16* x; int ld_x;   // MODE 0: hidden states [T, H] the routed rows are gathered from
+  const int32_t* row_token;   // grouped row -> token (MODE 0: gather, MODE 1: combine)
   const float* row_gate;      // MODE 1
   float* acc;                 // MODE 1 atomic:  [T, H]
   float* y[2];                // MODE 1 deterministic: routed [P, H], shared [N_s*T, H]
   int deterministic;
+  int gather;                 // MODE 0: routed rows come from x through the loader warps (else from the tmA_r map)
   int* status;
 };
 
@@ -117,7 +125,7 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, int tile, i
 
 // MODE 0: GEMM-1 + SwiGLU.  MODE 1: GEMM-2 + combine.
 template <int MODE>
-__global__ void __launch_bounds__(G_THREADS, 1)
+__global__ void __launch_bounds__(MODE == 0 ? G_THREADS_G1 : G_THREADS, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__ CUtensorMap tmA_s,
               const __grid_constant__ CUtensorMap tmB0_r, const __grid_constant__ CUtensorMap tmB1_r,
               const __grid_constant__ CUtensorMap tmB0_s, const __grid_constant__ CUtensorMap tmB1_s,
@@ -141,9 +149,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   pdl_launch_dependents();
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < G_STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
+    // GEMM-1: a stage is full when the producer's TMA bytes have landed AND every loader thread's copies have
+    for (int i = 0; i < G_STAGES; ++i) { mbar_init(&full_bar[i], (MODE == 0 && p.gather) ? 1 + G_LOADERS : 1); mbar_init(&empty_bar[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&tfull_bar[i], 1); mbar_init(&tempty_bar[i], 128); }
-    for (int i = 0; i < G_SCHED; ++i) { mbar_init(&sfull_bar[i], 1); mbar_init(&sempty_bar[i], 5); }   // issuer + 4 epilogue warps
+    // readers of a tile id: issuer + 4 epilogue warps (+ 4 loader warps in GEMM-1)
+    for (int i = 0; i < G_SCHED; ++i) { mbar_init(&sfull_bar[i], 1); mbar_init(&sempty_bar[i], (MODE == 0 && p.gather) ? 9 : 5); }
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -165,7 +175,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   if (warp == 0) {
     // ------------------------------------------------------------ scheduler + TMA producer
     if (lane == 0) {
-      tma_prefetch_desc(&tmA_r); tma_prefetch_desc(&tmB0_r); tma_prefetch_desc(&tmB1_r);
+      tma_prefetch_desc(&tmA_r);
+      tma_prefetch_desc(&tmB0_r); tma_prefetch_desc(&tmB1_r);
       if (p.shared_mtiles) { tma_prefetch_desc(&tmA_s); tma_prefetch_desc(&tmB0_s); tma_prefetch_desc(&tmB1_s); }
       const uint64_t pol_stream = l2_policy_evict_first();
       int stage = 0; uint32_t phase = 0;
@@ -189,14 +200,17 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         // shared experts, activation tiles) keeps the default priority: tiles that share data
         // are adjacent in the order, so plain LRU keeps it resident for as long as it is needed.
         const bool stream_b = ti.seg == 0 && ti.single;
+        // GEMM-1 reads a routed M-tile's rows straight from x through the token list (loader warps,
+        // cp.async): the TMA engine, whose row rate bounds the weight stream, carries weights only
+        const bool gather_a = MODE == 0 && p.gather && ti.seg == 0;
         const int a_row = ti.row0 + ti.group_local * sg.a_group_stride;
         const int b_y0 = ti.group_local * sg.b_rows_per_group + ti.nb * (MODE == 0 ? 128 : 256);
         const int b_y1 = MODE == 0 ? b_y0 : b_y0 + 128;
         for (int kb = 0; kb < sg.k_blocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           unsigned char* sA = smem + stage * G_STAGE_BYTES;
-          mbar_arrive_expect_tx(&full_bar[stage], G_STAGE_BYTES);
-          tma_load_2d(sA, mA, &full_bar[stage], kb * G_BK, a_row);
+          mbar_arrive_expect_tx(&full_bar[stage], gather_a ? G_B_BYTES : G_STAGE_BYTES);
+          if (!gather_a) tma_load_2d(sA, mA, &full_bar[stage], kb * G_BK, a_row);
           if (stream_b) {
             tma_load_2d_hint(sA + G_A_BYTES, mB0, &full_bar[stage], kb * G_BK, b_y0, pol_stream);
             tma_load_2d_hint(sA + G_A_BYTES + G_B_BYTES / 2, mB1, &full_bar[stage], kb * G_BK, b_y1, pol_stream);
@@ -230,6 +244,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         const uint32_t d_tmem = tmem_base + as * 256;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { ok = false; break; }
+          if (MODE == 0 && p.gather) fence_proxy_async_smem();   // rows written by the loader warps' cp.async
           tc_fence_after();
           const uint32_t sA = smem_u32(smem + stage * G_STAGE_BYTES);
           const uint64_t da = umma_desc_sw128(sA);
@@ -243,6 +258,55 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         if (!ok) break;
         umma_commit(&tfull_bar[as]);        // accumulator complete
         if (++as == 2) { as = 0; aphase ^= 1; }
+      }
+      if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+    }
+  } else if (warp >= 6) {
+    // ------------------------------------------------------------ row loaders (GEMM-1 only, warps 6..9)
+    // Every stage of a routed tile: 128 rows x 128 bytes of x, row r = token row_token[row0 + r],
+    // written where a TMA box with the 128-byte swizzle would put them (16-byte chunk c of row r at
+    // r*128 + ((c ^ (r & 7)) * 16)).  Eight lanes cover one row, a thread serves rows q, q+16, ...
+    // For other tiles the loaders only keep the stage barriers in step.
+    if (MODE == 0 && p.gather) {
+      const int lt = threadIdx.x - G_THREADS;      // 0..127
+      const int chunk = lt & 7, rq = lt >> 3;      // rq 0..15
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      const __nv_bfloat16* xg = p.x;
+      for (uint32_t it = 0; ok; ++it) {
+        const int slot = it % G_SCHED;
+        const uint32_t sph = (it / G_SCHED) & 1;
+        if (!mbar_wait(&sfull_bar[slot], sph, abort_flag)) { ok = false; break; }
+        const int tile = ring[slot];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sempty_bar[slot]);
+        if (tile < 0) break;
+        const TileInfo ti = decode_tile(p, tile, n_mt_r);
+        const Segment& sg = p.seg[ti.seg];
+        const bool gather_a = ti.seg == 0;
+        const __nv_bfloat16* src[8];
+        uint32_t dst_off[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int r = rq + 16 * i;
+          const bool valid = gather_a && r < ti.rows;
+          const long long tok = valid ? p.row_token[ti.row0 + r] : -1;
+          src[i] = valid ? xg + tok * p.ld_x + chunk * 8 : nullptr;
+          dst_off[i] = (uint32_t)(r * 128 + ((chunk ^ (r & 7)) << 4));
+        }
+        for (int kb = 0; kb < sg.k_blocks; ++kb) {
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          if (gather_a) {
+            const uint32_t sA = smem_u32(smem + stage * G_STAGE_BYTES);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              if (src[i]) cp_async_16(sA + dst_off[i], src[i] + kb * G_BK);
+            cp_async_arrive_noinc(&full_bar[stage]);
+          } else {
+            mbar_arrive(&full_bar[stage]);
+          }
+          if (++stage == G_STAGES) { stage = 0; phase ^= 1; }
+        }
       }
       if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
@@ -389,9 +453,10 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   const int mtps = (int)((a.T + G_BM - 1) / G_BM);
   const uint64_t p_rows = (uint64_t)a.p_max;
 
-  CUtensorMap A1r, A1s, G1r, U1r, G1s, U1s, A2r, A2s, D2r, D2s;
+  CUtensorMap A1s, G1r, U1r, G1s, U1s, A2r, A2s, D2r, D2s;
   bool ok = true;
-  ok &= make_map(h, &A1r, a.xp, p_rows, H, 128);
+  CUtensorMap A1r;
+  ok &= make_map(h, &A1r, a.gather_in_gemm ? a.x : a.xp, a.gather_in_gemm ? (uint64_t)a.T : p_rows, H, 128);
   ok &= make_map(h, &G1r, a.w->w_gate, (uint64_t)E * I, H, 128);
   ok &= make_map(h, &U1r, a.w->w_up, (uint64_t)E * I, H, 128);
   ok &= make_map(h, &A2r, a.act, p_rows, I, 128);
@@ -403,7 +468,7 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
     ok &= make_map(h, &A2s, a.act_sh, (uint64_t)Ns * a.T, Is, 128);
     ok &= make_map(h, &D2s, a.w->ws_down, (uint64_t)Ns * H, Is, 128);
   } else {
-    A1s = A1r; G1s = G1r; U1s = U1r; A2s = A2r; D2s = D2r;
+    A1s = G1r; G1s = G1r; U1s = U1r; A2s = A2r; D2s = D2r;   // never dereferenced without shared experts
   }
   if (!ok) return FMMOE_ERR_CUDA;
 
@@ -414,6 +479,7 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   p1.seg[1] = Segment{Ns ? (Is + 127) / 128 : 0, H / G_BK, Is, Is, 0, (int)a.T, Is};
   p1.act[0] = static_cast<__nv_bfloat16*>(a.act); p1.act[1] = static_cast<__nv_bfloat16*>(a.act_sh);
   p1.status = a.d_status;
+  p1.x = static_cast<const __nv_bfloat16*>(a.x); p1.ld_x = H; p1.row_token = a.row_token; p1.gather = a.gather_in_gemm;
   p1.tile_counter = a.tile_counters;
 
   GemmParams p2 = p1;
@@ -429,7 +495,7 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
     h->tc_attr_set = true;
   }
   const int grid = h->sm_count;
-  { ProfScope ps(h, FMMOE_KERNEL_GEMM1, s); FMMOE_CUDA_TRY(launch_pdl(ffn_tc_kernel<0>, dim3(grid), dim3(G_THREADS), G_SMEM_BYTES, s, 1, A1r, A1s, G1r, U1r, G1s, U1s, p1)); }
+  { ProfScope ps(h, FMMOE_KERNEL_GEMM1, s); FMMOE_CUDA_TRY(launch_pdl(ffn_tc_kernel<0>, dim3(grid), dim3(a.gather_in_gemm ? G_THREADS_G1 : G_THREADS), G_SMEM_BYTES, s, 1, A1r, A1s, G1r, U1r, G1s, U1s, p1)); }
   FMMOE_CUDA_TRY(cudaGetLastError());
   { ProfScope ps(h, FMMOE_KERNEL_GEMM2, s); FMMOE_CUDA_TRY(launch_pdl(ffn_tc_kernel<1>, dim3(grid), dim3(G_THREADS), G_SMEM_BYTES, s, 1, A2r, A2s, D2r, D2r, D2s, D2s, p2)); }
   FMMOE_CUDA_TRY(cudaGetLastError());

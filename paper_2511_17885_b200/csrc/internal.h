@@ -173,8 +173,12 @@ struct FfnArgs {   // both paths
   float* acc;            // atomic mode
   float* y; float* ysh;  // deterministic mode
   int deterministic;
+  int gather_in_gemm;    // bf16: GEMM-1 gathers the routed rows of x itself (xp is not read)
   int* d_status;
 };
+// Large batches: skip the expert-ordered copy of x and let GEMM-1's loader warps gather the rows.
+// Small batches are bound by the weight stream, where the copy + plain TMA boxes are faster.
+static inline bool gather_rows_in_gemm(int64_t T) { return T >= 12288; }
 fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05
 fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);   // fp32 FMA
 
