@@ -44,10 +44,8 @@ bool plan_workspace(const fmmoe_layer_desc& d, int64_t T, uint32_t flags, WsPlan
   p->max_mtiles = (int32_t)(d.n_experts + P / block_m + 1);
   size_t o = 0;
   auto take = [&](size_t bytes) { const size_t at = o; o = align_up(o + bytes, 256); return at; };
-  p->zero_off = 0;
   p->misc_off = take(8 * 4);
   p->acc_off = take(det ? 0 : Tz * H * 4);
-  p->zero_bytes = o;
   p->blk_cnt_off = take((size_t)d.n_experts * ((Tz + 31) / 32 + 4) * 4);
   p->topk_idx_off = take(P * 4);
   p->topk_w_off = take(P * 4);

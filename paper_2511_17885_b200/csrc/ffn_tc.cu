@@ -66,7 +66,6 @@ struct GemmParams {
   const MTile* mtiles;        // routed M-tiles
   const int32_t* n_mtiles;    // device: number of routed M-tiles
   int32_t* tile_counter;      // device: next tile to hand out (zero at launch)
-  int n_experts;
   int shared_mtiles;          // N_s * ceil(T/128), host-known
   int mt_per_shared;          // ceil(T/128)
   long long T;
@@ -473,7 +472,7 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   if (!ok) return FMMOE_ERR_CUDA;
 
   GemmParams p1 = {};
-  p1.mtiles = a.mtiles; p1.n_mtiles = a.n_mtiles; p1.n_experts = E;
+  p1.mtiles = a.mtiles; p1.n_mtiles = a.n_mtiles;
   p1.shared_mtiles = Ns * mtps; p1.mt_per_shared = mtps; p1.T = a.T;
   p1.seg[0] = Segment{(I + 127) / 128, H / G_BK, I, I, 0, 0, I};
   p1.seg[1] = Segment{Ns ? (Is + 127) / 128 : 0, H / G_BK, Is, Is, 0, (int)a.T, Is};

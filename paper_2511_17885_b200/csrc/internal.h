@@ -50,7 +50,6 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 
 // Workspace layout of fmmoe_route / fmmoe_moe_forward (byte offsets).
 struct WsPlan {
-  size_t zero_off, zero_bytes;  // region cleared at the start of every call
   size_t blk_cnt_off;           // int32 [E][ceil(T/32)] per-block expert counts / offsets (not cleared)
   size_t misc_off;              // int32 [8]: [0] number of routed M-tiles, [1],[2] GEMM tile counters
   size_t acc_off;               // fp32 [T,H] combine accumulator (atomic mode)

@@ -39,7 +39,6 @@ struct PruneDev {
   int32_t* vis_list;   // [T] token index of the v-th vision token of sequence b at seq_off[b]+v
   double* sim;         // [windows]
   double* asum;        // [windows]
-  uint8_t* action;     // [windows] 0 keep, 1 merge, 2 drop
   // outputs
   void* x_out; uint8_t* is_visual_out; int32_t* keep_idx; uint8_t* kind;
   int32_t* keep_idx_ws; uint8_t* kind_ws;   // always-present copies in the workspace
@@ -536,7 +535,7 @@ extern "C" __attribute__((visibility("default"))) int64_t fmmoe_prune_kept_count
 }
 
 namespace {
-struct PruneWs { size_t vrank, vis_list, sim, asum, action, keep_idx, kind, total; };
+struct PruneWs { size_t vrank, vis_list, sim, asum, keep_idx, kind, total; };
 PruneWs plan_prune(int64_t T) {
   PruneWs w; size_t o = 0;
   const size_t nw = (size_t)T / 2 + 1;
@@ -544,7 +543,6 @@ PruneWs plan_prune(int64_t T) {
   w.vis_list = o; o = align_up(o + (size_t)T * 4, 256);
   w.sim = o; o = align_up(o + nw * 8, 256);
   w.asum = o; o = align_up(o + nw * 8, 256);
-  w.action = o; o = align_up(o + nw, 256);
   w.keep_idx = o; o = align_up(o + (size_t)T * 4, 256);
   w.kind = o; o = align_up(o + (size_t)T, 256);
   w.total = o;
@@ -602,7 +600,6 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
   a.dtype = dtype; a.alpha = p->alpha;
   a.vrank = reinterpret_cast<int32_t*>(ws + wp.vrank); a.vis_list = reinterpret_cast<int32_t*>(ws + wp.vis_list);
   a.sim = reinterpret_cast<double*>(ws + wp.sim); a.asum = reinterpret_cast<double*>(ws + wp.asum);
-  a.action = reinterpret_cast<uint8_t*>(ws + wp.action);
   a.keep_idx_ws = reinterpret_cast<int32_t*>(ws + wp.keep_idx); a.kind_ws = reinterpret_cast<uint8_t*>(ws + wp.kind);
   a.x_out = x_out; a.is_visual_out = is_visual_out; a.keep_idx = keep_idx; a.kind = kind;
   a.status = h->d_status;
@@ -630,7 +627,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
     PruneSeqs rel = sq;
     for (int i = 0; i <= nb; ++i) rel.win_off[i] -= win_base;
     PruneDev al = a;
-    al.sim = a.sim + win_base; al.asum = a.asum + win_base; al.action = a.action + win_base;
+    al.sim = a.sim + win_base; al.asum = a.asum + win_base;
     { ProfScope ps(h, FMMOE_KERNEL_PRUNE_INDEX, s); FMMOE_CUDA_TRY(launch_pdl(vis_index_kernel, dim3(nb), dim3(1024), 0, s, 1, al, rel)); }
     FMMOE_CUDA_TRY(cudaGetLastError());
     h->launches += 1;
