@@ -40,7 +40,8 @@ namespace fmmoe {
 constexpr int G_BM = TC_BLOCK_M;   // 128
 constexpr int G_BK = 64;           // one 128-byte swizzle atom of bf16
 constexpr int G_STAGES = 4;
-constexpr int G_SCHED = 4;         // slots of the tile-id ring
+constexpr int G_SCHED = 4;         // slots of the tile ring
+constexpr int G_SLOT_INTS = 8;     // a slot: tile id (-1: no more tiles) + the decoded TileInfo
 constexpr int G_A_BYTES = G_BM * G_BK * 2;          // 16 KB
 constexpr int G_B_BYTES = 2 * 128 * G_BK * 2;       // 32 KB (two 128-row boxes)
 constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;
@@ -50,7 +51,7 @@ constexpr int G_THREADS_G1 = G_THREADS + G_LOADERS;
 constexpr int G_TMEM_COLS = 512;
 constexpr int G_EPI_LD = 33;                                 // padded row of the epilogue transpose buffer
 constexpr int G_EPI_BYTES = 4 * 32 * G_EPI_LD * 4;           // one 32x32 fp32 block per epilogue warp
-constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_EPI_BYTES + 1024 /*align*/ + 384 /*barriers, tile ring*/;
 
 struct Segment {          // routed experts (0) or shared experts (1)
   int n_nblocks;          // N-blocks per group
@@ -122,6 +123,16 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, int tile, i
   return ti;
 }
 
+// A slot of the tile ring as the producer publishes it and the other roles read it.
+__device__ __forceinline__ void slot_store(volatile int* s, int tile, const TileInfo& ti) {
+  s[0] = tile; s[1] = ti.seg; s[2] = ti.group_local; s[3] = ti.row0; s[4] = ti.rows; s[5] = ti.nb; s[6] = ti.single;
+}
+__device__ __forceinline__ TileInfo slot_load(const volatile int* s) {
+  TileInfo ti;
+  ti.seg = s[1]; ti.group_local = s[2]; ti.row0 = s[3]; ti.rows = s[4]; ti.nb = s[5]; ti.single = s[6] != 0;
+  return ti;
+}
+
 // MODE 0: GEMM-1 + SwiGLU.  MODE 1: GEMM-2 + combine.
 template <int MODE>
 __global__ void __launch_bounds__(MODE == 0 ? G_THREADS_G1 : G_THREADS, 1)
@@ -140,8 +151,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   uint64_t* tempty_bar = tfull_bar + 2;        // [2]
   uint64_t* sfull_bar = tempty_bar + 2;        // [G_SCHED]
   uint64_t* sempty_bar = sfull_bar + G_SCHED;  // [G_SCHED]
-  volatile int* ring = reinterpret_cast<volatile int*>(sempty_bar + G_SCHED);   // [G_SCHED]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(ring) + G_SCHED);
+  volatile int* ring = reinterpret_cast<volatile int*>(sempty_bar + G_SCHED);   // [G_SCHED][G_SLOT_INTS]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(ring) + G_SCHED * G_SLOT_INTS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -180,16 +191,21 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
       const uint64_t pol_stream = l2_policy_evict_first();
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (uint32_t it = 0; ok; ++it) {
-        const int slot = it % G_SCHED;
-        const uint32_t sph = (it / G_SCHED) & 1;
-        if (!mbar_wait(&sempty_bar[slot], sph ^ 1, abort_flag)) { ok = false; break; }
-        int tile = atomicAdd(p.tile_counter, 1);
-        if (tile >= total_tiles) tile = -1;
-        ring[slot] = tile;
+      // Publishes the tile claimed as `raw` under sequence number `seq` (decoded, so that no other
+      // role touches global memory to learn what it is).  1: a tile, 0: no tiles left, -1: timeout.
+      auto publish = [&](uint32_t seq, int raw, TileInfo& ti) -> int {
+        const int slot = seq % G_SCHED;
+        const uint32_t sph = (seq / G_SCHED) & 1;
+        if (!mbar_wait(&sempty_bar[slot], sph ^ 1, abort_flag)) return -1;
+        const int tile = raw < total_tiles ? raw : -1;
+        if (tile >= 0) ti = decode_tile(p, tile, n_mt_r);
+        slot_store(ring + slot * G_SLOT_INTS, tile, ti);
         mbar_arrive(&sfull_bar[slot]);
-        if (tile < 0) break;
-        const TileInfo ti = decode_tile(p, tile, n_mt_r);
+        return tile >= 0;
+      };
+      TileInfo ti = {}, ti_next = {};
+      int have = publish(0, atomicAdd(p.tile_counter, 1), ti);
+      for (uint32_t it = 0; have == 1; ++it) {
         const Segment& sg = p.seg[ti.seg];
         const CUtensorMap* mA = ti.seg ? &tmA_s : &tmA_r;
         const CUtensorMap* mB0 = ti.seg ? &tmB0_s : &tmB0_r;
@@ -205,7 +221,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         const int a_row = ti.row0 + ti.group_local * sg.a_group_stride;
         const int b_y0 = ti.group_local * sg.b_rows_per_group + ti.nb * (MODE == 0 ? 128 : 256);
         const int b_y1 = MODE == 0 ? b_y0 : b_y0 + 128;
+        // The next tile is claimed half-way through this one and decoded while the last stages of
+        // this one are still in flight, so the ring never drains between tiles.
+        const int kb_claim = sg.k_blocks >> 1, kb_publish = sg.k_blocks - 1;
+        int raw_next = 0, have_next = 0;
         for (int kb = 0; kb < sg.k_blocks; ++kb) {
+          if (kb == kb_claim) raw_next = atomicAdd(p.tile_counter, 1);
+          if (kb == kb_publish) {
+            have_next = publish(it + 1, raw_next, ti_next);
+            if (have_next < 0) { ok = false; break; }
+          }
           if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           unsigned char* sA = smem + stage * G_STAGE_BYTES;
           mbar_arrive_expect_tx(&full_bar[stage], gather_a ? G_B_BYTES : G_STAGE_BYTES);
@@ -219,8 +244,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
           }
           if (++stage == G_STAGES) { stage = 0; phase ^= 1; }
         }
+        if (!ok) break;
+        ti = ti_next; have = have_next;
       }
-      if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+      if (!ok || have < 0) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ UMMA issuer
@@ -233,11 +260,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         const int slot = it % G_SCHED;
         const uint32_t sph = (it / G_SCHED) & 1;
         if (!mbar_wait(&sfull_bar[slot], sph, abort_flag)) { ok = false; break; }
-        const int tile = ring[slot];
+        const int tile = ring[slot * G_SLOT_INTS];
+        const int seg = ring[slot * G_SLOT_INTS + 1];
         mbar_arrive(&sempty_bar[slot]);
         if (tile < 0) break;
-        const TileInfo ti = decode_tile(p, tile, n_mt_r);
-        const int k_blocks = p.seg[ti.seg].k_blocks;
+        const int k_blocks = p.seg[seg].k_blocks;
         if (!mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + as * 256;
@@ -276,11 +303,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         const int slot = it % G_SCHED;
         const uint32_t sph = (it / G_SCHED) & 1;
         if (!mbar_wait(&sfull_bar[slot], sph, abort_flag)) { ok = false; break; }
-        const int tile = ring[slot];
+        const int tile = ring[slot * G_SLOT_INTS];
+        const TileInfo ti = slot_load(ring + slot * G_SLOT_INTS);
         __syncwarp();
         if (lane == 0) mbar_arrive(&sempty_bar[slot]);
         if (tile < 0) break;
-        const TileInfo ti = decode_tile(p, tile, n_mt_r);
         const Segment& sg = p.seg[ti.seg];
         const bool gather_a = ti.seg == 0;
         const __nv_bfloat16* src[8];
@@ -320,11 +347,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
       const int slot = it % G_SCHED;
       const uint32_t sph = (it / G_SCHED) & 1;
       if (!mbar_wait(&sfull_bar[slot], sph, abort_flag)) { ok = false; break; }
-      const int tile = ring[slot];
+      const int tile = ring[slot * G_SLOT_INTS];
+      const TileInfo ti = slot_load(ring + slot * G_SLOT_INTS);
       __syncwarp();
       if (lane == 0) mbar_arrive(&sempty_bar[slot]);
       if (tile < 0) break;
-      const TileInfo ti = decode_tile(p, tile, n_mt_r);
       const Segment& sg = p.seg[ti.seg];
       if (!mbar_wait(&tfull_bar[as], aphase, abort_flag)) { ok = false; break; }
       tc_fence_after();
