@@ -371,8 +371,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-            const float a0 = g0 / (1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
-            const float a1 = g1 / (1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
+            const float a0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
+            const float a1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
             const __nv_bfloat162 h = __floats2bfloat162_rn(a0, a1);
             stg32[lane * 17 + i] = *reinterpret_cast<const uint32_t*>(&h);
           }
