@@ -153,6 +153,33 @@ fmmoe_status fmmoe_moe_forward_host(fmmoe_handle *handle, const fmmoe_layer_desc
                                     uint8_t *is_visual_dev, void *workspace, size_t workspace_bytes,
                                     void *cuda_stream);
 
+/* Pipelined host I/O.  The paper has no counterpart: these calls only overlap the PCIe copies of
+ * consecutive, independent batches with the layer itself, for callers whose activations live in
+ * host memory.  Each handle owns one upload and one download stream (created by the first of these
+ * calls on the handle).
+ *
+ * fmmoe_moe_forward_host_async: as fmmoe_moe_forward_host, but returns as soon as everything is
+ * enqueued: the uploads of x_host / is_visual_host run on the upload stream, the layer on
+ * cuda_stream after them, the copy to out_host (skipped if out_host is NULL) on the download
+ * stream after the layer.  Host buffers should be pinned.  A batch in flight owns its workspace,
+ * out_dev, is_visual_dev and host buffers until a ticket taken after it has been waited for: give
+ * every batch in flight its own set (two sets alternate for a depth of two).
+ * fmmoe_download_async: copies bytes from src_dev to dst_host on the download stream, after the
+ * work enqueued on cuda_stream so far (e.g. the rows fmmoe_prune_visual has just produced).
+ * fmmoe_host_fence: returns a ticket for everything enqueued on the download stream so far.
+ * fmmoe_host_wait: blocks the calling thread until the downloads covered by the ticket are in
+ * host memory (at most 64 tickets may be outstanding).
+ * Errors: FMMOE_ERR_INVALID_ARG (NULL or unknown ticket), FMMOE_ERR_WORKSPACE, FMMOE_ERR_CUDA. */
+fmmoe_status fmmoe_moe_forward_host_async(fmmoe_handle *handle, const fmmoe_layer_desc *desc, const fmmoe_weights *w,
+                                          const void *x_host, const uint8_t *is_visual_host, int64_t n_tokens,
+                                          uint32_t flags, void *out_host, const fmmoe_route_out *route,
+                                          void *out_dev, uint8_t *is_visual_dev, void *workspace,
+                                          size_t workspace_bytes, void *cuda_stream);
+fmmoe_status fmmoe_download_async(fmmoe_handle *handle, void *dst_host, const void *src_dev, size_t bytes,
+                                  void *cuda_stream);
+fmmoe_status fmmoe_host_fence(fmmoe_handle *handle, uint64_t *ticket);
+fmmoe_status fmmoe_host_wait(fmmoe_handle *handle, uint64_t ticket);
+
 /* Optional per-kernel timeline.  While enabled, every kernel the handle launches is
  * bracketed by CUDA events on the launching stream (host-side event objects only; no
  * device memory).  fmmoe_profile_read synchronises the device and returns the summed

@@ -83,6 +83,11 @@ def lib() -> C.CDLL:
     L.fmmoe_moe_forward_host.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), vp, vp, i64, u32, vp,
                                          C.POINTER(RouteOut), vp, vp, vp, sz, vp]
     L.fmmoe_moe_forward_host.restype = C.c_int
+    L.fmmoe_moe_forward_host_async.argtypes = L.fmmoe_moe_forward_host.argtypes
+    L.fmmoe_moe_forward_host_async.restype = C.c_int
+    L.fmmoe_download_async.argtypes = [vp, vp, vp, sz, vp]; L.fmmoe_download_async.restype = C.c_int
+    L.fmmoe_host_fence.argtypes = [vp, C.POINTER(C.c_uint64)]; L.fmmoe_host_fence.restype = C.c_int
+    L.fmmoe_host_wait.argtypes = [vp, C.c_uint64]; L.fmmoe_host_wait.restype = C.c_int
     L.fmmoe_profile_enable.argtypes = [vp, C.c_int]; L.fmmoe_profile_enable.restype = C.c_int
     L.fmmoe_profile_reset.argtypes = [vp]; L.fmmoe_profile_reset.restype = C.c_int
     L.fmmoe_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_double), C.POINTER(i64)]
@@ -190,6 +195,7 @@ class Handle:
         self.device = device
         _check(lib().fmmoe_create(C.byref(self._h), device), "fmmoe_create")
         self._ws: Optional[torch.Tensor] = None
+        self._ws_slots: Dict[int, torch.Tensor] = {}   # one workspace per batch in flight (pipelined host I/O)
 
     def close(self):
         if self._h:
@@ -286,6 +292,46 @@ class Handle:
                                             _ptr(out_dev), _ptr(is_visual_dev), wsp, wsn, _stream()),
                "fmmoe_moe_forward_host")
         return out_host
+
+    def fmmoe_moe_forward_host_async(self, desc: LayerDesc, w: Weights, x_host: torch.Tensor,
+                                     is_visual_host: torch.Tensor, flags: int, out_host: Optional[torch.Tensor],
+                                     slot: int, route: Optional[Dict[str, torch.Tensor]] = None,
+                                     out_dev: Optional[torch.Tensor] = None,
+                                     is_visual_dev: Optional[torch.Tensor] = None):
+        """Pipelined host-buffer variant: returns once the upload, the layer and the download are enqueued.
+        `slot` selects the workspace of this batch in flight (its staging area is being written by the upload
+        stream while other batches compute); take a ticket with fmmoe_host_fence and wait for it before the
+        slot and its buffers are reused."""
+        T = x_host.shape[0]
+        ro = RouteOut(**{k: v.data_ptr() for k, v in route.items()}) if route else None
+        assert not x_host.is_cuda and x_host.is_contiguous() and (out_host is None or not out_host.is_cuda)
+        need = fmmoe_workspace_bytes(desc, T, flags) + int(lib().fmmoe_host_staging_bytes(C.byref(desc), T))
+        ws = self._ws_slots.get(slot)
+        if ws is None or ws.numel() < need + 256:
+            ws = self._ws_slots[slot] = torch.empty(need + 256, dtype=torch.uint8, device=f"cuda:{self.device}")
+        base = ws.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        _check(lib().fmmoe_moe_forward_host_async(
+            self._h, C.byref(desc), C.byref(w), C.c_void_p(x_host.data_ptr()), C.c_void_p(is_visual_host.data_ptr()),
+            T, flags, C.c_void_p(out_host.data_ptr()) if out_host is not None else None,
+            C.byref(ro) if ro is not None else None, _ptr(out_dev), _ptr(is_visual_dev), C.c_void_p(aligned),
+            C.c_size_t(ws.numel() - (aligned - base)), _stream()), "fmmoe_moe_forward_host_async")
+
+    def fmmoe_download_async(self, dst_host: torch.Tensor, src_dev: torch.Tensor):
+        """Device -> host copy on the handle's download stream, after the work enqueued on the current stream."""
+        assert not dst_host.is_cuda and src_dev.is_cuda and dst_host.is_contiguous() and src_dev.is_contiguous()
+        n = src_dev.numel() * src_dev.element_size()
+        assert dst_host.numel() * dst_host.element_size() >= n
+        _check(lib().fmmoe_download_async(self._h, C.c_void_p(dst_host.data_ptr()), _ptr(src_dev), n, _stream()),
+               "fmmoe_download_async")
+
+    def fmmoe_host_fence(self) -> int:
+        t = C.c_uint64(0)
+        _check(lib().fmmoe_host_fence(self._h, C.byref(t)), "fmmoe_host_fence")
+        return int(t.value)
+
+    def fmmoe_host_wait(self, ticket: int):
+        _check(lib().fmmoe_host_wait(self._h, C.c_uint64(ticket)), "fmmoe_host_wait")
 
     # ---- Section 3.2
     def fmmoe_prune_visual(self, p: PruneParams, probs: torch.Tensor, attn: Optional[torch.Tensor], x: torch.Tensor,

@@ -161,6 +161,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
   h->launches = 0;
   h->d_status = nullptr; h->h_status = nullptr; h->encode_tiled = nullptr;
   h->tc_attr_set = false; h->profiling = false; h->ev_used = 0;
+  h->pipe_ready = false; h->pipe_next = 0; h->ticket_next = 0;
   { const char* dbg = getenv("FMMOE_DEBUG_SYNC"); h->debug_sync = dbg && dbg[0] == '1'; h->debug_seq = 0; }
   if (cudaMalloc(&h->d_status, 256) != cudaSuccess || cudaMemset(h->d_status, 0, 256) != cudaSuccess ||
       cudaMallocHost(&h->h_status, 256) != cudaSuccess) {
@@ -183,6 +184,12 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_destroy(fmm
   if (h->d_status) cudaFree(h->d_status);
   if (h->h_status) cudaFreeHost(h->h_status);
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+  if (h->pipe_ready) {
+    cudaStreamSynchronize(h->up_stream); cudaStreamSynchronize(h->down_stream);
+    for (cudaEvent_t e : h->pipe_ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->ticket_ev) cudaEventDestroy(e);
+    cudaStreamDestroy(h->up_stream); cudaStreamDestroy(h->down_stream);
+  }
   delete h;
   return FMMOE_OK;
 }
@@ -300,6 +307,86 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward
   if (st != FMMOE_OK) return st;
   FMMOE_CUDA_TRY(cudaMemcpyAsync(out_host, dout, xb, cudaMemcpyDeviceToHost, s));
   FMMOE_CUDA_TRY(cudaStreamSynchronize(s));
+  return FMMOE_OK;
+}
+
+// ---------------------------------------------------------------- pipelined host I/O
+// Copies run on two streams of the handle, one per direction, ordered against the caller's compute
+// stream by events, so that the upload of one batch, the layer of the previous one and the download
+// of the one before overlap.  Nothing here waits on the host except fmmoe_host_wait.
+static fmmoe_status pipe_init(fmmoe_handle* h) {
+  if (h->pipe_ready) return FMMOE_OK;
+  FMMOE_CUDA_TRY(cudaSetDevice(h->device));
+  FMMOE_CUDA_TRY(cudaStreamCreateWithFlags(&h->up_stream, cudaStreamNonBlocking));
+  FMMOE_CUDA_TRY(cudaStreamCreateWithFlags(&h->down_stream, cudaStreamNonBlocking));
+  for (cudaEvent_t& e : h->pipe_ev) FMMOE_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  for (cudaEvent_t& e : h->ticket_ev) FMMOE_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  h->pipe_ready = true;
+  return FMMOE_OK;
+}
+static cudaEvent_t pipe_event(fmmoe_handle* h) { return h->pipe_ev[h->pipe_next++ % fmmoe_handle::kPipeEvents]; }
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward_host_async(
+    fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w, const void* x_host, const uint8_t* is_visual_host,
+    int64_t T, uint32_t flags, void* out_host, const fmmoe_route_out* route, void* out_dev, uint8_t* is_visual_dev,
+    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!h || !desc_ok(d) || T < 0) return FMMOE_ERR_INVALID_ARG;
+  if (T > 0 && (!x_host || !is_visual_host)) return FMMOE_ERR_INVALID_ARG;
+  const size_t elem = d->dtype == FMMOE_BF16 ? 2 : 4;
+  const size_t xb = (size_t)T * d->hidden * elem;
+  const size_t stage = fmmoe_host_staging_bytes(d, T);
+  const size_t inner = fmmoe_workspace_bytes(d, T, flags);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < stage + inner) return FMMOE_ERR_WORKSPACE;
+  if (T == 0) return FMMOE_OK;
+  fmmoe_status st = pipe_init(h);
+  if (st != FMMOE_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  char* dx = ws;
+  char* dout = out_dev ? static_cast<char*>(out_dev) : ws + align_up(xb, 256);
+  uint8_t* dvis = is_visual_dev ? is_visual_dev : reinterpret_cast<uint8_t*>(ws + 2 * align_up(xb, 256));
+  const cudaEvent_t uploaded = pipe_event(h);
+  FMMOE_CUDA_TRY(cudaMemcpyAsync(dx, x_host, xb, cudaMemcpyHostToDevice, h->up_stream));
+  FMMOE_CUDA_TRY(cudaMemcpyAsync(dvis, is_visual_host, (size_t)T, cudaMemcpyHostToDevice, h->up_stream));
+  FMMOE_CUDA_TRY(cudaEventRecord(uploaded, h->up_stream));
+  FMMOE_CUDA_TRY(cudaStreamWaitEvent(s, uploaded, 0));
+  st = fmmoe_moe_forward(h, d, w, dx, dvis, T, flags, dout, route, ws + stage, workspace_bytes - stage, s);
+  if (st != FMMOE_OK) return st;
+  if (out_host) {
+    const cudaEvent_t computed = pipe_event(h);
+    FMMOE_CUDA_TRY(cudaEventRecord(computed, s));
+    FMMOE_CUDA_TRY(cudaStreamWaitEvent(h->down_stream, computed, 0));
+    FMMOE_CUDA_TRY(cudaMemcpyAsync(out_host, dout, xb, cudaMemcpyDeviceToHost, h->down_stream));
+  }
+  return FMMOE_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_download_async(fmmoe_handle* h, void* dst_host, const void* src_dev,
+                                                                                     size_t bytes, void* cuda_stream) {
+  if (!h || (bytes && (!dst_host || !src_dev))) return FMMOE_ERR_INVALID_ARG;
+  if (bytes == 0) return FMMOE_OK;
+  const fmmoe_status st = pipe_init(h);
+  if (st != FMMOE_OK) return st;
+  const cudaEvent_t produced = pipe_event(h);
+  FMMOE_CUDA_TRY(cudaEventRecord(produced, static_cast<cudaStream_t>(cuda_stream)));
+  FMMOE_CUDA_TRY(cudaStreamWaitEvent(h->down_stream, produced, 0));
+  FMMOE_CUDA_TRY(cudaMemcpyAsync(dst_host, src_dev, bytes, cudaMemcpyDeviceToHost, h->down_stream));
+  return FMMOE_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_host_fence(fmmoe_handle* h, uint64_t* ticket) {
+  if (!h || !ticket) return FMMOE_ERR_INVALID_ARG;
+  const fmmoe_status st = pipe_init(h);
+  if (st != FMMOE_OK) return st;
+  FMMOE_CUDA_TRY(cudaEventRecord(h->ticket_ev[h->ticket_next % fmmoe_handle::kTickets], h->down_stream));
+  *ticket = h->ticket_next++;
+  return FMMOE_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_host_wait(fmmoe_handle* h, uint64_t ticket) {
+  if (!h || !h->pipe_ready || ticket >= h->ticket_next) return FMMOE_ERR_INVALID_ARG;
+  // a slot that a later fence has reused completes after the ticket asked for: waiting on it is safe
+  FMMOE_CUDA_TRY(cudaEventSynchronize(h->ticket_ev[ticket % fmmoe_handle::kTickets]));
   return FMMOE_OK;
 }
 

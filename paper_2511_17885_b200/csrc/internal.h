@@ -28,6 +28,15 @@ struct fmmoe_handle {
   size_t ev_used;
   struct ProfRec { int id; size_t start, stop; };
   std::vector<ProfRec> prof;
+  // pipelined host I/O (created on first use): one stream per copy direction, a ring of events that
+  // order them against the caller's compute stream, and a ring of events behind the host tickets
+  static constexpr int kPipeEvents = 32, kTickets = 64;
+  bool pipe_ready;
+  cudaStream_t up_stream, down_stream;
+  cudaEvent_t pipe_ev[kPipeEvents];
+  uint64_t pipe_next;
+  cudaEvent_t ticket_ev[kTickets];
+  uint64_t ticket_next;
 };
 
 namespace fmmoe {

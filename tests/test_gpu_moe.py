@@ -147,3 +147,52 @@ def test_forward_host_variant_and_empty():
     out = handle().fmmoe_moe_forward(desc, ws, torch.zeros(0, H, dtype=torch.bfloat16, device="cuda"),
                                      torch.zeros(0, dtype=torch.uint8, device="cuda"), 1)
     assert out.shape == (0, H)
+
+
+def test_pipelined_host_batches_match_the_device_path():
+    """Five different batches through the pipelined host-buffer calls, two in flight: each batch's layer
+    output and pruned rows (downloaded on the library's copy stream) equal the device-resident path's."""
+    r = np.random.default_rng(11)
+    T, H, E, I_, K, Kv = 300, 128, 8, 128, 2, 1
+    w = random_layer(r, "bf16", H, E, I_, 0, 0)
+    wd = upload_weights(w, "bf16"); ws = B.make_weights(wd)
+    desc = B.make_desc(H, E, I_, 0, 0, K, Kv, torch.bfloat16)
+    hd = handle()
+    seq_off, n_vis = [0, T], [200]
+    pp = B.prune_params(5, 0.05)
+    n_ret = [100]
+    route = {"probs": torch.empty(T, E, dtype=torch.float32, device="cuda")}
+    xs = [torch.from_numpy(I.round_to_storage(r.standard_normal((T, H)), "bf16")).to(torch.bfloat16).pin_memory()
+          for _ in range(5)]
+    mask_np = np.zeros(T, np.uint8); mask_np[:200] = 1
+    mask_h = torch.from_numpy(mask_np).pin_memory()
+    slots = [{"out_dev": torch.empty(T, H, dtype=torch.bfloat16, device="cuda"),
+              "mask_dev": torch.empty(T, dtype=torch.uint8, device="cuda"), "ticket": None} for _ in range(2)]
+    got = []
+    for i, xh in enumerate(xs):
+        sl = slots[i % 2]
+        if sl["ticket"] is not None:
+            hd.fmmoe_host_wait(sl["ticket"])
+        out_h = torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
+        hd.fmmoe_moe_forward_host_async(desc, ws, xh, mask_h, B.FLAG_REDUCE_ON, out_h, slot=i % 2, route=route,
+                                        out_dev=sl["out_dev"], is_visual_dev=sl["mask_dev"])
+        pr = hd.fmmoe_prune_visual(pp, route["probs"], None, sl["out_dev"], sl["mask_dev"], seq_off, n_vis, n_ret,
+                                   want_aux=False)
+        pr_h = torch.empty(pr["x_out"].shape, dtype=torch.bfloat16).pin_memory()
+        hd.fmmoe_download_async(pr_h, pr["x_out"])
+        sl["keep"] = pr["x_out"]
+        sl["ticket"] = hd.fmmoe_host_fence()
+        got.append((out_h, pr_h, sl["ticket"]))
+    for out_h, pr_h, t in got:
+        hd.fmmoe_host_wait(t)
+    hd.check_status()
+    mask_d = dev(mask_np)
+    for xh, (out_h, pr_h, _) in zip(xs, got):
+        ref = hd.fmmoe_moe_forward(desc, ws, xh.cuda(), mask_d, B.FLAG_REDUCE_ON, route=route)
+        pr = hd.fmmoe_prune_visual(pp, route["probs"], None, ref, mask_d, seq_off, n_vis, n_ret, want_aux=False)
+        # the combine adds in a different order from call to call (atomics): compare within the bf16 tolerance
+        assert row_rel_err(out_h.float().numpy(), ref.float().cpu().numpy()) < 2e-2
+        assert pr_h.shape == pr["x_out"].shape
+        assert row_rel_err(pr_h.float().numpy(), pr["x_out"].float().cpu().numpy()) < 2e-2
+    with pytest.raises(B.FmmoeError):
+        hd.fmmoe_host_wait(1 << 40)
