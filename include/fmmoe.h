@@ -242,6 +242,23 @@ fmmoe_status fmmoe_prune_visual(fmmoe_handle *handle, const fmmoe_prune_params *
                                 int64_t *out_seq_off /* host [n_seq+1] */,
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Section 3.1 followed by Section 3.2 in one call: the layer (as fmmoe_moe_forward) and one pruning
+ * stage (as fmmoe_prune_visual) applied to the layer's output `out`, with identical results.  What the
+ * single call adds: the scoring and selection half of the pruning stage (Eq. 6-15) reads only the
+ * routing probabilities and the mask, so it is enqueued on a stream of the handle as soon as the router
+ * has run and executes beside the expert GEMMs; the row gather / merge (Eq. 16-18) follows the layer on
+ * cuda_stream, which is also where everything is ordered again before the call's last kernel.
+ * route must be non-NULL with route->probs set ([T, E] fp32); seq_off[n_seq] must equal n_tokens.
+ * workspace: fmmoe_workspace_bytes() + fmmoe_prune_workspace_bytes() bytes, 256-byte aligned.
+ * All other arguments, outputs and errors as in the two calls it replaces. */
+fmmoe_status fmmoe_moe_forward_prune(fmmoe_handle *handle, const fmmoe_layer_desc *desc, const fmmoe_weights *w,
+                                     const void *x, const uint8_t *is_visual, int64_t n_tokens, uint32_t flags,
+                                     void *out, const fmmoe_route_out *route, const fmmoe_prune_params *p,
+                                     const float *attn, const int64_t *seq_off, const int64_t *n_vis,
+                                     const int64_t *n_retain, int32_t n_seq, void *x_out, uint8_t *is_visual_out,
+                                     int32_t *keep_idx, uint8_t *kind, int64_t *out_seq_off, void *workspace,
+                                     size_t workspace_bytes, void *cuda_stream);
+
 /* Section 3.2.1, Eq. 7: cross-modal attention importance.  For every sequence, the attention
  * weights of its LAST token (the last text token of [T_v, T_t]) to all tokens of the sequence,
  * averaged over the attention heads:

@@ -83,6 +83,10 @@ def lib() -> C.CDLL:
     L.fmmoe_moe_forward_host.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), vp, vp, i64, u32, vp,
                                          C.POINTER(RouteOut), vp, vp, vp, sz, vp]
     L.fmmoe_moe_forward_host.restype = C.c_int
+    L.fmmoe_moe_forward_prune.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), vp, vp, i64, u32, vp,
+                                          C.POINTER(RouteOut), C.POINTER(PruneParams), vp, C.POINTER(i64),
+                                          C.POINTER(i64), C.POINTER(i64), i32, vp, vp, vp, vp, C.POINTER(i64), vp, sz, vp]
+    L.fmmoe_moe_forward_prune.restype = C.c_int
     L.fmmoe_moe_forward_host_async.argtypes = L.fmmoe_moe_forward_host.argtypes
     L.fmmoe_moe_forward_host_async.restype = C.c_int
     L.fmmoe_download_async.argtypes = [vp, vp, vp, sz, vp]; L.fmmoe_download_async.restype = C.c_int
@@ -361,6 +365,39 @@ class Handle:
                                         _ptr(attn), _ptr(x), _dtype_code(x.dtype), H, _ptr(is_visual), so, nv, nr, B,
                                         _ptr(x_out), _ptr(vis_out), _ptr(keep_idx), _ptr(kind), oo, wsp, wsn,
                                         _stream()), "fmmoe_prune_visual")
+        return {"x_out": x_out, "is_visual_out": vis_out, "keep_idx": keep_idx, "kind": kind,
+                "out_seq_off": [int(v) for v in oo]}
+
+    def fmmoe_moe_forward_prune(self, desc: LayerDesc, w: Weights, x: torch.Tensor, is_visual: torch.Tensor,
+                                flags: int, out: torch.Tensor, route: Dict[str, torch.Tensor], p: PruneParams,
+                                attn: Optional[torch.Tensor], seq_off, n_vis, n_retain, want_aux: bool = True):
+        """Eq. 1-5 then Eq. 6-18 in one call (selection beside the expert GEMMs).  `route` must hold "probs".
+        Returns the dict fmmoe_prune_visual returns."""
+        T, H = x.shape
+        B = len(n_vis)
+        arr = C.c_int64 * (B + 1)
+        so = arr(*[int(v) for v in seq_off])
+        nv = (C.c_int64 * max(B, 1))(*[int(v) for v in n_vis])
+        nr = (C.c_int64 * max(B, 1))(*[int(v) for v in n_retain])
+        oo = arr()
+        t_out = 0
+        for b in range(B):
+            kept, _, _ = fmmoe_prune_kept_count(int(n_vis[b]), int(n_retain[b]), p)
+            if kept < 0:
+                raise FmmoeError(1, "fmmoe_prune_kept_count")
+            t_out += int(seq_off[b + 1]) - int(seq_off[b]) - int(n_vis[b]) + kept
+        dev = x.device
+        x_out = torch.empty((t_out, H), dtype=x.dtype, device=dev)
+        vis_out = torch.empty(t_out, dtype=torch.uint8, device=dev) if want_aux else None
+        keep_idx = torch.empty(t_out, dtype=torch.int32, device=dev) if want_aux else None
+        kind = torch.empty(t_out, dtype=torch.uint8, device=dev) if want_aux else None
+        ro = RouteOut(**{k: v.data_ptr() for k, v in route.items()})
+        need = fmmoe_workspace_bytes(desc, T, flags) + 256 + int(lib().fmmoe_prune_workspace_bytes(T, B))
+        wsp, wsn = self._ws_args(need)
+        _check(lib().fmmoe_moe_forward_prune(self._h, C.byref(desc), C.byref(w), _ptr(x), _ptr(is_visual), T, flags,
+                                             _ptr(out), C.byref(ro), C.byref(p), _ptr(attn), so, nv, nr, B, _ptr(x_out),
+                                             _ptr(vis_out), _ptr(keep_idx), _ptr(kind), oo, wsp, wsn, _stream()),
+               "fmmoe_moe_forward_prune")
         return {"x_out": x_out, "is_visual_out": vis_out, "keep_idx": keep_idx, "kind": kind,
                 "out_seq_off": [int(v) for v in oo]}
 

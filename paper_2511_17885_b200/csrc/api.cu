@@ -161,7 +161,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
   h->launches = 0;
   h->d_status = nullptr; h->h_status = nullptr; h->encode_tiled = nullptr;
   h->tc_attr_set = false; h->profiling = false; h->ev_used = 0;
-  h->pipe_ready = false; h->pipe_next = 0; h->ticket_next = 0;
+  h->pipe_ready = false; h->pipe_next = 0; h->ticket_next = 0; h->side_ready = false;
   { const char* dbg = getenv("FMMOE_DEBUG_SYNC"); h->debug_sync = dbg && dbg[0] == '1'; h->debug_seq = 0; }
   if (cudaMalloc(&h->d_status, 256) != cudaSuccess || cudaMemset(h->d_status, 0, 256) != cudaSuccess ||
       cudaMallocHost(&h->h_status, 256) != cudaSuccess) {
@@ -189,6 +189,11 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_destroy(fmm
     for (cudaEvent_t e : h->pipe_ev) cudaEventDestroy(e);
     for (cudaEvent_t e : h->ticket_ev) cudaEventDestroy(e);
     cudaStreamDestroy(h->up_stream); cudaStreamDestroy(h->down_stream);
+  }
+  if (h->side_ready) {
+    cudaStreamSynchronize(h->side_stream);
+    cudaEventDestroy(h->side_fork); cudaEventDestroy(h->side_join);
+    cudaStreamDestroy(h->side_stream);
   }
   delete h;
   return FMMOE_OK;
@@ -229,10 +234,13 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_route(fmmoe
   return run_route(h, *d, *w, x, is_visual, T, flags, r, need_permute, nullptr, s);
 }
 
-extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward(fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w,
-                                          const void* x, const uint8_t* is_visual, int64_t T, uint32_t flags, void* out,
-                                          const fmmoe_route_out* route, void* workspace, size_t workspace_bytes,
-                                          void* cuda_stream) {
+// The layer.  `after_route` (may be NULL) is called once the router and the permutation have been
+// enqueued: the routing record is then ordered on the stream, the expert GEMMs are not yet.
+struct AfterRoute { fmmoe_status (*fn)(void*); void* ctx; };
+static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w,
+                                 const void* x, const uint8_t* is_visual, int64_t T, uint32_t flags, void* out,
+                                 const fmmoe_route_out* route, void* workspace, size_t workspace_bytes,
+                                 void* cuda_stream, const AfterRoute* after_route) {
   fmmoe_status st = check_common(h, d, w, x, is_visual, T, true);
   if (st != FMMOE_OK) return st;
   if (T > 0 && (!out || !aligned16(out) || out == x)) return FMMOE_ERR_INVALID_ARG;
@@ -247,6 +255,10 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward
   // the router clears the scheduler words and (atomic mode) the fp32 accumulator it owns rows of
   st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, det ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s);
   if (st != FMMOE_OK) return st;
+  if (after_route) {
+    st = after_route->fn(after_route->ctx);
+    if (st != FMMOE_OK) return st;
+  }
 
   FfnArgs fa = {};
   fa.d = d; fa.w = w; fa.x = x; fa.T = T; fa.p_max = pl.p_max;
@@ -275,6 +287,74 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward
   fin.dtype = d->dtype; fin.add_residual = (flags & FMMOE_FLAG_RESIDUAL) ? 1 : 0; fin.deterministic = det;
   fin.acc = fa.acc; fin.y = fa.y; fin.ysh = fa.ysh; fin.inv_row = r.inv_row; fin.topk_w = r.topk_w;
   return launch_finalize(h, fin, s);
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward(fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w,
+                                          const void* x, const uint8_t* is_visual, int64_t T, uint32_t flags, void* out,
+                                          const fmmoe_route_out* route, void* workspace, size_t workspace_bytes,
+                                          void* cuda_stream) {
+  return forward_impl(h, d, w, x, is_visual, T, flags, out, route, workspace, workspace_bytes, cuda_stream, nullptr);
+}
+
+// ---------------------------------------------------------------- layer + pruning stage in one call
+namespace {
+struct FusedPrune {
+  fmmoe_handle* h; const fmmoe_prune_params* p; const float* probs; int32_t n_experts; const float* attn;
+  const void* x; int32_t dtype, hidden; const uint8_t* is_visual; const int64_t* seq_off; const int64_t* n_vis;
+  const int64_t* n_retain; int32_t n_seq; void* x_out; uint8_t* is_visual_out; int32_t* keep_idx; uint8_t* kind;
+  int64_t* out_seq_off; void* ws; size_t ws_bytes; cudaStream_t s;
+};
+fmmoe_status fused_run(const FusedPrune& f, int phases, cudaStream_t s_select, cudaStream_t s_rows) {
+  return prune_visual_phases(f.h, f.p, f.probs, f.n_experts, f.attn, f.x, f.dtype, f.hidden, f.is_visual, f.seq_off,
+                             f.n_vis, f.n_retain, f.n_seq, f.x_out, f.is_visual_out, f.keep_idx, f.kind, f.out_seq_off,
+                             f.ws, f.ws_bytes, phases, s_select, s_rows);
+}
+// after the router: the selection half of the pruning pass goes to the side stream
+fmmoe_status fused_after_route(void* ctx) {
+  const FusedPrune& f = *static_cast<const FusedPrune*>(ctx);
+  FMMOE_CUDA_TRY(cudaEventRecord(f.h->side_fork, f.s));
+  FMMOE_CUDA_TRY(cudaStreamWaitEvent(f.h->side_stream, f.h->side_fork, 0));
+  const fmmoe_status st = fused_run(f, 1, f.h->side_stream, f.h->side_stream);
+  if (st != FMMOE_OK) return st;
+  FMMOE_CUDA_TRY(cudaEventRecord(f.h->side_join, f.h->side_stream));
+  return FMMOE_OK;
+}
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward_prune(
+    fmmoe_handle* h, const fmmoe_layer_desc* d, const fmmoe_weights* w, const void* x, const uint8_t* is_visual,
+    int64_t T, uint32_t flags, void* out, const fmmoe_route_out* route, const fmmoe_prune_params* p, const float* attn,
+    const int64_t* seq_off, const int64_t* n_vis, const int64_t* n_retain, int32_t n_seq, void* x_out,
+    uint8_t* is_visual_out, int32_t* keep_idx, uint8_t* kind, int64_t* out_seq_off, void* workspace,
+    size_t workspace_bytes, void* cuda_stream) {
+  if (!h || !desc_ok(d) || T < 0 || !route || !route->probs || !seq_off || n_seq < 0) return FMMOE_ERR_INVALID_ARG;
+  if ((n_seq ? seq_off[n_seq] : 0) != T) return FMMOE_ERR_INVALID_ARG;
+  const size_t layer_ws = fmmoe_workspace_bytes(d, T, flags);
+  const size_t prune_ws = fmmoe_prune_workspace_bytes(T, n_seq);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < layer_ws + prune_ws) return FMMOE_ERR_WORKSPACE;
+  if (!h->side_ready) {
+    FMMOE_CUDA_TRY(cudaSetDevice(h->device));
+    FMMOE_CUDA_TRY(cudaStreamCreateWithFlags(&h->side_stream, cudaStreamNonBlocking));
+    FMMOE_CUDA_TRY(cudaEventCreateWithFlags(&h->side_fork, cudaEventDisableTiming));
+    FMMOE_CUDA_TRY(cudaEventCreateWithFlags(&h->side_join, cudaEventDisableTiming));
+    h->side_ready = true;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  FusedPrune f = {h, p, route->probs, d->n_experts, attn, out, d->dtype, d->hidden, is_visual, seq_off, n_vis, n_retain,
+                  n_seq, x_out, is_visual_out, keep_idx, kind, out_seq_off, ws + align_up(layer_ws, 256),
+                  workspace_bytes - align_up(layer_ws, 256), s};
+  if (T == 0) return fused_run(f, 3, s, s);   // nothing to enqueue: validation and the output layout only
+  // every argument check of the pruning pass happens before anything is enqueued
+  {
+    const fmmoe_status st = fused_run(f, 0, s, s);
+    if (st != FMMOE_OK) return st;
+  }
+  const AfterRoute hook = {fused_after_route, &f};
+  fmmoe_status st = forward_impl(h, d, w, x, is_visual, T, flags, out, route, ws, layer_ws, cuda_stream, &hook);
+  if (st != FMMOE_OK) return st;
+  FMMOE_CUDA_TRY(cudaStreamWaitEvent(s, h->side_join, 0));
+  return fused_run(f, 2, s, s);
 }
 
 extern "C" __attribute__((visibility("default"))) size_t fmmoe_host_staging_bytes(const fmmoe_layer_desc* d, int64_t T) {

@@ -37,6 +37,10 @@ struct fmmoe_handle {
   uint64_t pipe_next;
   cudaEvent_t ticket_ev[kTickets];
   uint64_t ticket_next;
+  // fmmoe_moe_forward_prune: the selection half of the pruning pass runs beside the expert GEMMs
+  bool side_ready;
+  cudaStream_t side_stream;
+  cudaEvent_t side_fork, side_join;
 };
 
 namespace fmmoe {
@@ -195,5 +199,13 @@ struct FinalizeArgs {
   const float* acc; const float* y; const float* ysh; const int32_t* inv_row; const float* topk_w;
 };
 fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_t s);
+
+// fmmoe_prune_visual in two phases (bit 0: ranks, scores, selection on s_select; bit 1: rows on s_rows)
+fmmoe_status prune_visual_phases(fmmoe_handle* h, const fmmoe_prune_params* p, const float* probs, int32_t n_experts,
+                                 const float* attn, const void* x, int32_t dtype, int32_t hidden,
+                                 const uint8_t* is_visual, const int64_t* seq_off, const int64_t* n_vis,
+                                 const int64_t* n_retain, int32_t n_seq, void* x_out, uint8_t* is_visual_out,
+                                 int32_t* keep_idx, uint8_t* kind, int64_t* out_seq_off, void* workspace,
+                                 size_t workspace_bytes, int phases, cudaStream_t s_select, cudaStream_t s_rows);
 
 }  // namespace fmmoe

@@ -556,13 +556,17 @@ extern "C" __attribute__((visibility("default"))) size_t fmmoe_prune_workspace_b
   return plan_prune(n_tokens).total + 256;
 }
 
-extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visual(fmmoe_handle* h, const fmmoe_prune_params* p, const float* probs,
-                                           int32_t n_experts, const float* attn, const void* x, int32_t dtype,
-                                           int32_t hidden, const uint8_t* is_visual, const int64_t* seq_off,
-                                           const int64_t* n_vis, const int64_t* n_retain, int32_t n_seq, void* x_out,
-                                           uint8_t* is_visual_out, int32_t* keep_idx, uint8_t* kind,
-                                           int64_t* out_seq_off, void* workspace, size_t workspace_bytes,
-                                           void* cuda_stream) {
+// The pruning pass in two phases: phase 1 (vision ranks, window scores, selection + compaction map)
+// needs the routing probabilities and the mask only, phase 2 (row gather / merge) needs the rows.
+// phases & 1 enqueues phase 1 on s_select, phases & 2 enqueues phase 2 on s_rows.  A caller that
+// uses two streams orders phase 2 after phase 1 itself.
+fmmoe_status fmmoe::prune_visual_phases(fmmoe_handle* h, const fmmoe_prune_params* p, const float* probs,
+                                        int32_t n_experts, const float* attn, const void* x, int32_t dtype,
+                                        int32_t hidden, const uint8_t* is_visual, const int64_t* seq_off,
+                                        const int64_t* n_vis, const int64_t* n_retain, int32_t n_seq, void* x_out,
+                                        uint8_t* is_visual_out, int32_t* keep_idx, uint8_t* kind,
+                                        int64_t* out_seq_off, void* workspace, size_t workspace_bytes,
+                                        int phases, cudaStream_t s_select, cudaStream_t s_rows) {
   if (!h || !prune_params_ok(p) || !seq_off || !n_vis || !n_retain || !out_seq_off || n_seq < 0)
     return FMMOE_ERR_INVALID_ARG;
   if (n_experts < 1 || hidden < 1 || (dtype != FMMOE_F32 && dtype != FMMOE_BF16)) return FMMOE_ERR_INVALID_ARG;
@@ -591,7 +595,6 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
   while ((int64_t)sel_pad < max_nf) sel_pad <<= 1;
   const size_t sel_smem = (sel_pad > 1024 ? sel_pad : 1024) * 8 + sel_pad;   // sort keys + action bytes of the longest sequence
   if (sel_smem > (size_t)h->max_smem_optin - 1024) return FMMOE_ERR_UNSUPPORTED;
-  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);
 
   PruneDev a = {};
@@ -628,19 +631,23 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
     for (int i = 0; i <= nb; ++i) rel.win_off[i] -= win_base;
     PruneDev al = a;
     al.sim = a.sim + win_base; al.asum = a.asum + win_base;
-    { ProfScope ps(h, FMMOE_KERNEL_PRUNE_INDEX, s); FMMOE_CUDA_TRY(launch_pdl(vis_index_kernel, dim3(nb), dim3(1024), 0, s, 1, al, rel)); }
-    FMMOE_CUDA_TRY(cudaGetLastError());
-    h->launches += 1;
-    if (n_win > 0) {
-      { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SCORE, s); FMMOE_CUDA_TRY(launch_pdl(window_score_kernel, dim3((n_win + 7) / 8), dim3(256), 0, s, 1, al, rel)); }
+    if (phases & 1) {
+      cudaStream_t s = s_select;
+      { ProfScope ps(h, FMMOE_KERNEL_PRUNE_INDEX, s); FMMOE_CUDA_TRY(launch_pdl(vis_index_kernel, dim3(nb), dim3(1024), 0, s, 1, al, rel)); }
+      FMMOE_CUDA_TRY(cudaGetLastError());
+      h->launches += 1;
+      if (n_win > 0) {
+        { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SCORE, s); FMMOE_CUDA_TRY(launch_pdl(window_score_kernel, dim3((n_win + 7) / 8), dim3(256), 0, s, 1, al, rel)); }
+        FMMOE_CUDA_TRY(cudaGetLastError());
+        h->launches += 1;
+      }
+      { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SELECT, s); FMMOE_CUDA_TRY(launch_pdl(select_kernel, dim3(nb), dim3(1024), sel_smem, s, 1, al, rel)); }
       FMMOE_CUDA_TRY(cudaGetLastError());
       h->launches += 1;
     }
-    { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SELECT, s); FMMOE_CUDA_TRY(launch_pdl(select_kernel, dim3(nb), dim3(1024), sel_smem, s, 1, al, rel)); }
-    FMMOE_CUDA_TRY(cudaGetLastError());
-    h->launches += 1;
     const long long rows = rel.out_off[nb] - rel.out_off[0];
-    if (rows > 0) {
+    if ((phases & 2) && rows > 0) {
+      cudaStream_t s = s_rows;
       ProfScope ps(h, FMMOE_KERNEL_PRUNE_COMPACT, s);
       if (dtype == FMMOE_BF16)
         FMMOE_CUDA_TRY(launch_pdl(compact_kernel<__nv_bfloat16>, dim3((unsigned)rows), dim3(256), 0, s, 1, al, rel, (long long)rel.out_off[0], (long long)rows));
@@ -652,6 +659,18 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
     win_base += n_win;
   }
   return FMMOE_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visual(fmmoe_handle* h, const fmmoe_prune_params* p, const float* probs,
+                                           int32_t n_experts, const float* attn, const void* x, int32_t dtype,
+                                           int32_t hidden, const uint8_t* is_visual, const int64_t* seq_off,
+                                           const int64_t* n_vis, const int64_t* n_retain, int32_t n_seq, void* x_out,
+                                           uint8_t* is_visual_out, int32_t* keep_idx, uint8_t* kind,
+                                           int64_t* out_seq_off, void* workspace, size_t workspace_bytes,
+                                           void* cuda_stream) {
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  return prune_visual_phases(h, p, probs, n_experts, attn, x, dtype, hidden, is_visual, seq_off, n_vis, n_retain, n_seq,
+                             x_out, is_visual_out, keep_idx, kind, out_seq_off, workspace, workspace_bytes, 3, s, s);
 }
 
 // ---------------------------------------------------------------------------------------

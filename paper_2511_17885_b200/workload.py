@@ -29,7 +29,7 @@ def upload_weights(w: Dict[str, Optional[np.ndarray]], dtype: str, device: str) 
 class LayerWorkload:
     """One MoE layer over one batch of sequences, followed by one pruning stage.
 
-    step()      : inputs resident in HBM  -> fmmoe_moe_forward + fmmoe_prune_visual
+    step()      : inputs resident in HBM  -> fmmoe_moe_forward_prune (layer, then the pruning stage on its output)
     step_host() : inputs in pinned host memory -> fmmoe_moe_forward_host (H2D, layer, D2H of the
                   layer output) + fmmoe_prune_visual on the device copy + D2H of the pruned rows
     """
@@ -75,11 +75,18 @@ class LayerWorkload:
     def n_tokens(self) -> int:
         return self.cfg.n_tokens
 
-    def step(self):
-        self.h.fmmoe_moe_forward(self.desc, self.ws, self.x, self.mask, self.flags, out=self.out, route=self.route)
-        if self.prune is not None:
+    def step(self, fused: bool = True):
+        if self.prune is not None and not fused:     # the same work as two calls, every kernel on one stream
+            self.h.fmmoe_moe_forward(self.desc, self.ws, self.x, self.mask, self.flags, out=self.out, route=self.route)
             self.last = self.h.fmmoe_prune_visual(self.pp, self.route["probs"], self.attn, self.out, self.mask,
                                                   self.seq_off, self.n_vis, self.n_retain)
+            return self.last
+        if self.prune is not None:
+            self.last = self.h.fmmoe_moe_forward_prune(self.desc, self.ws, self.x, self.mask, self.flags, self.out,
+                                                       self.route, self.pp, self.attn, self.seq_off, self.n_vis,
+                                                       self.n_retain)
+        else:
+            self.h.fmmoe_moe_forward(self.desc, self.ws, self.x, self.mask, self.flags, out=self.out, route=self.route)
         return self.last
 
     def step_host(self):

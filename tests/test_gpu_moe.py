@@ -196,3 +196,47 @@ def test_pipelined_host_batches_match_the_device_path():
         assert row_rel_err(pr_h.float().numpy(), pr["x_out"].float().cpu().numpy()) < 2e-2
     with pytest.raises(B.FmmoeError):
         hd.fmmoe_host_wait(1 << 40)
+
+
+@pytest.mark.parametrize("use_attn", [False, True])
+def test_layer_and_pruning_in_one_call_equals_the_two_calls(use_attn):
+    """fmmoe_moe_forward_prune (selection on a side stream beside the GEMMs) against fmmoe_moe_forward followed by
+    fmmoe_prune_visual: the same keep-set bit for bit; with the fixed-order combine also the same rows bit for bit."""
+    r = np.random.default_rng(21)
+    H, E, I_, K, Kv = 128, 16, 128, 4, 2
+    seq_off, n_vis = [0, 700, 1030, 1500], [520, 200, 331]
+    T = seq_off[-1]
+    mask_np = np.zeros(T, np.uint8)
+    for b in range(3):
+        idx = r.permutation(seq_off[b + 1] - seq_off[b])[:n_vis[b]] + seq_off[b]   # vision tokens interleaved with text
+        mask_np[idx] = 1
+    n_ret = [260, 50, 331]
+    w = random_layer(r, "bf16", H, E, I_, 1, 64)
+    wd = upload_weights(w, "bf16"); ws = B.make_weights(wd)
+    desc = B.make_desc(H, E, I_, 1, 64, K, Kv, torch.bfloat16)
+    x = dev(I.round_to_storage(r.standard_normal((T, H)), "bf16"), torch.bfloat16)
+    mask = dev(mask_np)
+    attn = dev(r.random(T).astype(np.float32)) if use_attn else None
+    pp = B.prune_params(3, 0.1, 0.6 if use_attn else 1.0)
+    hd = handle()
+    for flags in (B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC, B.FLAG_REDUCE_ON | B.FLAG_RESIDUAL):
+        route_a = {"probs": torch.empty(T, E, dtype=torch.float32, device="cuda")}
+        route_b = {"probs": torch.empty(T, E, dtype=torch.float32, device="cuda")}
+        out_a = hd.fmmoe_moe_forward(desc, ws, x, mask, flags, route=route_a)
+        ref = hd.fmmoe_prune_visual(pp, route_a["probs"], attn, out_a, mask, seq_off, n_vis, n_ret)
+        out_b = torch.empty_like(x)
+        for _ in range(2):   # twice: the side stream's second use must be ordered after the first
+            got = hd.fmmoe_moe_forward_prune(desc, ws, x, mask, flags, out_b, route_b, pp, attn, seq_off, n_vis, n_ret)
+        hd.check_status()
+        assert got["out_seq_off"] == ref["out_seq_off"]
+        assert torch.equal(route_a["probs"], route_b["probs"])
+        for k in ("keep_idx", "kind", "is_visual_out"):
+            assert torch.equal(got[k], ref[k]), k
+        if flags & B.FLAG_DETERMINISTIC:
+            assert torch.equal(out_a, out_b) and torch.equal(got["x_out"], ref["x_out"])
+        else:
+            assert row_rel_err(host(got["x_out"]), host(ref["x_out"])) < 2e-2
+    # argument errors surface before anything is enqueued
+    with pytest.raises(B.FmmoeError):
+        hd.fmmoe_moe_forward_prune(desc, ws, x, mask, B.FLAG_REDUCE_ON, out_b, route_b, pp, attn, [0, 700, 1030, 1499],
+                                   n_vis, n_ret)
