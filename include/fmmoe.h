@@ -164,6 +164,9 @@ fmmoe_status fmmoe_moe_forward_host(fmmoe_handle *handle, const fmmoe_layer_desc
  * stream after the layer.  Host buffers should be pinned.  A batch in flight owns its workspace,
  * out_dev, is_visual_dev and host buffers until a ticket taken after it has been waited for: give
  * every batch in flight its own set (two sets alternate for a depth of two).
+ * fmmoe_upload_async: copies bytes from src_host to dst_dev on the upload stream and makes the work
+ * enqueued on cuda_stream AFTER this call wait for the copy (earlier work on cuda_stream is not waited
+ * for: dst_dev must not be in use by it; the ticket rule above covers that).
  * fmmoe_download_async: copies bytes from src_dev to dst_host on the download stream, after the
  * work enqueued on cuda_stream so far (e.g. the rows fmmoe_prune_visual has just produced).
  * fmmoe_host_fence: returns a ticket for everything enqueued on the download stream so far.
@@ -175,6 +178,8 @@ fmmoe_status fmmoe_moe_forward_host_async(fmmoe_handle *handle, const fmmoe_laye
                                           uint32_t flags, void *out_host, const fmmoe_route_out *route,
                                           void *out_dev, uint8_t *is_visual_dev, void *workspace,
                                           size_t workspace_bytes, void *cuda_stream);
+fmmoe_status fmmoe_upload_async(fmmoe_handle *handle, void *dst_dev, const void *src_host, size_t bytes,
+                                void *cuda_stream);
 fmmoe_status fmmoe_download_async(fmmoe_handle *handle, void *dst_host, const void *src_dev, size_t bytes,
                                   void *cuda_stream);
 fmmoe_status fmmoe_host_fence(fmmoe_handle *handle, uint64_t *ticket);

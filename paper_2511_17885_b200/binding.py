@@ -90,6 +90,7 @@ def lib() -> C.CDLL:
     L.fmmoe_moe_forward_host_async.argtypes = L.fmmoe_moe_forward_host.argtypes
     L.fmmoe_moe_forward_host_async.restype = C.c_int
     L.fmmoe_download_async.argtypes = [vp, vp, vp, sz, vp]; L.fmmoe_download_async.restype = C.c_int
+    L.fmmoe_upload_async.argtypes = [vp, vp, vp, sz, vp]; L.fmmoe_upload_async.restype = C.c_int
     L.fmmoe_host_fence.argtypes = [vp, C.POINTER(C.c_uint64)]; L.fmmoe_host_fence.restype = C.c_int
     L.fmmoe_host_wait.argtypes = [vp, C.c_uint64]; L.fmmoe_host_wait.restype = C.c_int
     L.fmmoe_profile_enable.argtypes = [vp, C.c_int]; L.fmmoe_profile_enable.restype = C.c_int
@@ -181,8 +182,9 @@ def fmmoe_stack_output_layout(stages, n_layers: int, seq_off, n_vis):
 
 
 def make_weights(w: Dict[str, Optional[torch.Tensor]]) -> Weights:
-    """Device tensors -> pointer struct.  The caller keeps the tensors alive."""
+    """Device tensors -> pointer struct.  The struct keeps a reference to every tensor it points into."""
     ws = Weights()
+    ws._tensors = dict(w)
     for name, _ in Weights._fields_:
         t = w.get(name)
         if t is not None:
@@ -320,6 +322,14 @@ class Handle:
             T, flags, C.c_void_p(out_host.data_ptr()) if out_host is not None else None,
             C.byref(ro) if ro is not None else None, _ptr(out_dev), _ptr(is_visual_dev), C.c_void_p(aligned),
             C.c_size_t(ws.numel() - (aligned - base)), _stream()), "fmmoe_moe_forward_host_async")
+
+    def fmmoe_upload_async(self, dst_dev: torch.Tensor, src_host: torch.Tensor):
+        """Host -> device copy on the handle's upload stream; later work on the current stream waits for it."""
+        assert dst_dev.is_cuda and not src_host.is_cuda and dst_dev.is_contiguous() and src_host.is_contiguous()
+        n = src_host.numel() * src_host.element_size()
+        assert dst_dev.numel() * dst_dev.element_size() >= n
+        _check(lib().fmmoe_upload_async(self._h, _ptr(dst_dev), C.c_void_p(src_host.data_ptr()), n, _stream()),
+               "fmmoe_upload_async")
 
     def fmmoe_download_async(self, dst_host: torch.Tensor, src_dev: torch.Tensor):
         """Device -> host copy on the handle's download stream, after the work enqueued on the current stream."""

@@ -441,6 +441,19 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_moe_forward
   return FMMOE_OK;
 }
 
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_upload_async(fmmoe_handle* h, void* dst_dev, const void* src_host,
+                                                                                   size_t bytes, void* cuda_stream) {
+  if (!h || (bytes && (!dst_dev || !src_host))) return FMMOE_ERR_INVALID_ARG;
+  if (bytes == 0) return FMMOE_OK;
+  const fmmoe_status st = pipe_init(h);
+  if (st != FMMOE_OK) return st;
+  const cudaEvent_t uploaded = pipe_event(h);
+  FMMOE_CUDA_TRY(cudaMemcpyAsync(dst_dev, src_host, bytes, cudaMemcpyHostToDevice, h->up_stream));
+  FMMOE_CUDA_TRY(cudaEventRecord(uploaded, h->up_stream));
+  FMMOE_CUDA_TRY(cudaStreamWaitEvent(static_cast<cudaStream_t>(cuda_stream), uploaded, 0));
+  return FMMOE_OK;
+}
+
 extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_download_async(fmmoe_handle* h, void* dst_host, const void* src_dev,
                                                                                      size_t bytes, void* cuda_stream) {
   if (!h || (bytes && (!dst_host || !src_dev))) return FMMOE_ERR_INVALID_ARG;

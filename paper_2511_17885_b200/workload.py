@@ -105,30 +105,36 @@ class LayerWorkload:
 
     def _pipe_slots(self):
         if getattr(self, "_slots", None) is None:
-            self._slots = [{"out_dev": torch.empty_like(self.x), "mask_dev": torch.empty_like(self.mask),
+            self._slots = [{"x_dev": torch.empty_like(self.x), "out_dev": torch.empty_like(self.x),
+                            "mask_dev": torch.empty_like(self.mask),
                             "out_host": torch.empty_like(self.x_host).pin_memory(), "pruned_host": None,
                             "pruned_dev": None, "ticket": None} for _ in range(self.PIPE_DEPTH)]
         return self._slots
 
     def step_host_async(self, i: int):
         """Batch i of a stream of independent batches whose activations live in pinned host memory: the upload
-        of batch i overlaps the layer of batch i-1 and the downloads of batch i-2 (fmmoe_moe_forward_host_async,
-        fmmoe_prune_visual, fmmoe_download_async).  Every batch is uploaded, computed and downloaded in full
+        of batch i overlaps the layer of batch i-1 and the downloads of batch i-2 (fmmoe_upload_async, the same
+        device call as step(), fmmoe_download_async).  Every batch is uploaded, computed and downloaded in full
         (layer output and pruned rows); drain_host() returns when all results are in host memory."""
         sl = self._pipe_slots()[i % self.PIPE_DEPTH]
         if sl["ticket"] is not None:
             self.h.fmmoe_host_wait(sl["ticket"])       # the slot's previous batch is fully on the host
-        self.h.fmmoe_moe_forward_host_async(self.desc, self.ws, self.x_host, self.mask_host, self.flags, sl["out_host"],
-                                            slot=i % self.PIPE_DEPTH, route=self.route, out_dev=sl["out_dev"],
-                                            is_visual_dev=sl["mask_dev"])
+        self.h.fmmoe_upload_async(sl["x_dev"], self.x_host)
+        self.h.fmmoe_upload_async(sl["mask_dev"], self.mask_host)
         if self.prune is not None:
-            r = self.h.fmmoe_prune_visual(self.pp, self.route["probs"], self.attn, sl["out_dev"], sl["mask_dev"],
-                                          self.seq_off, self.n_vis, self.n_retain, want_aux=False)
+            r = self.h.fmmoe_moe_forward_prune(self.desc, self.ws, sl["x_dev"], sl["mask_dev"], self.flags, sl["out_dev"],
+                                               self.route, self.pp, self.attn, self.seq_off, self.n_vis, self.n_retain,
+                                               want_aux=False)
             if sl["pruned_host"] is None or sl["pruned_host"].shape != r["x_out"].shape:
                 sl["pruned_host"] = torch.empty(r["x_out"].shape, dtype=r["x_out"].dtype).pin_memory()
             sl["pruned_dev"] = r["x_out"]              # stays referenced until the slot's ticket has been waited for
+            self.h.fmmoe_download_async(sl["out_host"], sl["out_dev"])
             self.h.fmmoe_download_async(sl["pruned_host"], r["x_out"])
             self.pruned_host = sl["pruned_host"]
+        else:
+            self.h.fmmoe_moe_forward(self.desc, self.ws, sl["x_dev"], sl["mask_dev"], self.flags, out=sl["out_dev"],
+                                     route=self.route)
+            self.h.fmmoe_download_async(sl["out_host"], sl["out_dev"])
         sl["ticket"] = self.h.fmmoe_host_fence()
         return sl
 

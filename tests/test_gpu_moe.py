@@ -240,3 +240,35 @@ def test_layer_and_pruning_in_one_call_equals_the_two_calls(use_attn):
     with pytest.raises(B.FmmoeError):
         hd.fmmoe_moe_forward_prune(desc, ws, x, mask, B.FLAG_REDUCE_ON, out_b, route_b, pp, attn, [0, 700, 1030, 1499],
                                    n_vis, n_ret)
+
+
+def test_upload_and_download_streams_order_against_the_compute_stream():
+    """fmmoe_upload_async -> device call -> fmmoe_download_async, four batches over two buffer sets."""
+    r = np.random.default_rng(31)
+    T, H, E, I_, K, Kv = 260, 128, 8, 128, 2, 1
+    w = random_layer(r, "bf16", H, E, I_, 0, 0)
+    wd = upload_weights(w, "bf16"); ws = B.make_weights(wd)
+    desc = B.make_desc(H, E, I_, 0, 0, K, Kv, torch.bfloat16)
+    hd = handle()
+    mask = dev((r.random(T) < 0.6).astype(np.uint8))
+    xs = [torch.from_numpy(I.round_to_storage(r.standard_normal((T, H)), "bf16")).to(torch.bfloat16).pin_memory()
+          for _ in range(4)]
+    sets = [{"x": torch.empty(T, H, dtype=torch.bfloat16, device="cuda"),
+             "out": torch.empty(T, H, dtype=torch.bfloat16, device="cuda"), "ticket": None} for _ in range(2)]
+    res = []
+    for i, xh in enumerate(xs):
+        st = sets[i % 2]
+        if st["ticket"] is not None:
+            hd.fmmoe_host_wait(st["ticket"])
+        hd.fmmoe_upload_async(st["x"], xh)
+        hd.fmmoe_moe_forward(desc, ws, st["x"], mask, B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC, out=st["out"])
+        oh = torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
+        hd.fmmoe_download_async(oh, st["out"])
+        st["ticket"] = hd.fmmoe_host_fence()
+        res.append((oh, st["ticket"]))
+    for oh, t in res:
+        hd.fmmoe_host_wait(t)
+    hd.check_status()
+    for xh, (oh, _) in zip(xs, res):
+        ref = hd.fmmoe_moe_forward(desc, ws, xh.cuda(), mask, B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC)
+        assert torch.equal(oh, ref.cpu())
