@@ -35,17 +35,25 @@ __global__ void __launch_bounds__(P_THREADS) scan_kernel(const PermuteDev a) {
   for (int e = warp; e < a.E; e += P_THREADS / 32) {
     int32_t* row = a.blk_cnt + (long long)e * a.n_blk;
     int running = 0;
-    for (int b0 = 0; b0 < a.n_blk; b0 += 32) {
-      const int b = b0 + lane;
-      const int v = b < a.n_blk ? row[b] : 0;
-      int incl = v;
+    for (int b0 = 0; b0 < a.n_blk; b0 += 128) {   // four independent loads per lane, then the scans
+      int v[4];
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += n;
+      for (int j = 0; j < 4; ++j) {
+        const int b = b0 + 32 * j + lane;
+        v[j] = b < a.n_blk ? row[b] : 0;
       }
-      if (b < a.n_blk) row[b] = running + incl - v;
-      running += __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int b = b0 + 32 * j + lane;
+        int incl = v[j];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int n = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += n;
+        }
+        if (b < a.n_blk) row[b] = running + incl - v[j];
+        running += __shfl_sync(0xffffffffu, incl, 31);
+      }
     }
     if (lane == 0) s_cnt[e] = running;
   }
