@@ -66,6 +66,7 @@ struct Segment {          // routed experts (0) or shared experts (1)
 struct GemmParams {
   const MTile* mtiles;        // routed M-tiles
   const int32_t* n_mtiles;    // device: number of routed M-tiles
+  int max_mtiles;             // capacity of `mtiles` (a corrupt count must not walk past it)
   int32_t* tile_counter;      // device: next tile to hand out (zero at launch)
   int shared_mtiles;          // N_s * ceil(T/128), host-known
   int mt_per_shared;          // ceil(T/128)
@@ -179,7 +180,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   // barriers, tensor memory and descriptors are set up; everything below reads what earlier
   // kernels of the stream wrote
   pdl_wait();
-  const int n_mt_r = p.n_mtiles ? *p.n_mtiles : 0;
+  const int n_mt_r = p.n_mtiles ? min(max(*p.n_mtiles, 0), p.max_mtiles) : 0;
   const int total_tiles = n_mt_r * p.seg[0].n_nblocks + p.shared_mtiles * p.seg[1].n_nblocks;
 
   if (warp == 0) {
@@ -499,7 +500,7 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   if (!ok) return FMMOE_ERR_CUDA;
 
   GemmParams p1 = {};
-  p1.mtiles = a.mtiles; p1.n_mtiles = a.n_mtiles;
+  p1.mtiles = a.mtiles; p1.n_mtiles = a.n_mtiles; p1.max_mtiles = a.max_mtiles;
   p1.shared_mtiles = Ns * mtps; p1.mt_per_shared = mtps; p1.T = a.T;
   p1.seg[0] = Segment{(I + 127) / 128, H / G_BK, I, I, 0, 0, I};
   p1.seg[1] = Segment{Ns ? (Is + 127) / 128 : 0, H / G_BK, Is, Is, 0, (int)a.T, Is};
