@@ -253,7 +253,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------ UMMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(G_BM, 256);
+      // A tile with at most 64 valid rows runs as M = 64 MMAs: same duration, half the datapaths
+      // switching (at batch 1 the GPU sits at its power cap, where that buys clock)
+      constexpr uint32_t idesc128 = umma_idesc_bf16(G_BM, 256), idesc64 = umma_idesc_bf16(64, 256);
       int stage = 0; uint32_t phase = 0;
       int as = 0; uint32_t aphase = 0;
       bool ok = true;
@@ -263,6 +265,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         if (!mbar_wait(&sfull_bar[slot], sph, abort_flag)) { ok = false; break; }
         const int tile = ring[slot * G_SLOT_INTS];
         const int seg = ring[slot * G_SLOT_INTS + 1];
+        const uint32_t idesc = ring[slot * G_SLOT_INTS + 4] <= 64 ? idesc64 : idesc128;
         mbar_arrive(&sempty_bar[slot]);
         if (tile < 0) break;
         const int k_blocks = p.seg[seg].k_blocks;
@@ -340,7 +343,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int q = warp & 3;                 // TMEM lane quarter this warp may access
-    const int r = q * 32 + lane;            // row of the tile held by this thread
     float* stg = epi + q * 32 * G_EPI_LD;   // this warp's 32 x 32 transpose block
     int as = 0; uint32_t aphase = 0;
     bool ok = true;
@@ -357,8 +359,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
       if (!mbar_wait(&tfull_bar[as], aphase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + as * 256 + (static_cast<uint32_t>(q * 32) << 16);
-      const int rows_w = ti.rows - q * 32;   // valid rows among this warp's 32 (may be <= 0)
-      const long long out_row0 = (long long)ti.row0 + q * 32 + (long long)ti.group_local * sg.out_group_stride;
+      // M = 128: row i of the tile sits in TMEM lane i.  M = 64 (tiles of at most 64 rows): row i sits in
+      // lane 32 * (i / 16) + i % 16, so each warp's lane quarter holds 16 rows in its lanes 0..15.
+      const int rpw = ti.rows <= 64 ? 16 : 32;          // rows per warp
+      const int r = q * rpw + lane;                     // row of the tile held by this thread (if lane < rpw)
+      const int rows_w = min(ti.rows - q * rpw, rpw);   // valid rows among this warp's (may be <= 0)
+      const long long out_row0 = (long long)ti.row0 + q * rpw + (long long)ti.group_local * sg.out_group_stride;
       if (MODE == 0) {
         uint32_t* stg32 = reinterpret_cast<uint32_t*>(stg);   // [32][17] packed bf16 pairs
         __nv_bfloat16* dst0 = p.act[ti.seg] + out_row0 * sg.ld_out + ti.nb * 128;
