@@ -272,3 +272,21 @@ def test_upload_and_download_streams_order_against_the_compute_stream():
     for xh, (oh, _) in zip(xs, res):
         ref = hd.fmmoe_moe_forward(desc, ws, xh.cuda(), mask, B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC)
         assert torch.equal(oh, ref.cpu())
+
+
+def test_host_tickets_survive_the_ring_wrapping_around():
+    """More fences than the handle keeps events for: every ticket, however old, can still be waited for."""
+    hd = handle()
+    src = torch.arange(1024, dtype=torch.int32, device="cuda")
+    dst = torch.zeros(1024, dtype=torch.int32).pin_memory()
+    tickets = []
+    for i in range(150):
+        src.add_(1)
+        hd.fmmoe_download_async(dst, src)
+        tickets.append(hd.fmmoe_host_fence())
+    assert tickets == list(range(tickets[0], tickets[0] + 150))
+    for t in (tickets[0], tickets[70], tickets[-1]):
+        hd.fmmoe_host_wait(t)
+    assert torch.equal(dst, src.cpu())
+    with pytest.raises(B.FmmoeError):
+        hd.fmmoe_host_wait(tickets[-1] + 1)
