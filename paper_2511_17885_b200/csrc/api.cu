@@ -107,7 +107,7 @@ static fmmoe_status check_common(fmmoe_handle* h, const fmmoe_layer_desc* d, con
 
 static fmmoe_status run_route(fmmoe_handle* h, const fmmoe_layer_desc& d, const fmmoe_weights& w, const void* x,
                               const uint8_t* is_visual, int64_t T, uint32_t flags, const RoutePtrs& r,
-                              bool need_permute, float* acc_zero, cudaStream_t s) {
+                              bool need_permute, float* acc_zero, cudaStream_t s, void* gather_xp = nullptr) {
   RouteArgs ra;
   ra.x = x; ra.router_w = w.router_w; ra.router_b = w.router_b; ra.is_visual = is_visual;
   ra.T = T; ra.H = d.hidden; ra.E = d.n_experts; ra.K = d.top_k; ra.Kv = d.top_k_vis;
@@ -124,6 +124,8 @@ static fmmoe_status run_route(fmmoe_handle* h, const fmmoe_layer_desc& d, const 
   pa.block_m = d.dtype == FMMOE_BF16 ? TC_BLOCK_M : F32_BLOCK_M;
   pa.expert_off = r.expert_off; pa.row_token = r.row_token; pa.row_gate = r.row_gate; pa.inv_row = r.inv_row;
   pa.mtiles = r.mtiles; pa.n_mtiles = r.misc;
+  pa.gather_x = gather_xp ? x : nullptr; pa.gather_xp = gather_xp;
+  pa.gather_row_bytes = d.hidden * (d.dtype == FMMOE_BF16 ? 2 : 4);
   return launch_permute(h, pa, s);
 }
 
@@ -253,7 +255,10 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   const bool det = flags & FMMOE_FLAG_DETERMINISTIC;
   const RoutePtrs r = bind_route(pl, ws, route);
   // the router clears the scheduler words and (atomic mode) the fp32 accumulator it owns rows of
-  st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, det ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s);
+  // bf16 at small batch: the permutation's scatter pass also writes the expert-grouped copy of x
+  const bool copy_rows = d->dtype == FMMOE_BF16 && !gather_rows_in_gemm(T);
+  st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, det ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s,
+                 copy_rows ? ws + pl.xp_off : nullptr);
   if (st != FMMOE_OK) return st;
   if (after_route) {
     st = after_route->fn(after_route->ctx);
@@ -272,10 +277,6 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   fa.deterministic = det; fa.d_status = h->d_status;
   if (d->dtype == FMMOE_BF16) {
     fa.gather_in_gemm = gather_rows_in_gemm(T) ? 1 : 0;
-    if (!fa.gather_in_gemm) {
-      st = launch_gather_rows(h, x, r.row_token, r.expert_off, d->n_experts, pl.p_max, d->hidden, 2, fa.xp, s);
-      if (st != FMMOE_OK) return st;
-    }
     st = launch_ffn_tc(h, fa, s);
   } else {
     st = launch_ffn_f32(h, fa, s);

@@ -170,10 +170,10 @@ struct PermuteArgs {
   int64_t T; int K, E; int block_m;
   int32_t* expert_off; int32_t* row_token; float* row_gate; int32_t* inv_row;
   MTile* mtiles; int32_t* n_mtiles;
+  // optional: also write the expert-grouped copy of x (xp[row] = x[token]) in the scatter pass
+  const void* gather_x; void* gather_xp; int gather_row_bytes;
 };
 fmmoe_status launch_permute(fmmoe_handle* h, const PermuteArgs& a, cudaStream_t s);
-fmmoe_status launch_gather_rows(fmmoe_handle* h, const void* x, const int32_t* row_token, const int32_t* expert_off,
-                                int E, int64_t p_max, int H, int elem_bytes, void* xp, cudaStream_t s);
 
 struct FfnArgs {   // both paths
   const fmmoe_layer_desc* d; const fmmoe_weights* w;

@@ -9,6 +9,7 @@
 //   scan_kernel    : per expert an exclusive scan of the block counts (in place), the scan of
 //                    the expert totals (expert_off) and the list of 128-row M-tiles
 //   scatter_kernel : row = expert_off[e] + block offset + in-block rank, for every pair
+//   scatter_gather_kernel : the same, and the pair's row of x copied to its row of the expert-grouped copy
 #include <cuda_bf16.h>
 
 #include "internal.h"
@@ -110,22 +111,36 @@ __global__ void __launch_bounds__(256) scatter_kernel(const PermuteDev a) {
   a.inv_row[i] = row;
 }
 
-// Copy the routed rows of X into expert-grouped order: xp[row] = x[row_token[row]].
-// One warp per row, 16-byte accesses.
-__global__ void gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ row_token,
-                                   const int32_t* __restrict__ expert_off, int E, long long p_max, int row_vec,
-                                   uint4* __restrict__ xp) {
+// scatter_kernel and gather_rows_kernel in one pass for small batches: one warp per (token, slot)
+// pair computes the pair's row (lane 0, as scatter_kernel does) and then copies the token's row of X
+// to that row of the expert-grouped copy.  Saves a dependent launch on the way to GEMM-1.
+__global__ void __launch_bounds__(256) scatter_gather_kernel(const PermuteDev a, const uint4* __restrict__ x, int row_vec,
+                                                             uint4* __restrict__ xp) {
   pdl_launch_dependents();
   pdl_wait();
-  const int P = expert_off[E];
-  const int warps = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
-  for (long long row = (long long)blockIdx.x * warps + (threadIdx.x >> 5); row < P; row += (long long)gridDim.x * warps) {
-    const long long t = row_token[row];
-    const uint4* src = x + t * row_vec;
-    uint4* dst = xp + row * row_vec;
-    for (int i = lane; i < row_vec; i += 32) dst[i] = src[i];
+  const long long i = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (i >= a.T * a.K) return;
+  const long long t = i / a.K;
+  int row = -1;
+  if (lane == 0) {
+    const int e = a.topk_idx[i];
+    if (e >= 0 && e < a.E) {
+      row = a.expert_off[e] + a.blk_cnt[(long long)e * a.n_blk + (int)(t / a.blk_tokens)] + a.inv_row[i];
+      if (row < 0 || row >= a.expert_off[a.E]) {
+        row = -1;                            // cannot happen for a consistent routing record
+      } else {
+        a.row_token[row] = (int32_t)t;
+        a.row_gate[row] = a.topk_w[i];
+        a.inv_row[i] = row;
+      }
+    }
   }
+  row = __shfl_sync(0xffffffffu, row, 0);
+  if (row < 0) return;
+  const uint4* src = x + t * row_vec;
+  uint4* dst = xp + (long long)row * row_vec;
+  for (int j = lane; j < row_vec; j += 32) dst[j] = src[j];
 }
 
 fmmoe_status launch_permute(fmmoe_handle* h, const PermuteArgs& a, cudaStream_t s) {
@@ -139,28 +154,15 @@ fmmoe_status launch_permute(fmmoe_handle* h, const PermuteArgs& a, cudaStream_t 
   {
     ProfScope ps(h, FMMOE_KERNEL_PERMUTE, s);
     FMMOE_CUDA_TRY(launch_pdl(scan_kernel, dim3(1), dim3(P_THREADS), 0, s, 1, d));
-    FMMOE_CUDA_TRY(launch_pdl(scatter_kernel, dim3((unsigned)((pairs + 255) / 256)), dim3(256), 0, s, 1, d));
+    if (a.gather_x) {
+      FMMOE_CUDA_TRY(launch_pdl(scatter_gather_kernel, dim3((unsigned)((pairs + 7) / 8)), dim3(256), 0, s, 1, d,
+                                static_cast<const uint4*>(a.gather_x), a.gather_row_bytes / 16, static_cast<uint4*>(a.gather_xp)));
+    } else {
+      FMMOE_CUDA_TRY(launch_pdl(scatter_kernel, dim3((unsigned)((pairs + 255) / 256)), dim3(256), 0, s, 1, d));
+    }
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 2;
-  return FMMOE_OK;
-}
-
-fmmoe_status launch_gather_rows(fmmoe_handle* h, const void* x, const int32_t* row_token, const int32_t* expert_off,
-                                int E, int64_t p_max, int H, int elem_bytes, void* xp, cudaStream_t s) {
-  if (p_max == 0) return FMMOE_OK;
-  const int row_vec = H * elem_bytes / 16;
-  const int threads = 256;
-  long long blocks = (p_max + 7) / 8;
-  const long long cap = (long long)h->sm_count * 8;
-  if (blocks > cap) blocks = cap;
-  {
-    ProfScope ps(h, FMMOE_KERNEL_GATHER, s);
-    FMMOE_CUDA_TRY(launch_pdl(gather_rows_kernel, dim3((unsigned)blocks), dim3(threads), 0, s, 1, static_cast<const uint4*>(x), row_token,
-                              expert_off, E, (long long)p_max, row_vec, static_cast<uint4*>(xp)));
-  }
-  FMMOE_CUDA_TRY(cudaGetLastError());
-  h->launches += 1;
   return FMMOE_OK;
 }
 
