@@ -29,7 +29,7 @@ WORKLOADS = ("C0", "C1", "C2", "C2x4", "C3", "C4")
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
 # ncu captures summarised under profiles/ (null until a capture for that workload exists).
-NCU_TRAFFIC_BYTES = {"C1": {"gemm1": 871.3e6, "gemm2": 502.4e6}}   # profiles/kernels_c1_full_set.md
+NCU_TRAFFIC_BYTES = {"C1": {"gemm1": 870.6e6, "gemm2": 502.8e6}}   # profiles/kernels_c1_full_set.md
 
 
 def load_peaks():
