@@ -236,6 +236,9 @@ def test_layer_and_pruning_in_one_call_equals_the_two_calls(use_attn):
             assert torch.equal(out_a, out_b) and torch.equal(got["x_out"], ref["x_out"])
         else:
             assert row_rel_err(host(got["x_out"]), host(ref["x_out"])) < 2e-2
+        # within one call the pruned rows are the call's own layer output: copied rows bit for bit
+        copied = got["kind"] != 2
+        assert torch.equal(got["x_out"][copied], out_b[got["keep_idx"][copied].long()])
     # argument errors surface before anything is enqueued
     with pytest.raises(B.FmmoeError):
         hd.fmmoe_moe_forward_prune(desc, ws, x, mask, B.FLAG_REDUCE_ON, out_b, route_b, pp, attn, [0, 700, 1030, 1499],
