@@ -203,13 +203,41 @@ class StackWorkload:
                                    self.seq_off, self.n_vis, 0, x_out=self.x_out, is_visual_out=self.mask_out)
         return self.x_out
 
+    PIPE_DEPTH = 2   # batches in flight in the pipelined end-to-end step
+
     def step_host(self):
-        self.x.copy_(self.x_host, non_blocking=True)
-        self.mask.copy_(self.mask_host, non_blocking=True)
+        """One batch at a time: upload, the stack, download, host-side wait (all through the library's calls)."""
+        self.h.fmmoe_upload_async(self.x, self.x_host)
+        self.h.fmmoe_upload_async(self.mask, self.mask_host)
         self.step()
-        self.out_host.copy_(self.x_out, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        self.h.fmmoe_download_async(self.out_host, self.x_out)
+        self.h.fmmoe_host_wait(self.h.fmmoe_host_fence())
         return self.out_host
+
+    def step_host_async(self, i: int):
+        """Batch i of a stream of independent batches in pinned host memory, PIPE_DEPTH in flight: the upload of
+        batch i overlaps the stack of batch i-1 and the download of batch i-2."""
+        if getattr(self, "_slots", None) is None:
+            self._slots = [{"x": torch.empty_like(self.x), "mask": torch.empty_like(self.mask),
+                            "x_out": torch.empty_like(self.x_out), "mask_out": torch.empty_like(self.mask_out),
+                            "out_host": torch.empty_like(self.out_host).pin_memory(), "ticket": None}
+                           for _ in range(self.PIPE_DEPTH)]
+        sl = self._slots[i % self.PIPE_DEPTH]
+        if sl["ticket"] is not None:
+            self.h.fmmoe_host_wait(sl["ticket"])
+        self.h.fmmoe_upload_async(sl["x"], self.x_host)
+        self.h.fmmoe_upload_async(sl["mask"], self.mask_host)
+        self.h.fmmoe_stack_forward(self.desc, self.wstructs, self.reduce_from, self.stages, sl["x"], sl["mask"],
+                                   self.seq_off, self.n_vis, 0, x_out=sl["x_out"], is_visual_out=sl["mask_out"])
+        self.h.fmmoe_download_async(sl["out_host"], sl["x_out"])
+        sl["ticket"] = self.h.fmmoe_host_fence()
+        return sl
+
+    def drain_host(self):
+        for sl in getattr(self, "_slots", None) or []:
+            if sl["ticket"] is not None:
+                self.h.fmmoe_host_wait(sl["ticket"])
+                sl["ticket"] = None
 
     def h2d_bytes(self) -> int:
         return self.x_host.numel() * self.x_host.element_size() + self.mask_host.numel()
