@@ -188,7 +188,9 @@ fmmoe_status fmmoe_host_wait(fmmoe_handle *handle, uint64_t ticket);
 /* Optional per-kernel timeline.  While enabled, every kernel the handle launches is
  * bracketed by CUDA events on the launching stream (host-side event objects only; no
  * device memory).  fmmoe_profile_read synchronises the device and returns the summed
- * duration and the number of launches of one kernel since the last reset. */
+ * duration and the number of launches of one kernel since the last reset.
+ * FMMOE_KERNEL_PERMUTE covers the scan and the scatter pass (which also writes the expert-ordered copy of x
+ * at small batch); FMMOE_KERNEL_GATHER is kept for numbering only and reports no launches. */
 enum {
   FMMOE_KERNEL_ROUTE = 0, FMMOE_KERNEL_PERMUTE = 1, FMMOE_KERNEL_GATHER = 2, FMMOE_KERNEL_GEMM1 = 3,
   FMMOE_KERNEL_GEMM2 = 4, FMMOE_KERNEL_FINALIZE = 5, FMMOE_KERNEL_PRUNE_INDEX = 6, FMMOE_KERNEL_PRUNE_SCORE = 7,
