@@ -103,6 +103,7 @@ class ClockSampler:
 
     def __init__(self, index):
         self.samples, self.reasons, self.max_mhz, self.ok = [], set(), None, False
+        self.power_w = []
         self._stop = threading.Event()
         try:
             import pynvml
@@ -110,6 +111,10 @@ class ClockSampler:
             self.nv = pynvml
             self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM))
+            try:
+                self.power_limit_w = pynvml.nvmlDeviceGetEnforcedPowerLimit(self.dev) / 1000.0
+            except Exception:
+                self.power_limit_w = None
             self.ok = True
         except Exception:
             self.ok = False
@@ -120,6 +125,10 @@ class ClockSampler:
             return
         try:
             self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.dev, self.nv.NVML_CLOCK_SM)))
+            try:
+                self.power_w.append(self.nv.nvmlDeviceGetPowerUsage(self.dev) / 1000.0)
+            except Exception:
+                pass
             try:
                 r = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev))
             except Exception:
@@ -147,7 +156,9 @@ class ClockSampler:
 
     def summary(self):
         return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w": float(np.median(self.power_w)) if self.power_w else None,
+                "power_limit_w": getattr(self, "power_limit_w", None)}
 
 
 def settle_clocks(step, index, min_s=0.4, max_s=3.0):
