@@ -94,7 +94,11 @@ typedef struct {
 typedef struct fmmoe_handle fmmoe_handle;   /* opaque: device, SM count, status word, launch counter */
 
 /* Create a handle on CUDA device `device` (allocates a few hundred bytes of
- * device memory for the status word).  Not thread-safe per handle. */
+ * device memory for the status word, and loads the pruning kernels together with the
+ * built-in scratch array of fmmoe_prune_visual_static onto the device).  Not thread-safe
+ * per handle.  Environment, read once here: FMMOE_DEBUG_SYNC=1 synchronises after every
+ * kernel and reports the first failing one on stderr; FMMOE_GATHER_MIN_TOKENS=n moves the
+ * token count from which GEMM-1 gathers the routed rows itself (default 12288). */
 fmmoe_status fmmoe_create(fmmoe_handle **handle, int device);
 fmmoe_status fmmoe_destroy(fmmoe_handle *handle);
 const char  *fmmoe_status_string(fmmoe_status s);
@@ -338,14 +342,20 @@ fmmoe_status fmmoe_stack_forward(fmmoe_handle *handle, const fmmoe_layer_desc *d
  *     (fmmoe_profile_enable) in such a setting: it creates event objects on demand.
  *   - Limit: seq_off[n_seq] <= FMMOE_STATIC_PRUNE_MAX_TOKENS tokens per call; more returns
  *     FMMOE_ERR_TOO_LARGE before anything is enqueued.
- *   - The first call on each device looks up the array's device address (a one-time
- *     set-up step guarded by a mutex); make that first call before starting any stream
- *     capture on that device.
+ *   - All set-up happens in fmmoe_create, with the handle's device current: the pruning
+ *     kernels and the array are loaded onto the device there (under CUDA's lazy module
+ *     loading that is the moment their device memory is taken), the array's device address
+ *     is looked up and cached per device, and the selection kernel's shared-memory limit is
+ *     raised.  So create the handle at start-up, while the process can still obtain device
+ *     memory, and before starting any stream capture on that device; the pruning call
+ *     itself then does no set-up at all.
  *   - All calls on a device share the one array, and it keeps whatever the previous call
- *     left in it.  No part of it needs clearing (each pass writes every word before reading
- *     it), but two calls whose kernels may overlap on the GPU - different streams, or
- *     different host threads - race on it: serialise them, or use fmmoe_prune_visual with
- *     separate workspaces. */
+ *     left in it.  No part of it needs clearing: a pass writes what it reads, and every
+ *     index a kernel takes from the array is range-checked, so a call whose mask contradicts
+ *     its n_vis (reported as FMMOE_ERR_INTERNAL by fmmoe_get_status) cannot be led out of
+ *     bounds by the previous call's leftovers.  But two calls whose kernels may overlap on
+ *     the GPU - different streams, or different host threads - race on it: serialise them,
+ *     or use fmmoe_prune_visual with separate workspaces. */
 #define FMMOE_STATIC_PRUNE_MAX_TOKENS 32768
 fmmoe_status fmmoe_prune_visual_static(fmmoe_handle *handle, const fmmoe_prune_params *p,
                                        const float *probs, int32_t n_experts, const float *attn,

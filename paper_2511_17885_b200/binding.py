@@ -473,6 +473,23 @@ class Handle:
         nv = (C.c_int64 * max(B, 1))(*[int(v) for v in n_vis])
         nr = (C.c_int64 * max(B, 1))(*[int(v) for v in n_retain])
         oo = arr()
+        # The kernels write T' rows whatever the buffers hold, so the outputs are checked here against the
+        # data-independent output size (host arithmetic only, nothing is allocated).  Problems beyond the
+        # built-in scratch are left to the library, which refuses them before it touches any buffer.
+        if int(seq_off[B]) <= STATIC_PRUNE_MAX_TOKENS:
+            t_out = 0
+            for b in range(B):
+                kept, _, _ = fmmoe_prune_kept_count(int(n_vis[b]), int(n_retain[b]), p)
+                if kept < 0:
+                    raise FmmoeError(1, "fmmoe_prune_kept_count")
+                t_out += int(seq_off[b + 1]) - int(seq_off[b]) - int(n_vis[b]) + kept
+            if (tuple(x_out.shape) != (t_out, x.shape[1]) or x_out.dtype != x.dtype or x_out.device != x.device
+                    or not x_out.is_contiguous()):
+                raise ValueError(f"x_out must be a contiguous [{t_out}, {x.shape[1]}] {x.dtype} tensor on {x.device}")
+            for name, t, dt in (("is_visual_out", is_visual_out, torch.uint8), ("keep_idx", keep_idx, torch.int32),
+                                ("kind", kind, torch.uint8)):
+                if t is not None and (t.numel() < t_out or t.dtype != dt or t.device != x.device or not t.is_contiguous()):
+                    raise ValueError(f"{name} must be a contiguous {dt} tensor of at least {t_out} elements on {x.device}")
         _check(lib().fmmoe_prune_visual_static(self._h, C.byref(p), _ptr(probs), probs.shape[1], _ptr(attn), _ptr(x),
                                                _dtype_code(x.dtype), x.shape[1], _ptr(is_visual), so, nv, nr, B,
                                                _ptr(x_out), _ptr(is_visual_out), _ptr(keep_idx), _ptr(kind), oo,

@@ -162,7 +162,14 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
   h->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
   h->launches = 0;
   h->d_status = nullptr; h->h_status = nullptr; h->encode_tiled = nullptr;
-  h->tc_attr_set = false; h->profiling = false; h->ev_used = 0;
+  h->tc_attr_set = false; h->route_attr_set = false; h->route_f32_attr_mask = 0; h->profiling = false; h->ev_used = 0;
+  h->gather_min_tokens = kGatherMinTokensDefault;
+  if (const char* g = getenv("FMMOE_GATHER_MIN_TOKENS")) {
+    char* end = nullptr;
+    const long long v = strtoll(g, &end, 10);
+    if (end != g && v >= 0) h->gather_min_tokens = v;
+  }
+  h->wait_budget_ns = 2000000000ull;
   h->pipe_ready = false; h->pipe_next = 0; h->ticket_next = 0; h->side_ready = false;
   { const char* dbg = getenv("FMMOE_DEBUG_SYNC"); h->debug_sync = dbg && dbg[0] == '1'; h->debug_seq = 0; }
   if (cudaMalloc(&h->d_status, 256) != cudaSuccess || cudaMemset(h->d_status, 0, 256) != cudaSuccess ||
@@ -176,6 +183,11 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
       qres == cudaDriverEntryPointSuccess)
     h->encode_tiled = fn;
+  if (prune_prepare(h) != FMMOE_OK) {
+    cudaFree(h->d_status); cudaFreeHost(h->h_status);
+    delete h;
+    return FMMOE_ERR_CUDA;
+  }
   *out = h;
   return FMMOE_OK;
 }
@@ -256,7 +268,7 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   const RoutePtrs r = bind_route(pl, ws, route);
   // the router clears the scheduler words and (atomic mode) the fp32 accumulator it owns rows of
   // bf16 at small batch: the permutation's scatter pass also writes the expert-grouped copy of x
-  const bool copy_rows = d->dtype == FMMOE_BF16 && !gather_rows_in_gemm(T);
+  const bool copy_rows = d->dtype == FMMOE_BF16 && !gather_rows_in_gemm(h, T);
   st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, det ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s,
                  copy_rows ? ws + pl.xp_off : nullptr);
   if (st != FMMOE_OK) return st;
@@ -276,7 +288,7 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   fa.ysh = det ? reinterpret_cast<float*>(ws + pl.ysh_off) : nullptr;
   fa.deterministic = det; fa.d_status = h->d_status;
   if (d->dtype == FMMOE_BF16) {
-    fa.gather_in_gemm = gather_rows_in_gemm(T) ? 1 : 0;
+    fa.gather_in_gemm = gather_rows_in_gemm(h, T) ? 1 : 0;
     st = launch_ffn_tc(h, fa, s);
   } else {
     st = launch_ffn_f32(h, fa, s);

@@ -20,6 +20,10 @@ struct fmmoe_handle {
   int64_t launches;     // kernels launched through this handle
   void* encode_tiled;   // cuTensorMapEncodeTiled entry point
   bool tc_attr_set;     // dynamic shared memory opt-in done for the tensor-core kernels
+  bool route_attr_set;  // ... for the bf16 router
+  uint32_t route_f32_attr_mask;   // ... for the fp32 router instantiations (bit = logits per lane)
+  int64_t gather_min_tokens;      // from this many tokens on GEMM-1 gathers the routed rows of x itself
+  uint64_t wait_budget_ns;        // time budget of every bounded device-side wait
   // optional kernel timeline
   bool profiling;
   bool debug_sync;      // FMMOE_DEBUG_SYNC=1: synchronise after every kernel and report the first CUDA error on stderr
@@ -190,7 +194,10 @@ struct FfnArgs {   // both paths
 };
 // Large batches: skip the expert-ordered copy of x and let GEMM-1's loader warps gather the rows.
 // Small batches are bound by the weight stream, where the copy + plain TMA boxes are faster.
-static inline bool gather_rows_in_gemm(int64_t T) { return T >= 12288; }
+// The threshold is a property of the handle (default 12,288 tokens; FMMOE_GATHER_MIN_TOKENS, read once
+// in fmmoe_create, overrides it so that either path can be exercised at any size).
+constexpr int64_t kGatherMinTokensDefault = 12288;
+static inline bool gather_rows_in_gemm(const fmmoe_handle* h, int64_t T) { return T >= h->gather_min_tokens; }
 fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05
 fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);   // fp32 FMA
 
@@ -199,6 +206,9 @@ struct FinalizeArgs {
   const float* acc; const float* y; const float* ysh; const int32_t* inv_row; const float* topk_w;
 };
 fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_t s);
+
+// start-up work of the pruning pass (module load, scratch address, shared-memory opt-in); device current
+fmmoe_status prune_prepare(fmmoe_handle* h);
 
 // fmmoe_prune_visual in two phases (bit 0: ranks, scores, selection on s_select; bit 1: rows on s_rows)
 fmmoe_status prune_visual_phases(fmmoe_handle* h, const fmmoe_prune_params* p, const float* probs, int32_t n_experts,

@@ -84,7 +84,12 @@ __global__ void __launch_bounds__(1024) vis_index_kernel(const PruneDev a, const
     if (tid == 0) s_running = running + s_warp[31];
     __syncthreads();
   }
-  if (tid == 0 && s_running != sq.n_vis[b]) atomicCAS(a.status, 0, DEV_INTERNAL);
+  // A mask with fewer set bytes than the host's count leaves the tail of this sequence's list unwritten;
+  // the scoring and merge kernels index probs and x with these entries, so they must hold a token of the
+  // sequence whatever the mask says (the mismatch itself is reported through the status word).
+  const int found = s_running;
+  for (int i = found + tid; i < sq.n_vis[b]; i += 1024) a.vis_list[lo + i] = (int32_t)lo;
+  if (tid == 0 && found != sq.n_vis[b]) atomicCAS(a.status, 0, DEV_INTERNAL);
 }
 
 // ------------------------------------------------------------------ window scores
@@ -160,9 +165,13 @@ __global__ void __launch_bounds__(256) window_score_kernel(const PruneDev a, con
   while (b + 1 < sq.n_seq && gw >= sq.win_off[b + 1]) ++b;
   const int i = gw - sq.win_off[b];
   int32_t members[MAXW];
+  const long long s_lo = sq.seq_off[b], s_hi = sq.seq_off[b + 1];
 #pragma unroll
-  for (int k = 0; k < MAXW; ++k)
-    members[k] = k < a.W ? a.vis_list[sq.seq_off[b] + (long long)i * a.W + k] : 0;
+  for (int k = 0; k < MAXW; ++k) {
+    long long tkn = k < a.W ? a.vis_list[s_lo + (long long)i * a.W + k] : s_lo;
+    if (tkn < s_lo || tkn >= s_hi) tkn = s_lo;   // only with a mask that contradicts the host's count (status word set)
+    members[k] = (int32_t)tkn;
+  }
   switch (a.W) {
     case 2: score_window<2>(a, members, lane, a.sim + gw, a.asum + gw); break;
     case 3: score_window<3>(a, members, lane, a.sim + gw, a.asum + gw); break;
@@ -426,20 +435,33 @@ __global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const Pr
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const T* X = static_cast<const T*>(a.x);
   T* O = static_cast<T*>(a.x_out) + row * a.H;
+  int b = 0;
+  while (b + 1 < sq.n_seq && row >= sq.out_off[b + 1]) ++b;
   const long long t0 = a.keep_idx_ws[row];
   const int kd = a.kind_ws[row];
+  if (t0 < sq.seq_off[b] || t0 >= sq.seq_off[b + 1]) {
+    // a slot the selection pass did not fill: only possible when the mask contradicts the host's vision
+    // count (reported through the status word).  Never index x with it.
+    uint4* dst = reinterpret_cast<uint4*>(O);
+    for (int i = tid; i < a.H / N; i += 256) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
   if (kd != 2) {
     const uint4* src = reinterpret_cast<const uint4*>(X + t0 * a.H);
     uint4* dst = reinterpret_cast<uint4*>(O);
     for (int i = tid; i < a.H / N; i += 256) dst[i] = src[i];
     return;
   }
-  int b = 0;
-  while (b + 1 < sq.n_seq && row >= sq.out_off[b + 1]) ++b;
-  const int v0 = a.vrank[t0];
+  int v0 = a.vrank[t0];
+  if (v0 < 0 || v0 + a.W > sq.n_vis[b]) v0 = 0;   // inconsistent mask / count (status word set): stay inside the list
+  const long long s_lo = sq.seq_off[b], s_hi = sq.seq_off[b + 1];
   long long mem[MAXW];
 #pragma unroll
-  for (int k = 0; k < MAXW; ++k) mem[k] = k < a.W ? a.vis_list[sq.seq_off[b] + v0 + k] : 0;
+  for (int k = 0; k < MAXW; ++k) {
+    long long tkn = k < a.W ? a.vis_list[s_lo + v0 + k] : s_lo;
+    if (tkn < s_lo || tkn >= s_hi) tkn = s_lo;
+    mem[k] = tkn;
+  }
   const float invW = 1.f / (float)a.W;
   // pass 1: squared norms of the members and of the mean
   float part[MAXW + 1];
@@ -607,8 +629,7 @@ fmmoe_status fmmoe::prune_visual_phases(fmmoe_handle* h, const fmmoe_prune_param
   a.x_out = x_out; a.is_visual_out = is_visual_out; a.keep_idx = keep_idx; a.kind = kind;
   a.status = h->d_status;
 
-  if (sel_smem > 48 * 1024)
-    FMMOE_CUDA_TRY(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_smem));
+  // select_kernel's dynamic shared-memory opt-in was raised to the device's maximum once, in fmmoe_create
 
   int win_base = 0;
   for (int b0 = 0; b0 < n_seq; b0 += MAXS) {
@@ -716,6 +737,26 @@ void* static_scratch_for(int device) {
 }
 }  // namespace
 
+// Called by fmmoe_create with the handle's device current.  Everything the pruning pass would
+// otherwise do lazily on its first call happens here, at start-up, while the process can still
+// obtain device memory: the module that holds the pruning kernels and the scratch array is loaded
+// (under lazy module loading that is when the array and the kernel code are placed in device
+// memory), the array's device address is looked up and cached, and select_kernel's dynamic
+// shared-memory limit is raised once to the device's maximum, so that no later call has to.
+fmmoe_status fmmoe::prune_prepare(fmmoe_handle* h) {
+  cudaFuncAttributes fa;
+  FMMOE_CUDA_TRY(cudaFuncGetAttributes(&fa, vis_index_kernel));
+  FMMOE_CUDA_TRY(cudaFuncGetAttributes(&fa, window_score_kernel));
+  FMMOE_CUDA_TRY(cudaFuncGetAttributes(&fa, select_kernel));
+  FMMOE_CUDA_TRY(cudaFuncGetAttributes(&fa, compact_kernel<__nv_bfloat16>));
+  FMMOE_CUDA_TRY(cudaFuncGetAttributes(&fa, compact_kernel<float>));
+  FMMOE_CUDA_TRY(cudaFuncGetAttributes(&fa, select_kernel));
+  FMMOE_CUDA_TRY(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      h->max_smem_optin - (int)fa.sharedSizeBytes));
+  if (!static_scratch_for(h->device)) return FMMOE_ERR_CUDA;
+  return FMMOE_OK;
+}
+
 extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visual_static(
     fmmoe_handle* h, const fmmoe_prune_params* p, const float* probs, int32_t n_experts, const float* attn,
     const void* x, int32_t dtype, int32_t hidden, const uint8_t* is_visual, const int64_t* seq_off,
@@ -733,9 +774,11 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_prune_visua
   if (cur != h->device) return FMMOE_ERR_INVALID_ARG;   // the handle's device must be current
   void* scratch = static_scratch_for(cur);
   if (!scratch) return FMMOE_ERR_CUDA;
-  // Nothing in the scratch has to start at zero: every word a kernel of this pass reads was
-  // written earlier in the same pass (vision ranks and lists, window scores, actions, the
-  // compaction map), so the previous call's leftovers are never observed.
+  // Nothing in the scratch has to start at zero: a pass writes the vision ranks and lists, the
+  // window scores and the compaction map before it reads them.  The one exception is a call
+  // whose mask contradicts its n_vis: slots the pass then leaves unwritten hold the previous
+  // call's values; the kernels range-check every index they take from the scratch, and the
+  // mismatch is reported through the status word.
   return fmmoe_prune_visual(h, p, probs, n_experts, attn, x, dtype, hidden, is_visual, seq_off, n_vis, n_retain,
                             n_seq, x_out, is_visual_out, keep_idx, kind, out_seq_off, scratch,
                             (size_t)FMMOE_STATIC_PRUNE_SCRATCH_BYTES, cuda_stream);

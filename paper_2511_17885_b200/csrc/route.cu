@@ -553,7 +553,11 @@ static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s)
   CUtensorMap mx, mw;
   if (!route_map(h, &mx, d.x, (uint64_t)d.T, (uint64_t)d.H, RT_BM)) return FMMOE_ERR_CUDA;
   if (!route_map(h, &mw, d.w, (uint64_t)d.E, (uint64_t)d.H, (uint32_t)d.e_pad)) return FMMOE_ERR_CUDA;
-  FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  if (!h->route_attr_set) {   // once per handle: the largest size any shape can ask for
+    FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->max_smem_optin));
+    h->route_attr_set = true;
+  }
+  if (smem > (size_t)h->max_smem_optin) return FMMOE_ERR_UNSUPPORTED;
   const int tiles = (int)((d.T + RT_BM - 1) / RT_BM);
   {
     ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
@@ -569,7 +573,10 @@ static fmmoe_status launch_nt(fmmoe_handle* h, const RouteDev& d, int grid, cuda
   const int e_pad = NT * 32;
   const size_t tail = (size_t)R_BM * (e_pad + 1) * 4 + (size_t)e_pad * 4;
   const size_t smem = (size_t)(R_BM + e_pad) * 33 * 4 + tail;
-  FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_f32_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  if (!(h->route_f32_attr_mask & (1u << NT))) {
+    FMMOE_CUDA_TRY(cudaFuncSetAttribute(route_f32_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    h->route_f32_attr_mask |= 1u << NT;
+  }
   {
     ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
     FMMOE_CUDA_TRY(launch_pdl(route_f32_kernel<NT>, dim3(grid), dim3(R_THREADS), smem, s, 1, d));

@@ -293,3 +293,56 @@ def test_host_tickets_survive_the_ring_wrapping_around():
     assert torch.equal(dst, src.cpu())
     with pytest.raises(B.FmmoeError):
         hd.fmmoe_host_wait(tickets[-1] + 1)
+
+
+def _rows_per_expert_case(counts, n_text_extra, H=128, I_=192, seed=41):
+    """Tokens whose first choice is fixed by construction, so that expert e receives exactly counts[e] first-choice
+    rows: vision tokens (K_v = 1) carry their whole weight on that expert.  `n_text_extra` text tokens (K = 2) all
+    take the last two experts, which therefore hold several M-tiles."""
+    r = np.random.default_rng(seed)
+    E = len(counts) + 2
+    assign = np.concatenate([np.full(c, e) for e, c in enumerate(counts)]).astype(np.int64)
+    r.shuffle(assign)
+    T = assign.size + n_text_extra
+    x = 0.25 * r.standard_normal((T, H))
+    mask = np.ones(T, np.uint8)
+    mask[assign.size:] = 0
+    w = random_layer(r, "bf16", H, E, I_, 0, 0)
+    router = np.zeros((E, H))
+    for e in range(E):
+        router[e, e] = 1.0                      # logit of expert e = x[t, e]
+    w["router_w"] = I.round_to_storage(router, "bf16")
+    x[np.arange(assign.size), assign] = 8.0     # first choice of every vision token
+    x[assign.size:, E - 2] = 8.0                # text tokens: the two big experts
+    x[assign.size:, E - 1] = 6.0
+    return I.round_to_storage(x, "bf16"), mask, w, E
+
+
+@pytest.mark.parametrize("gather_min", ["0", None])
+def test_rows_per_expert_boundaries_on_both_gemm1_row_paths(gather_min, monkeypatch):
+    """Experts holding 0, 1, 16, 17, 64, 65, 128 and 129 rows (and two with several hundred), EVERY output row
+    against the oracle, on both ways GEMM-1 obtains its routed rows: the expert-ordered copy written by the
+    scatter pass (default at this size) and the in-GEMM gather by token (forced through the handle's threshold,
+    which is otherwise only reached from 12,288 tokens on)."""
+    counts = [0, 1, 16, 17, 64, 65, 128, 129]
+    x, mask, w, E = _rows_per_expert_case(counts, n_text_extra=300)
+    if gather_min is not None:
+        monkeypatch.setenv("FMMOE_GATHER_MIN_TOKENS", gather_min)
+    h = B.Handle(0)                                  # the threshold is read once, when the handle is created
+    monkeypatch.delenv("FMMOE_GATHER_MIN_TOKENS", raising=False)
+    T, H = x.shape
+    I_ = w["w_gate"].shape[1]
+    desc = B.make_desc(H, E, I_, 0, 0, 2, 1, torch.bfloat16)
+    wd = upload_weights(w, "bf16"); ws = B.make_weights(wd)
+    route = {"logits": torch.empty(T, E, dtype=torch.float32, device="cuda"),
+             "topk_idx": torch.empty(T, 2, dtype=torch.int32, device="cuda"),
+             "expert_off": torch.empty(E + 1, dtype=torch.int32, device="cuda")}
+    for flags in (B.FLAG_REDUCE_ON, B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC):
+        out = h.fmmoe_moe_forward(desc, ws, dev(x, torch.bfloat16), dev(mask), flags, route=route)
+        h.check_status()
+        got_counts = np.diff(host(route["expert_off"]))
+        assert got_counts[:len(counts)].tolist() == counts and got_counts[-1] == 300 and got_counts[-2] == 300
+        ref = O.moe_forward(x, mask, w, 2, 1, True, logits32=host(route["logits"]))
+        assert np.array_equal(host(route["topk_idx"]), ref["topk_idx"])
+        assert row_rel_err(host(out), ref["out"]) < 2e-2
+    h.close()

@@ -129,3 +129,38 @@ def test_prune_c0_and_c3_keep_sets():
     assert B.fmmoe_prune_kept_count(3328, 2496, p)[0] == 2500
     assert B.fmmoe_prune_kept_count(3328, 1664, B.prune_params(5, 0.05))[0] == 1666
     assert B.fmmoe_prune_kept_count(3328, 832, B.prune_params(5, 0.1))[0] == 836
+
+
+@pytest.mark.parametrize("static", [False, True])
+def test_mask_one_bit_short_of_n_vis_is_reported_not_followed(static):
+    """The host says a sequence holds n_vis vision tokens, the mask sets one byte fewer.  The pass must end with
+    FMMOE_ERR_INTERNAL from the status word - and must not index probs or x with list entries it never wrote,
+    whatever the scratch held before (here: the leftovers of a larger earlier call, or a poisoned workspace).
+    The next ordinary call on the same handle is unaffected."""
+    h = handle()
+    r = np.random.default_rng(77)
+    H, E, W = 128, 16, 3
+    p = B.prune_params(W, 0.1)
+    # an earlier, longer call leaves large token indices behind in the shared scratch
+    check_prune("bf16", [3000], H, E, W, 0.5, 0.1, 1.0, False, seed=78)
+    L = 400
+    mask = np.zeros(L, np.uint8); mask[:301] = 1
+    n_vis_true = 301
+    x = dev(I.round_to_storage(r.standard_normal((L, H)), "bf16"), torch.bfloat16)
+    probs = dev(softmax_rows(r, L, E))
+    bad = mask.copy(); bad[300] = 0                         # one set byte fewer than the count the host passes
+    kept, _, _ = B.fmmoe_prune_kept_count(n_vis_true, 150, p)
+    t_out = L - n_vis_true + kept
+    if static:
+        x_out = torch.zeros((t_out, H), dtype=torch.bfloat16, device="cuda")
+        h.fmmoe_prune_visual_static(p, probs, None, x, dev(bad), [0, L], [n_vis_true], [150], x_out)
+    else:
+        h._ws = None                                        # a fresh workspace, poisoned with out-of-range indices
+        ws = h.workspace(int(B.lib().fmmoe_prune_workspace_bytes(L, 1)))
+        ws.fill_(0x7f)                                      # every int32 word reads 0x7f7f7f7f
+        out = h.fmmoe_prune_visual(p, probs, None, x, dev(bad), [0, L], [n_vis_true], [150])
+        assert out["x_out"].shape[0] == t_out
+    assert h.get_status() == 6                              # FMMOE_ERR_INTERNAL, read and cleared
+    torch.cuda.synchronize()                                # no fault: the context is still usable
+    # the consistent call right after it passes parity
+    check_prune("bf16", [L], H, E, W, 0.5, 0.1, 1.0, False, seed=79)

@@ -82,14 +82,20 @@ def test_scores_hand_example():
 def test_gamma_hat_closed_form_and_printed_table():
     rows = [tuple(map(float, l.split())) for l in open(os.path.join(GOLD, "gamma_hat_table.txt"))
             if l.strip() and not l.startswith("#")]
-    grid = [0.025, 0.05, 0.1, 0.15]
+    assert [r for r, _, _ in rows] == [0.75, 0.5, 0.25]
+    closed = []
     for r, beta_p, gh_p in rows:
         beta = O.stage_beta(r, 3)
         assert abs(round(beta, 2) - beta_p) < 1e-9                 # printed 0.91 / 0.79 / 0.63
-        gh = O.gamma_hat(beta, 5)
-        # printed value = closed form floored onto the experiment grid (to grid resolution)
-        floored = max(g for g in grid if g <= gh + 0.004)
-        assert abs(floored - gh_p) < 1e-12, (r, gh, floored, gh_p)
+        closed.append(O.gamma_hat(beta, 5))
+    # the three printed bounds, one by one (W = 5, three stages):
+    #   75 %: closed form 0.0252 -> printed 0.025 (the closed form to three decimals)
+    assert abs(closed[0] - 0.0252) < 5e-5 and rows[0][2] == 0.025 and abs(closed[0] - rows[0][2]) < 5e-4
+    #   25 %: closed form 0.1469 -> printed 0.15 (to two decimals)
+    assert abs(closed[2] - 0.1469) < 5e-5 and rows[2][2] == 0.15 and round(closed[2], 2) == rows[2][2]
+    #   50 %: closed form 0.0650, the paper prints 0.05: its own inconsistency (0.05 is the merge rate the
+    #   experiments use at 50 %, a value below the bound); recorded here, not reconciled
+    assert abs(closed[1] - 0.0650) < 5e-5 and rows[1][2] == 0.05 and closed[1] > rows[1][2]
     # the identity the bound is derived from: merging alone removes all eps tokens
     for n_v, eta, W in [(1000, 800, 5), (2304, 1152, 3), (3328, 2496, 5)]:
         gh = O.gamma_hat(eta / n_v, W)

@@ -258,3 +258,28 @@ def test_appendix_c_angle_identity_with_orthonormal_experts():
 def test_moe_flops_matches_appendix_e_formula():
     B, L, H, E, Sm, K = 2, 100, 64, 16, 32, 4
     assert O.moe_flops(B * L, B * L * K, H, E, Sm) == 2 * B * L * H * E + 6 * B * L * H * Sm * K
+
+
+def test_moe_flops_counted_multiply_adds_with_shared_experts():
+    """Every term of moe_flops against a literal count of the multiply-adds of Eq. 1 and Eq. 4 on a tiny layer:
+    a matrix-vector product of an [out, in] matrix is out*in multiply-adds = 2*out*in FLOPs; an expert is three of
+    them (gate, up, down); a token runs its selected routed experts and every shared expert."""
+    T, H, E, Sm, Ns, Ss = 7, 6, 5, 4, 2, 3
+    k_t = [3, 1, 1, 3, 1, 3, 1]                      # experts per token (K = 3 for text, K_v = 1 for vision)
+    flops = 0
+    for t in range(T):
+        for e in range(E):                           # Eq. 1: one dot product of length H per expert
+            for h in range(H):
+                flops += 2
+        for j in range(k_t[t]):                      # Eq. 4, routed: gate and up [Sm, H], down [H, Sm]
+            for mat_out, mat_in in ((Sm, H), (Sm, H), (H, Sm)):
+                for o in range(mat_out):
+                    for i in range(mat_in):
+                        flops += 2
+        for s in range(Ns):                          # Eq. 4, shared: every token, every shared expert
+            for mat_out, mat_in in ((Ss, H), (Ss, H), (H, Ss)):
+                for o in range(mat_out):
+                    for i in range(mat_in):
+                        flops += 2
+    assert O.moe_flops(T, sum(k_t), H, E, Sm, Ns, Ss) == flops
+    assert O.moe_flops(T, sum(k_t), H, E, Sm) == flops - Ns * T * 6 * H * Ss      # the shared term on its own
