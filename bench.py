@@ -1,18 +1,31 @@
 #!/usr/bin/env python
 """Benchmark of the FastMMoE MoE-layer hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload all|C0|C1|C2|C2x4|C3|C4] [--impl reference]
 
 One "step" = one pass of the whole hot path over one batch of synthetic tokens:
 router + top-k + gates, permute-by-expert, grouped SwiGLU expert GEMMs + shared
-experts, weighted combine (fmmoe_moe_forward), then routing-aware pruning of the layer
-output with that layer's routing probabilities (fmmoe_prune_visual).
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+experts, weighted combine, then routing-aware pruning of the layer output with that
+layer's routing probabilities (fmmoe_moe_forward_prune); for the 24-layer stack a step
+is the whole stack (fmmoe_stack_forward).
+
+The default (`--workload all`) prints ONE JSON line whose top-level fields are the
+largest single-layer workload (the batch of four Qwen3-MoE-style sequences, 14,336
+tokens) and whose `configs` object holds one record per other workload (C0, C1, C2,
+C3, C4), each with its own timing, clocks, roofline and end-to-end figure.
+
+Timing: a block is exactly K steps between two CUDA events, with a barrier and a
+device synchronisation on both sides.  Whatever K is, blocks are repeated until the
+workload has at least `--min-seconds` of timed GPU work; the reported step time is the
+MEDIAN block (the best block and the SM clock of every block are given beside it).
+`--impl reference` times the CPU oracle instead.
 """
 from __future__ import annotations
 
 import argparse
+import gc
 import json
+import math
 import os
 import sys
 import threading
@@ -25,11 +38,15 @@ import numpy as np  # noqa: E402
 
 METRIC = "MoE-layer prefill tokens/s"
 UNIT = "tokens/s"
-WORKLOADS = ("C0", "C1", "C2", "C2x4", "C3", "C4")
+LAYER_WORKLOADS = ("C0", "C1", "C2", "C2x4", "C3")
+WORKLOADS = ("all",) + LAYER_WORKLOADS + ("C4",)
+HEADLINE = "C2x4"
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # the nominal peaks the metric names (8 TB/s, dense bf16)
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
-# ncu captures summarised under profiles/ (null until a capture for that workload exists).
-NCU_TRAFFIC_BYTES = {"C1": {"gemm1": 870.6e6, "gemm2": 502.8e6}}   # profiles/kernels_c1_full_set.md
+# DRAM bytes (read + written) one launch of a kernel moved under the profiler, per workload.
+# Each figure comes from one capture of that kernel on that workload; an entry is removed (null in
+# the output) when its kernel changes after the capture.
+NCU_TRAFFIC_BYTES = {}
 
 
 def load_peaks():
@@ -61,7 +78,9 @@ def describe(name, cfg, prune):
                         f"(W={prune.window}, gamma={prune.gamma}, attention-free score)",
             "tokens_per_step": cfg.n_tokens,
             "l2": "inputs larger than L2: every step streams the layer's expert weights "
-                  f"({weight_bytes(cfg) / 1e6:.0f} MB) from HBM"}
+                  f"({weight_bytes(cfg) / 1e6:.0f} MB) from HBM" if weight_bytes(cfg) > 126e6 else
+                  f"the layer's weights ({weight_bytes(cfg) / 1e6:.1f} MB) fit in L2: a launch-latency workload, "
+                  "timed with the L2 warm"}
 
 
 def weight_bytes(cfg):
@@ -71,9 +90,10 @@ def weight_bytes(cfg):
 
 
 # ------------------------------------------------------------------ algorithmic work per launch
-def kernel_work(cfg, kernel, P, touched, t_out=None):
+def kernel_work(cfg, kernel, P, touched, prune_rows=None):
     """(bytes, flops) one launch of `kernel` must move / compute for this workload.
-    P = routed pairs, touched = experts with at least one row."""
+    P = routed pairs, touched = experts with at least one row, prune_rows = (rows read, rows written) of the
+    compaction pass."""
     e = 2 if cfg.dtype == "bf16" else 4
     T, H, E, I_, Ns, Is, K = cfg.n_tokens, cfg.hidden, cfg.n_experts, cfg.inter, cfg.n_shared, cfg.shared_inter, cfg.top_k
     if kernel == "gemm1":
@@ -85,11 +105,17 @@ def kernel_work(cfg, kernel, P, touched, t_out=None):
     elif kernel == "route":
         b = T * H * e + E * H * e + T * K * 8 + T * E * 4
         f = 2 * T * H * E
-    elif kernel == "gather":
-        b = T * H * e + P * H * e
+    elif kernel == "permute":
+        b = T * K * 4 + 3 * P * 4
         f = 0
     elif kernel == "finalize":
         b = T * H * 4 + T * H * e
+        f = 0
+    elif kernel == "prune_score":
+        b = cfg.batch * cfg.n_vis * E * 4
+        f = 0
+    elif kernel == "prune_compact" and prune_rows is not None:
+        b = (prune_rows[0] + prune_rows[1]) * H * e
         f = 0
     else:
         b, f = 0, 0
@@ -98,11 +124,11 @@ def kernel_work(cfg, kernel, P, touched, t_out=None):
 
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
-    """Samples SM clock and clock-event reasons while the timed region runs (read-only NVML)."""
+    """Samples SM clock, board power and clock-event reasons while the timed region runs (read-only NVML)."""
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index):
-        self.samples, self.reasons, self.max_mhz, self.ok = [], set(), None, False
+        self.samples, self.times, self.reasons, self.max_mhz, self.ok = [], [], set(), None, False
         self.power_w = []
         self._stop = threading.Event()
         try:
@@ -124,7 +150,9 @@ class ClockSampler:
         if not self.ok:
             return
         try:
-            self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.dev, self.nv.NVML_CLOCK_SM)))
+            mhz = int(self.nv.nvmlDeviceGetClockInfo(self.dev, self.nv.NVML_CLOCK_SM))
+            self.samples.append(mhz)
+            self.times.append(time.perf_counter())
             try:
                 self.power_w.append(self.nv.nvmlDeviceGetPowerUsage(self.dev) / 1000.0)
             except Exception:
@@ -154,6 +182,10 @@ class ClockSampler:
         if self.th is not None:
             self.th.join(timeout=2)
 
+    def median_between(self, t0, t1):
+        v = [m for m, t in zip(self.samples, self.times) if t0 <= t <= t1]
+        return float(np.median(v)) if v else None
+
     def summary(self):
         return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(self.reasons), "samples": len(self.samples),
@@ -163,9 +195,8 @@ class ClockSampler:
 
 def settle_clocks(step, index, min_s=0.4, max_s=3.0):
     """Untimed load before the timed region, after the W warm-up steps: a GPU that has been idle ramps its SM
-    clock over the first tenths of a second of work, which would otherwise fall inside a short timed
-    region.  Runs `step` until the SM clock reads >= 95 % of its maximum or a power/thermal cap is active
-    (read-only NVML), for at least min_s and at most max_s seconds.  Returns the seconds spent."""
+    clock over the first tenths of a second of work.  Runs `step` until the SM clock reads >= 95 % of its
+    maximum or a power/thermal cap is active (read-only NVML), for at least min_s and at most max_s seconds."""
     import torch
     probe = ClockSampler(index)
     t0 = time.perf_counter()
@@ -184,6 +215,49 @@ def settle_clocks(step, index, min_s=0.4, max_s=3.0):
             if probe.reasons or (probe.samples and probe.samples[-1] >= 0.95 * probe.max_mhz):
                 break
     return time.perf_counter() - t0
+
+
+def timed_blocks(step, K, min_seconds, clocks, D, dev, max_blocks=400):
+    """Blocks of exactly K steps, each between two CUDA events on the current stream with a barrier and a
+    device synchronisation on both sides; repeated until min_seconds of timed GPU work has accumulated.
+    Block times are the MAX over ranks.  Returns per-block seconds and the median SM clock of each block."""
+    import torch
+    secs, mhz = [], []
+    total, n_blocks = 0.0, None
+    while True:
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        D.barrier(); torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ev0.record()
+        for _ in range(K):
+            step()
+        ev1.record()
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        D.barrier()
+        s = D.max_over_ranks(ev0.elapsed_time(ev1) * 1e-3, dev)
+        secs.append(s)
+        mhz.append(clocks.median_between(t0, t1))
+        total += s
+        if n_blocks is None:     # every rank runs the same number of blocks: decided from the first (max over ranks) time
+            n_blocks = int(min(max_blocks, max(3, math.ceil(min_seconds / max(s, 1e-6)))))
+        if len(secs) >= n_blocks:
+            break
+    return secs, mhz
+
+
+def block_stats(secs, mhz, K):
+    per_step = np.array(secs) / K
+    med = float(np.median(per_step))
+    m = [x for x in mhz if x is not None]
+    med_mhz = float(np.median(m)) if m else None
+    return {"blocks": len(secs), "steps_per_block": K, "gpu_seconds_timed": float(np.sum(secs)),
+            "ms_per_step_median": med * 1e3, "ms_per_step_best": float(per_step.min()) * 1e3,
+            "ms_per_step_p90": float(np.percentile(per_step, 90)) * 1e3,
+            "sm_mhz_median_of_blocks": med_mhz,
+            "sm_mhz_min_max_of_blocks": [float(min(m)), float(max(m))] if m else None,
+            # step time x SM clock: comparable between runs that sat at different power-capped clocks
+            "ms_x_mhz": med * 1e3 * med_mhz if med_mhz else None}, med
 
 
 # ------------------------------------------------------------------ oracle timing
@@ -214,8 +288,18 @@ def oracle_step(cfg, prune, xs, ms, so, nvs, w):
                    prune.alpha, prune.gamma)
 
 
-def time_oracle(name, cfg, prune, frac, steps, warmup):
-    import torch
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        nt = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if nt:
+            return int(max(nt))
+    except Exception:
+        pass
+    return 1
+
+
+def time_oracle(name, cfg, prune, frac, steps, warmup, one_thread_frac=None):
     xs, ms, so, nvs, w = oracle_sample(name, cfg, prune, frac)
     for _ in range(warmup):
         oracle_step(cfg, prune, xs, ms, so, nvs, w)
@@ -223,30 +307,42 @@ def time_oracle(name, cfg, prune, frac, steps, warmup):
     for _ in range(steps):
         oracle_step(cfg, prune, xs, ms, so, nvs, w)
     dt = time.perf_counter() - t0
-    cores = min(len(os.sched_getaffinity(0)), torch.get_num_threads() if torch.get_num_threads() > 0 else 1)
-    try:
-        from threadpoolctl import threadpool_info
-        nt = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
-        if nt:
-            cores = max(nt)
-    except Exception:
-        pass
+    threads = blas_threads()
     sample = (f"{xs.shape[0]} of {cfg.n_tokens} tokens of the workload (first {frac:.3g} of each sequence's visual "
-              f"and text tokens), route + experts + combine + pruning, fp64 numpy, {steps} pass(es)")
-    return xs.shape[0] * steps / dt, dt / max(steps, 1), int(cores), sample
+              f"and text tokens), route + experts + combine + pruning, fp64 numpy, {steps} pass(es); `cores` = BLAS "
+              f"threads used, of {len(os.sched_getaffinity(0))} host cores available")
+    one = None
+    if one_thread_frac:
+        try:
+            from threadpoolctl import threadpool_limits
+            xs1, ms1, so1, nvs1, _ = oracle_sample(name, cfg, prune, one_thread_frac)
+            with threadpool_limits(limits=1):
+                t1 = time.perf_counter()
+                oracle_step(cfg, prune, xs1, ms1, so1, nvs1, w)
+                one = xs1.shape[0] / (time.perf_counter() - t1)
+        except Exception:
+            one = None
+    return xs.shape[0] * steps / dt, dt / max(steps, 1), threads, sample, one
+
+
+def cpu_baseline_for(name, cfg, prune):
+    frac = 1.0 if cfg.n_tokens <= 4096 else 4096.0 / cfg.n_tokens
+    v, spp, cores, sample, one = time_oracle(name, cfg, prune, frac, 3, 0, one_thread_frac=frac / 8)
+    return {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "value_1_thread": one}
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", 0))
     if rank != 0:
         return 0
-    cfg, prune = workload_cfg(args.workload)
+    name = HEADLINE if args.workload == "all" else args.workload
+    cfg, prune = workload_cfg(name)
     frac = 1.0 if cfg.n_tokens <= 4096 else 4096.0 / cfg.n_tokens
-    value, spp, cores, sample = time_oracle(args.workload, cfg, prune, frac, max(args.steps, 1), args.warmup)
+    value, spp, cores, sample, _ = time_oracle(name, cfg, prune, frac, max(args.steps, 1), min(args.warmup, 1))
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": spp * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": describe(args.workload, cfg, prune),
+            "config": describe(name, cfg, prune),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -254,146 +350,159 @@ def run_reference(args):
     return 0
 
 
-# ------------------------------------------------------------------ the CUDA arm
-def run_ours(args):
+# ------------------------------------------------------------------ one layer workload on the GPU
+def roofline_of(kernel, b, f, per_launch_s, peaks, traffic):
+    t_hbm, t_tc = b / (peaks["hbm_gbs"] * 1e9), f / (peaks["tf_sustained"] * 1e12)
+    if t_hbm >= t_tc:
+        roof = {"bound": "hbm", "achieved": b / per_launch_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "peak_nominal": NOMINAL["hbm_gbs"]}
+    else:
+        roof = {"bound": "tensor", "achieved": f / per_launch_s / 1e12, "peak": peaks["tf_sustained"], "unit": "TFLOP/s",
+                "peak_nominal": NOMINAL["bf16_tflops"]}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["frac_of_nominal"] = roof["achieved"] / roof["peak_nominal"]
+    roof["traffic"] = traffic
+    roof.update({"kernel": kernel, "us_per_launch": per_launch_s * 1e6, "algorithmic_bytes": b, "algorithmic_flops": f,
+                 "peak_source": peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy)"),
+                 "tensor_tflops": f / per_launch_s / 1e12, "hbm_gbs": b / per_launch_s / 1e9})
+    return roof
+
+
+def measure_layer(name, args, D, rank, local, world, peaks, with_cpu):
     import torch
     from paper_2511_17885_b200 import binding as B
-    from paper_2511_17885_b200 import dist as D
     from paper_2511_17885_b200.workload import LayerWorkload
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
-    rank, local, world = D.init("nccl") if int(os.environ.get("WORLD_SIZE", 1)) > 1 else (0, 0, 1)
-    torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    cfg, prune = workload_cfg(args.workload)
-    peaks = load_peaks()
+    cfg, prune = workload_cfg(name)
     h = B.Handle(local)
     wl = LayerWorkload(cfg, h, device=local, prune=prune, token_seed=D.token_seed_for_rank(cfg.seed, rank))
-    K, W = args.steps, max(args.warmup, 0)
-
-    for _ in range(max(W, 1)):
+    K, W = max(args.steps, 1), max(args.warmup, 3)
+    for _ in range(W):
         wl.step()
     settle_s = settle_clocks(wl.step, local)
     h.check_status("warm-up")
     P, touched = wl.routing_stats()
 
-    # ---- device-resident timed region (no instrumentation inside)
+    # ---- device-resident timed blocks (no instrumentation inside)
     clocks = ClockSampler(local)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    D.barrier(); torch.cuda.synchronize()
     clocks.start()
     n0 = h.launch_count()
-    ev0.record()
-    for _ in range(K):
-        wl.step()
-    ev1.record()
-    clocks.sample_once()
-    torch.cuda.synchronize(); D.barrier()
-    launches = h.launch_count() - n0
+    secs, mhz = timed_blocks(wl.step, K, args.min_seconds, clocks, D, dev)
+    launches = (h.launch_count() - n0) // len(secs)
     h.check_status("timed region")
-    secs = ev0.elapsed_time(ev1) * 1e-3
-    value, tmax = D.aggregate_throughput(cfg.n_tokens * K, secs, dev)
+    stats, step_s = block_stats(secs, mhz, K)
+    value = cfg.n_tokens * world / step_s
 
-    # ---- the same K steps once more with every kernel launch bracketed by CUDA events on the
-    # launching stream: per-kernel durations for the roofline (the events cost a little, so the
-    # headline value comes from the uninstrumented region above).  This pass issues the layer and
-    # the pruning stage as two calls on one stream; the timed region above uses the single call
-    # that runs the selection kernels beside the expert GEMMs.
+    # ---- per-kernel durations: the same step with every kernel launch between two CUDA events on the
+    # launching stream (the layer and the pruning stage as two calls on one stream, so that a pair brackets
+    # one kernel).  Short kernels that can be repeated without changing their result are issued 50 times
+    # inside their pair, which amortises the launch latency a pair adds to a 10-30 us kernel.
     h.profile_reset()
-    h.profile_enable(True)
-    pv0, pv1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    pv0.record()
-    for _ in range(K):
-        wl.step(fused=False)     # one stream, so that an event pair brackets one kernel and nothing else
-    pv1.record()
+    h.profile_enable(50)
+    kp = max(3, min(K, 10))
+    for _ in range(kp):
+        wl.step(fused=False)
     torch.cuda.synchronize()
-    clocks.stop()
-    h.profile_enable(False)
+    h.profile_enable(0)
     prof = h.profile_read()
     h.check_status("instrumented region")
-    instrumented_ms = pv0.elapsed_time(pv1) / K
 
-    # ---- end-to-end region (host buffers in, host buffers out).  The K steps are K independent
-    # batches in pinned host memory; every one is uploaded, computed and downloaded (layer output and
-    # pruned rows) inside the timed region.  Three batches are in flight: the library's copy streams
-    # overlap the upload of batch i with the layer of batch i-1 and the downloads of batch i-2.
-    for i in range(min(max(W, 1), 3)):
+    # ---- end to end: host buffers in, host buffers out.  K independent batches in pinned host memory per
+    # block; every one is uploaded, computed and downloaded (layer output and pruned rows) inside the timed
+    # block, three in flight (upload of batch i beside the layer of batch i-1 and the downloads of batch i-2).
+    for i in range(3):
         wl.step_host_async(i)
     wl.drain_host()
-    D.barrier(); torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_wall0 = time.perf_counter()
-    e0.record()
-    for i in range(K):
-        wl.step_host_async(i)
-    wl.drain_host()                      # host-side wait: every result is in host memory
-    e1.record()
-    torch.cuda.synchronize(); D.barrier()
-    e2e_secs = max(e0.elapsed_time(e1) * 1e-3, time.perf_counter() - t_wall0)
-    e2e_value, _ = D.aggregate_throughput(cfg.n_tokens * K, e2e_secs, dev)
+    counter = [0]
+
+    def e2e_block_step():
+        wl.step_host_async(counter[0]); counter[0] += 1
+
+    def e2e_block(Kb):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        D.barrier(); torch.cuda.synchronize()
+        tw0 = time.perf_counter()
+        e0.record()
+        for _ in range(Kb):
+            e2e_block_step()
+        wl.drain_host()                      # host-side wait: every result is in host memory
+        e1.record()
+        torch.cuda.synchronize()
+        tw1 = time.perf_counter()
+        D.barrier()
+        return D.max_over_ranks(max(e0.elapsed_time(e1) * 1e-3, tw1 - tw0), dev), (tw0, tw1)
+
+    e_secs, e_mhz = [], []
+    first, span = e2e_block(K)
+    e_secs.append(first); e_mhz.append(clocks.median_between(*span))
+    for _ in range(int(min(200, max(2, math.ceil(args.min_seconds / max(first, 1e-6))))) - 1):
+        s, span = e2e_block(K)
+        e_secs.append(s); e_mhz.append(clocks.median_between(*span))
+    e_stats, e_step_s = block_stats(e_secs, e_mhz, K)
     h.check_status("end-to-end region")
     # the same without overlap: one batch at a time, the stream synchronised after every download
     for _ in range(2):
         wl.step_host()
     torch.cuda.synchronize()
     s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ks = max(3, min(K, 20))
     s0.record()
-    for _ in range(K):
+    for _ in range(ks):
         wl.step_host()
     s1.record()
     torch.cuda.synchronize(); D.barrier()
-    e2e_serial, _ = D.aggregate_throughput(cfg.n_tokens * K, s0.elapsed_time(s1) * 1e-3, dev)
-    h.check_status("end-to-end region (serial)")
+    e2e_serial = cfg.n_tokens * world / (D.max_over_ranks(s0.elapsed_time(s1) * 1e-3, dev) / ks)
+    h.check_status("end-to-end region (one batch at a time)")
+    clocks.stop()
 
-    # ---- roofline of the dominant kernel
+    # ---- rooflines
+    t_out = int(wl.last["x_out"].shape[0]) if wl.last is not None else 0
+    merged = wl.merged_rows() if wl.last is not None else 0
+    prune_rows = (t_out + merged * (prune.window - 1), t_out)
+    kernels = {}
+    tot_ms = max(sum(v["ms"] for v in prof.values()), 1e-12)
+    for k, v in prof.items():
+        if not v["launches"]:
+            continue
+        per_launch_s = v["ms"] * 1e-3 / v["launches"]
+        b, f = kernel_work(cfg, k, P, touched, prune_rows)
+        kernels[k] = {"us_per_launch": per_launch_s * 1e6, "launches_per_step": v["launches"] / kp,
+                      "us_per_step": v["ms"] * 1e3 / kp, "share": v["ms"] / tot_ms,
+                      "algorithmic_bytes": b, "hbm_gbs": b / per_launch_s / 1e9 if b else None,
+                      "frac_of_hbm_peak": b / per_launch_s / 1e9 / peaks["hbm_gbs"] if b else None,
+                      "tensor_tflops": f / per_launch_s / 1e12 if f else None}
     dom = max(prof, key=lambda k: prof[k]["ms"])
     per_launch_s = prof[dom]["ms"] * 1e-3 / max(prof[dom]["launches"], 1)
-    b, f = kernel_work(cfg, dom, P, touched)
-    t_hbm, t_tc = b / (peaks["hbm_gbs"] * 1e9), f / (peaks["tf_sustained"] * 1e12)
-    if t_hbm >= t_tc:
-        roof = {"bound": "hbm", "achieved": b / per_launch_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-    else:
-        roof = {"bound": "tensor", "achieved": f / per_launch_s / 1e12, "peak": peaks["tf_sustained"], "unit": "TFLOP/s"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.workload, {}).get(dom)
-    roof.update({"kernel": dom, "us_per_launch": per_launch_s * 1e6, "algorithmic_bytes": b, "algorithmic_flops": f,
-                 "peak_source": peaks["source"]})
+    b, f = kernel_work(cfg, dom, P, touched, prune_rows)
+    roof = roofline_of(dom, b, f, per_launch_s, peaks, NCU_TRAFFIC_BYTES.get(name, {}).get(dom))
     # whole step against the slower of (activated FLOPs at tensor peak, algorithmic bytes at HBM bandwidth)
-    tot_b = sum(kernel_work(cfg, k, P, touched)[0] for k in ("route", "gemm1", "gemm2")) \
-        - 2 * cfg.n_tokens * cfg.hidden * (2 if cfg.dtype == "bf16" else 4)   # X is read once, not three times
+    e = 2 if cfg.dtype == "bf16" else 4
+    tot_b = sum(kernel_work(cfg, k, P, touched)[0] for k in ("route", "gemm1", "gemm2")) - 2 * cfg.n_tokens * cfg.hidden * e
     tot_f = sum(kernel_work(cfg, k, P, touched)[1] for k in ("route", "gemm1", "gemm2"))
-    t_step = max(tot_b / (peaks["hbm_gbs"] * 1e9), tot_f / (peaks["tf_sustained"] * 1e12))
-    step_s = tmax / K
-    kernels = {k: {"us_per_step": v["ms"] * 1e3 / K, "launches_per_step": v["launches"] / K,
-                   "share": v["ms"] / max(sum(x["ms"] for x in prof.values()), 1e-12)}
-               for k, v in prof.items() if v["launches"]}
+    t_hbm, t_tc = tot_b / (peaks["hbm_gbs"] * 1e9), tot_f / (peaks["tf_sustained"] * 1e12)
+    t_step = max(t_hbm, t_tc)
+    t_step_nom = max(tot_b / (NOMINAL["hbm_gbs"] * 1e9), tot_f / (NOMINAL["bf16_tflops"] * 1e12))
 
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        frac = 1.0 if cfg.n_tokens <= 4096 else 4096.0 / cfg.n_tokens
-        v, spp, cores, sample = time_oracle(args.workload, cfg, prune, frac, 3, 0)
-        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
-
-    if rank == 0:
-        conf = describe(args.workload, cfg, prune)
-        conf.update({"routed_pairs": P, "experts_touched": touched, "parallelism": f"replicas x{world} (no collective)"})
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-                "ms_per_step": step_s * 1e3, "ms_per_step_instrumented": instrumented_ms,
-                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": cfg.dtype, "data": "synthetic", "config": conf,
-                "clocks": dict(clocks.summary(), settle_s=round(settle_s, 2)),
-                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(),
-                        "d2h_bytes_per_step": wl.d2h_bytes(), "batches_in_flight": wl.PIPE_DEPTH,
-                        "value_one_batch_at_a_time": e2e_serial},
-                "gpu_launches": int(launches),
-                "roofline": roof,
-                "step_roofline": {"frac": t_step / step_s, "t_bound_us": t_step * 1e6, "algorithmic_bytes": tot_b,
-                                  "activated_flops": tot_f, "peak_source": peaks["source"]},
-                "kernels": kernels,
-                "cpu_baseline": cpu}
-        print(json.dumps(line))
-    D.shutdown()
-    return 0
+    conf = describe(name, cfg, prune)
+    conf.update({"routed_pairs": P, "experts_touched": touched, "parallelism": f"replicas x{world} (no collective)"})
+    rec = {"value": value, "unit": UNIT, "ms_per_step": step_s * 1e3, "timing": stats, "dtype": cfg.dtype,
+           "config": conf,
+           "clocks": dict(clocks.summary(), settle_s=round(settle_s, 2)),
+           "e2e": {"value": cfg.n_tokens * world / e_step_s, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(),
+                   "d2h_bytes_per_step": wl.d2h_bytes(), "batches_in_flight": wl.PIPE_DEPTH, "timing": e_stats,
+                   "value_one_batch_at_a_time": e2e_serial},
+           "gpu_launches": int(launches * K),
+           "roofline": roof,
+           "step_roofline": {"frac": t_step / step_s, "frac_of_nominal": t_step_nom / step_s,
+                             "bound": "hbm" if t_hbm >= t_tc else "tensor", "t_bound_us": t_step * 1e6,
+                             "algorithmic_bytes": tot_b, "activated_flops": tot_f, "peak_source": peaks["source"]},
+           "kernels": kernels}
+    if with_cpu:
+        rec["cpu_baseline"] = cpu_baseline_for(name, cfg, prune)
+    del wl
+    h.close()
+    gc.collect(); torch.cuda.empty_cache()
+    return rec
 
 
 # ------------------------------------------------------------------ the 24-layer stack (C4)
@@ -420,7 +529,6 @@ def stack_flops(lc, shapes):
 
 def oracle_stack_sample(sc, n_layers_sample=2, n_tok=512):
     """Bounded CPU sample for the stack: the first n_tok tokens of sequence 0 through the first layers."""
-    import torch
     from paper_2511_17885_b200 import inputs as I
     from oracle import fmmoe_oracle as O
     lc = sc.layer
@@ -440,41 +548,27 @@ def oracle_stack_sample(sc, n_layers_sample=2, n_tok=512):
 
 
 def stack_cpu_baseline(sc, n_layers):
-    import torch
     n_tok, nl, dt = oracle_stack_sample(sc)
     # tokens/s through the whole stack, extrapolated from nl layers to n_layers
     value = n_tok / (dt * n_layers / nl)
-    cores = len(os.sched_getaffinity(0))
-    try:
-        from threadpoolctl import threadpool_info
-        nt = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
-        if nt:
-            cores = max(nt)
-    except Exception:
-        pass
     sample = (f"{n_tok} tokens of sequence 0 through the first {nl} of {n_layers} layers (router, experts, combine, "
-              f"residual; fp64 numpy; no pruning stage falls in these layers), time scaled by {n_layers}/{nl}")
-    return {"value": value, "unit": UNIT, "cores": int(cores), "kind": "oracle", "sample": sample}
+              f"residual; fp64 numpy; no pruning stage falls in these layers), time scaled by {n_layers}/{nl}; "
+              f"`cores` = BLAS threads used, of {len(os.sched_getaffinity(0))} host cores available")
+    return {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample}
 
 
-def run_stack(args):
+def measure_stack(args, D, rank, local, world, peaks, with_cpu):
     import torch
     from paper_2511_17885_b200 import binding as B
-    from paper_2511_17885_b200 import dist as D
     from paper_2511_17885_b200 import inputs as I
     from paper_2511_17885_b200.workload import StackWorkload
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
-    rank, local, world = D.init("nccl") if int(os.environ.get("WORLD_SIZE", 1)) > 1 else (0, 0, 1)
-    torch.cuda.set_device(local)
     dev = f"cuda:{local}"
     sc = I.C4
     n_layers = args.layers or sc.n_layers
-    peaks = load_peaks()
     h = B.Handle(local)
     wl = StackWorkload(sc, h, device=local, token_seed=D.token_seed_for_rank(sc.layer.seed, rank), n_layers=n_layers)
-    K, W = args.steps, max(args.warmup, 3)
-    for _ in range(W):
+    K, W = max(1, min(args.steps, 10)), max(args.warmup, 3)      # a stack step is 24 layers: at most 10 per block
+    for _ in range(min(W, 5)):
         wl.step()
     settle_s = settle_clocks(wl.step, local, min_s=0.2)
     h.check_status("warm-up")
@@ -482,54 +576,53 @@ def run_stack(args):
         raise SystemExit("bench.py: the stack's output is not finite")
     out_std = float(wl.x_out.float().std())
     clocks = ClockSampler(local)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    D.barrier(); torch.cuda.synchronize()
     clocks.start()
     n0 = h.launch_count()
-    ev0.record()
-    for _ in range(K):
-        wl.step()
-    ev1.record()
-    clocks.sample_once()
-    torch.cuda.synchronize(); D.barrier()
-    launches = h.launch_count() - n0
+    secs, mhz = timed_blocks(wl.step, K, args.min_seconds, clocks, D, dev)
+    launches = (h.launch_count() - n0) // len(secs)
     h.check_status("timed region")
-    value, tmax = D.aggregate_throughput(wl.n_tokens * K, ev0.elapsed_time(ev1) * 1e-3, dev)
+    stats, step_s = block_stats(secs, mhz, K)
+    value = wl.n_tokens * world / step_s
     # instrumented pass
-    h.profile_reset(); h.profile_enable(True)
-    kp = min(K, 3)
+    h.profile_reset(); h.profile_enable(1)
+    kp = 2
     for _ in range(kp):
         wl.step()
     torch.cuda.synchronize()
-    clocks.stop()
-    h.profile_enable(False)
+    h.profile_enable(0)
     prof = h.profile_read()
-    # end to end: K independent batches from pinned host memory, two in flight (upload of batch i beside the
-    # stack of batch i-1 and the download of batch i-2); then the same one batch at a time
+    # end to end: independent batches from pinned host memory, two in flight; then one batch at a time
     for i in range(2):
         wl.step_host_async(i)
     wl.drain_host()
+    ke = max(4, K)
     D.barrier(); torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_wall0 = time.perf_counter()
     e0.record()
-    for i in range(K):
-        wl.step_host_async(i)
+    n_e2e = 0
+    while True:
+        for i in range(ke):
+            wl.step_host_async(n_e2e + i)
+        n_e2e += ke
+        if (time.perf_counter() - t_wall0) >= args.min_seconds or n_e2e >= 400:
+            break
     wl.drain_host()
     e1.record()
     torch.cuda.synchronize(); D.barrier()
-    e2e_secs = max(e0.elapsed_time(e1) * 1e-3, time.perf_counter() - t_wall0)
-    e2e_value, _ = D.aggregate_throughput(wl.n_tokens * K, e2e_secs, dev)
+    e2e_secs = D.max_over_ranks(max(e0.elapsed_time(e1) * 1e-3, time.perf_counter() - t_wall0), dev)
+    e2e_value = wl.n_tokens * world * n_e2e / e2e_secs
     h.check_status("end-to-end region")
     wl.step_host()
     s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s0.record()
-    for _ in range(K):
+    for _ in range(4):
         wl.step_host()
     s1.record()
     torch.cuda.synchronize(); D.barrier()
-    e2e_serial, _ = D.aggregate_throughput(wl.n_tokens * K, s0.elapsed_time(s1) * 1e-3, dev)
+    e2e_serial = wl.n_tokens * world / (D.max_over_ranks(s0.elapsed_time(s1) * 1e-3, dev) / 4)
     h.check_status("end-to-end region (one batch at a time)")
+    clocks.stop()
 
     shapes = wl.layer_shapes()
     g1, g2, rt = stack_flops(sc.layer, shapes)
@@ -537,13 +630,17 @@ def run_stack(args):
     per_launch_s = prof[dom]["ms"] * 1e-3 / max(prof[dom]["launches"], 1)
     flops_per_launch = {"gemm1": g1, "gemm2": g2, "route": rt}.get(dom, 0.0) / n_layers
     roof = {"bound": "tensor", "achieved": flops_per_launch / per_launch_s / 1e12, "peak": peaks["tf_sustained"],
-            "unit": "TFLOP/s", "kernel": dom, "us_per_launch": per_launch_s * 1e6, "algorithmic_flops": flops_per_launch,
-            "traffic": NCU_TRAFFIC_BYTES.get("C4", {}).get(dom), "peak_source": peaks["source"] + " (sustained bf16)"}
+            "peak_nominal": NOMINAL["bf16_tflops"], "unit": "TFLOP/s", "kernel": dom, "us_per_launch": per_launch_s * 1e6,
+            "algorithmic_flops": flops_per_launch, "traffic": NCU_TRAFFIC_BYTES.get("C4", {}).get(dom),
+            "peak_source": peaks["source"] + " (sustained bf16)",
+            "note": "per-launch figures are the mean over the stack's layers (three different token counts)"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    step_s = tmax / K
+    roof["frac_of_nominal"] = roof["achieved"] / roof["peak_nominal"]
     t_bound = max((g1 + g2 + rt) / (peaks["tf_sustained"] * 1e12), n_layers * weight_bytes(sc.layer) / (peaks["hbm_gbs"] * 1e9))
-    kernels = {k: {"us_per_step": v["ms"] * 1e3 / kp, "launches_per_step": v["launches"] / kp,
-                   "share": v["ms"] / max(sum(x["ms"] for x in prof.values()), 1e-12)} for k, v in prof.items() if v["launches"]}
+    t_bound_nom = max((g1 + g2 + rt) / (NOMINAL["bf16_tflops"] * 1e12), n_layers * weight_bytes(sc.layer) / (NOMINAL["hbm_gbs"] * 1e9))
+    tot_ms = max(sum(x["ms"] for x in prof.values()), 1e-12)
+    kernels = {k: {"us_per_step": v["ms"] * 1e3 / kp, "launches_per_step": v["launches"] / kp, "share": v["ms"] / tot_ms}
+               for k, v in prof.items() if v["launches"]}
 
     # the unreduced, unpruned comparison run (K experts for every token, all tokens in every layer)
     dense = None
@@ -560,36 +657,38 @@ def run_stack(args):
         d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         d0.record()
-        for _ in range(3):
+        nd = 5
+        for _ in range(nd):
             wd.step()
         d1.record()
         torch.cuda.synchronize()
         dg1, dg2, drt = stack_flops(sc.layer, wd.layer_shapes())
-        dense = {"ms_per_step": d0.elapsed_time(d1) / 3, "moe_flops": dg1 + dg2 + drt,
-                 "activated_flops_saved": 1.0 - (g1 + g2 + rt) / (dg1 + dg2 + drt)}
+        dense = {"ms_per_step": d0.elapsed_time(d1) / nd, "moe_flops": dg1 + dg2 + drt,
+                 "activated_flops_saved": 1.0 - (g1 + g2 + rt) / (dg1 + dg2 + drt),
+                 "time_saved": 1.0 - step_s * 1e3 / (d0.elapsed_time(d1) / nd)}
         h.check_status("dense-k run")
+        del wd
 
-    cpu = stack_cpu_baseline(sc, n_layers) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
-    if rank == 0:
-        conf = stack_describe(sc, n_layers)
-        conf.update({"parallelism": f"replicas x{world} (no collective)", "tokens_per_layer": [t for t, _ in shapes],
-                     "final_tokens": wl.out_off[-1], "output_std": out_std,
-                     "weights": "N(0, 0.02^2); down-projections N(0, (0.02/sqrt(2*layers))^2) so that the norm-free "
-                                "residual stack stays at unit scale"})
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-                "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": sc.layer.dtype, "data": "synthetic", "config": conf,
-                "clocks": dict(clocks.summary(), settle_s=round(settle_s, 2)),
-                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(),
-                        "d2h_bytes_per_step": wl.d2h_bytes(), "batches_in_flight": wl.PIPE_DEPTH,
-                        "value_one_batch_at_a_time": e2e_serial},
-                "gpu_launches": int(launches), "roofline": roof,
-                "step_roofline": {"frac": t_bound / step_s, "t_bound_us": t_bound * 1e6, "activated_flops": g1 + g2 + rt,
-                                  "peak_source": peaks["source"]},
-                "kernels": kernels, "dense_k_unpruned": dense, "cpu_baseline": cpu}
-        print(json.dumps(line))
-    D.shutdown()
-    return 0
+    conf = stack_describe(sc, n_layers)
+    conf.update({"parallelism": f"replicas x{world} (no collective)", "tokens_per_layer": [t for t, _ in shapes],
+                 "final_tokens": wl.out_off[-1], "output_std": out_std,
+                 "weights": "N(0, 0.02^2); down-projections N(0, (0.02/sqrt(2*layers))^2) so that the norm-free "
+                            "residual stack stays at unit scale"})
+    rec = {"value": value, "unit": UNIT, "ms_per_step": step_s * 1e3, "timing": stats, "dtype": sc.layer.dtype,
+           "config": conf, "clocks": dict(clocks.summary(), settle_s=round(settle_s, 2)),
+           "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(),
+                   "d2h_bytes_per_step": wl.d2h_bytes(), "batches_in_flight": wl.PIPE_DEPTH, "batches_timed": n_e2e,
+                   "value_one_batch_at_a_time": e2e_serial},
+           "gpu_launches": int(launches * K), "roofline": roof,
+           "step_roofline": {"frac": t_bound / step_s, "frac_of_nominal": t_bound_nom / step_s, "bound": "tensor",
+                             "t_bound_us": t_bound * 1e6, "activated_flops": g1 + g2 + rt, "peak_source": peaks["source"]},
+           "kernels": kernels, "dense_k_unpruned": dense}
+    if with_cpu:
+        rec["cpu_baseline"] = stack_cpu_baseline(sc, n_layers)
+    del wl
+    h.close()
+    gc.collect(); torch.cuda.empty_cache()
+    return rec
 
 
 def run_stack_reference(args):
@@ -609,20 +708,59 @@ def run_stack_reference(args):
     return 0
 
 
+# ------------------------------------------------------------------ the CUDA arm
+def run_ours(args):
+    import torch
+    from paper_2511_17885_b200 import dist as D
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    rank, local, world = D.init("nccl") if int(os.environ.get("WORLD_SIZE", 1)) > 1 else (0, 0, 1)
+    torch.cuda.set_device(local)
+    peaks = load_peaks()
+    head = HEADLINE if args.workload == "all" else args.workload
+    others = [w for w in ("C0", "C1", "C2", "C3", "C4") if w != head] if args.workload == "all" else []
+    with_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
+
+    def measure(name, cpu):
+        if name == "C4":
+            return measure_stack(args, D, rank, local, world, peaks, cpu)
+        return measure_layer(name, args, D, rank, local, world, peaks, cpu)
+
+    rec = measure(head, with_cpu)
+    configs = {}
+    for name in others:
+        configs[name] = measure(name, False)
+    if rank == 0:
+        line = {"metric": METRIC, "value": rec["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": rec["ms_per_step"], "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": rec["dtype"], "data": "synthetic"}
+        for k, v in rec.items():
+            if k not in line:
+                line[k] = v
+        line.setdefault("cpu_baseline", None)
+        if configs:
+            line["configs"] = configs
+        print(json.dumps(line))
+    D.shutdown()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="C1", choices=WORKLOADS)
+    ap.add_argument("--workload", default="all", choices=WORKLOADS)
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="timed GPU work per workload and per region: blocks of --steps steps are repeated until it is reached")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="C4 only: run the first N layers of the stack")
     ap.add_argument("--no-dense", action="store_true", help="C4 only: skip the unreduced, unpruned comparison run")
     args = ap.parse_args()
-    if args.workload == "C4":
-        sys.exit(run_stack_reference(args) if args.impl == "reference" else run_stack(args))
-    sys.exit(run_reference(args) if args.impl == "reference" else run_ours(args))
+    if args.impl == "reference":
+        sys.exit(run_stack_reference(args) if args.workload == "C4" else run_reference(args))
+    sys.exit(run_ours(args))
 
 
 if __name__ == "__main__":

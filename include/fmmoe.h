@@ -98,7 +98,9 @@ typedef struct fmmoe_handle fmmoe_handle;   /* opaque: device, SM count, status 
  * built-in scratch array of fmmoe_prune_visual_static onto the device).  Not thread-safe
  * per handle.  Environment, read once here: FMMOE_DEBUG_SYNC=1 synchronises after every
  * kernel and reports the first failing one on stderr; FMMOE_GATHER_MIN_TOKENS=n moves the
- * token count from which GEMM-1 gathers the routed rows itself (default 12288). */
+ * token count from which GEMM-1 gathers the routed rows itself (default 12288);
+ * FMMOE_SMALL_M_MAX_TOKENS=n moves the token count below which the expert GEMMs run with the
+ * token rows as the MMA's N dimension (default 12288; 0 turns that form off). */
 fmmoe_status fmmoe_create(fmmoe_handle **handle, int device);
 fmmoe_status fmmoe_destroy(fmmoe_handle *handle);
 const char  *fmmoe_status_string(fmmoe_status s);
@@ -193,6 +195,12 @@ fmmoe_status fmmoe_host_wait(fmmoe_handle *handle, uint64_t ticket);
  * bracketed by CUDA events on the launching stream (host-side event objects only; no
  * device memory).  fmmoe_profile_read synchronises the device and returns the summed
  * duration and the number of launches of one kernel since the last reset.
+ * An event pair adds the kernel's launch latency to what it measures, which matters for
+ * kernels of 10-30 us.  fmmoe_profile_enable(handle, n) with n > 1 therefore issues every
+ * launch of a kernel that can be repeated without changing its result (the router, the
+ * finalize pass, the four pruning kernels) n times back to back inside its event pair and
+ * reports the duration divided by n; outputs are unchanged.  The permutation pass (in
+ * place) and the GEMMs (tile counters) always run once.
  * FMMOE_KERNEL_PERMUTE covers the scan and the scatter pass (which also writes the expert-ordered copy of x
  * at small batch); FMMOE_KERNEL_GATHER is kept for numbering only and reports no launches. */
 enum {
@@ -323,6 +331,20 @@ fmmoe_status fmmoe_stack_forward(fmmoe_handle *handle, const fmmoe_layer_desc *d
                                  const int64_t *n_vis /* host */, int32_t n_seq, uint32_t flags,
                                  void *x_out, uint8_t *is_visual_out, int64_t *out_seq_off /* host */,
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Self-test of the library's bounded device-side waits (no counterpart in the paper).  Every
+ * wait of a kernel on a barrier has a time budget; when it runs out the kernel records
+ * FMMOE_ERR_TIMEOUT in the status word, releases its tensor memory and returns, so that a protocol
+ * error ends as a status code with the context intact.  This call ARMS that path for the next
+ * fmmoe_moe_forward on the handle (bf16 layer in its small-M form, i.e. fewer tokens than
+ * FMMOE_SMALL_M_MAX_TOKENS, default 12288): that call's GEMM-1 runs as a single CTA whose
+ * producer stops before it issues any copy or arrival for k-block number `k_block` (0 = the first),
+ * and all of that call's waits use `budget_ns` (1 us .. 1 s) instead of the default 2 s.  Nothing
+ * faults and nothing spins without a limit: the issuing thread's wait for the missing stage
+ * expires, the other roles see the CTA's abort flag, and the kernel leaves through its ordinary
+ * tear-down.  The call's outputs are invalid; fmmoe_get_status returns FMMOE_ERR_TIMEOUT once and
+ * the handle is back to normal for the next call. */
+fmmoe_status fmmoe_test_expire_wait(fmmoe_handle *handle, uint64_t budget_ns, int32_t k_block);
 
 /* fmmoe_prune_visual without a caller-supplied workspace and without any allocation.
  * (The paper has no counterpart: this is a packaging variant of fmmoe_prune_visual above,

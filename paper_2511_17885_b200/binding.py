@@ -115,6 +115,7 @@ def lib() -> C.CDLL:
     L.fmmoe_stack_forward.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(Weights), i32, i32, C.POINTER(StackStage), i32,
                                       vp, vp, C.POINTER(i64), C.POINTER(i64), i32, u32, vp, vp, C.POINTER(i64), vp, sz, vp]
     L.fmmoe_stack_forward.restype = C.c_int
+    L.fmmoe_test_expire_wait.argtypes = [vp, C.c_uint64, i32]; L.fmmoe_test_expire_wait.restype = C.c_int
     L.fmmoe_prune_visual_static.argtypes = [vp, C.POINTER(PruneParams), vp, i32, vp, vp, i32, i32, vp,
                                             C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), i32,
                                             vp, vp, vp, vp, C.POINTER(i64), vp]
@@ -231,6 +232,10 @@ class Handle:
 
     def check_status(self, where: str = "fmmoe_get_status"):
         _check(self.get_status(), where)
+
+    def fmmoe_test_expire_wait(self, budget_ns: int, k_block: int):
+        """Self-test: arm the next fmmoe_moe_forward (small-M form) so that one of its bounded waits runs out."""
+        _check(lib().fmmoe_test_expire_wait(self._h, C.c_uint64(int(budget_ns)), int(k_block)), "fmmoe_test_expire_wait")
 
     def launch_count(self) -> int:
         return int(lib().fmmoe_launch_count(self._h))
@@ -411,6 +416,15 @@ class Handle:
         return {"x_out": x_out, "is_visual_out": vis_out, "keep_idx": keep_idx, "kind": kind,
                 "out_seq_off": [int(v) for v in oo]}
 
+    def prepare_forward_prune(self, desc: LayerDesc, w: Weights, x: torch.Tensor, is_visual: torch.Tensor, flags: int,
+                              out: torch.Tensor, route: Dict[str, torch.Tensor], p: PruneParams,
+                              attn: Optional[torch.Tensor], seq_off, n_vis, n_retain, want_aux: bool = True):
+        """fmmoe_moe_forward_prune with every argument marshalled once: the returned object's run() is a single
+        C call on the current stream that allocates nothing (outputs and the workspace are created here and reused
+        by every run).  For loops that issue the same call many times."""
+        return ForwardPruneCall(self, desc, w, x, is_visual, flags, out, route, p, attn, seq_off, n_vis, n_retain,
+                                want_aux)
+
     def fmmoe_attention_importance(self, q_last: torch.Tensor, k: torch.Tensor, seq_off, scale: Optional[float] = None,
                                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
         """Eq. 7: head-averaged attention of each sequence's last token to all its tokens.
@@ -495,3 +509,49 @@ class Handle:
                                                _ptr(x_out), _ptr(is_visual_out), _ptr(keep_idx), _ptr(kind), oo,
                                                _stream()), "fmmoe_prune_visual_static")
         return [int(v) for v in oo]
+
+
+class ForwardPruneCall:
+    """A marshalled fmmoe_moe_forward_prune call (see Handle.prepare_forward_prune).  `result` has the keys
+    fmmoe_moe_forward_prune returns; its tensors are overwritten by every run()."""
+
+    def __init__(self, handle: Handle, desc, w, x, is_visual, flags, out, route, p, attn, seq_off, n_vis, n_retain,
+                 want_aux):
+        T, H = x.shape
+        B = len(n_vis)
+        arr = C.c_int64 * (B + 1)
+        self.h = handle
+        self.so = arr(*[int(v) for v in seq_off])
+        self.nv = (C.c_int64 * max(B, 1))(*[int(v) for v in n_vis])
+        self.nr = (C.c_int64 * max(B, 1))(*[int(v) for v in n_retain])
+        self.oo = arr()
+        t_out = 0
+        for b in range(B):
+            kept, _, _ = fmmoe_prune_kept_count(int(n_vis[b]), int(n_retain[b]), p)
+            if kept < 0:
+                raise FmmoeError(1, "fmmoe_prune_kept_count")
+            t_out += int(seq_off[b + 1]) - int(seq_off[b]) - int(n_vis[b]) + kept
+        dev = x.device
+        self.x_out = torch.empty((t_out, H), dtype=x.dtype, device=dev)
+        self.vis_out = torch.empty(t_out, dtype=torch.uint8, device=dev) if want_aux else None
+        self.keep_idx = torch.empty(t_out, dtype=torch.int32, device=dev) if want_aux else None
+        self.kind = torch.empty(t_out, dtype=torch.uint8, device=dev) if want_aux else None
+        self.ro = RouteOut(**{k: v.data_ptr() for k, v in route.items()})
+        need = fmmoe_workspace_bytes(desc, T, flags) + 256 + int(lib().fmmoe_prune_workspace_bytes(T, B))
+        self.ws = torch.empty(need + 256, dtype=torch.uint8, device=dev)     # this call's own workspace
+        base = self.ws.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        self.keep = (desc, w, x, is_visual, out, route, p, attn)             # referenced for as long as the call lives
+        self.args = (handle._h, C.byref(desc), C.byref(w), _ptr(x), _ptr(is_visual), T, flags, _ptr(out),
+                     C.byref(self.ro), C.byref(p), _ptr(attn), self.so, self.nv, self.nr, B, _ptr(self.x_out),
+                     _ptr(self.vis_out), _ptr(self.keep_idx), _ptr(self.kind), self.oo, C.c_void_p(aligned),
+                     C.c_size_t(self.ws.numel() - (aligned - base)))
+        self.fn = lib().fmmoe_moe_forward_prune
+        self.result = {"x_out": self.x_out, "is_visual_out": self.vis_out, "keep_idx": self.keep_idx,
+                       "kind": self.kind, "out_seq_off": None}
+
+    def run(self):
+        _check(self.fn(*self.args, _stream()), "fmmoe_moe_forward_prune")
+        if self.result["out_seq_off"] is None:
+            self.result["out_seq_off"] = [int(v) for v in self.oo]
+        return self.result

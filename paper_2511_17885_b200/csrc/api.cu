@@ -45,7 +45,11 @@ bool plan_workspace(const fmmoe_layer_desc& d, int64_t T, uint32_t flags, WsPlan
   size_t o = 0;
   auto take = [&](size_t bytes) { const size_t at = o; o = align_up(o + bytes, 256); return at; };
   p->misc_off = take(8 * 4);
-  p->acc_off = take(det ? 0 : Tz * H * 4);
+  {
+    const size_t acc_bytes = Tz * H * 4;
+    const size_t pair_bytes = d.dtype == FMMOE_BF16 ? (P + (size_t)d.n_shared * Tz) * H * 2 : 0;
+    p->acc_off = take(det ? 0 : (acc_bytes > pair_bytes ? acc_bytes : pair_bytes));
+  }
   p->blk_cnt_off = take((size_t)d.n_experts * ((Tz + 31) / 32 + 4) * 4);
   p->topk_idx_off = take(P * 4);
   p->topk_w_off = take(P * 4);
@@ -162,7 +166,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
   h->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
   h->launches = 0;
   h->d_status = nullptr; h->h_status = nullptr; h->encode_tiled = nullptr;
-  h->tc_attr_set = false; h->route_attr_set = false; h->route_f32_attr_mask = 0; h->profiling = false; h->ev_used = 0;
+  h->tc_attr_set = false; h->route_attr_set = false; h->route_f32_attr_mask = 0; h->profiling = false; h->prof_repeat = 1; h->ev_used = 0;
   h->gather_min_tokens = kGatherMinTokensDefault;
   if (const char* g = getenv("FMMOE_GATHER_MIN_TOKENS")) {
     char* end = nullptr;
@@ -170,6 +174,20 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
     if (end != g && v >= 0) h->gather_min_tokens = v;
   }
   h->wait_budget_ns = 2000000000ull;
+  h->sm_attr_set = false;
+  h->small_m_max_tokens = kGatherMinTokensDefault;
+  if (const char* g = getenv("FMMOE_SMALL_M_MAX_TOKENS")) {
+    char* end = nullptr;
+    const long long v = strtoll(g, &end, 10);
+    if (end != g && v >= 0) h->small_m_max_tokens = v;
+  }
+  h->test_withhold_stage = -1; h->test_budget_ns = 0;
+  h->pair_min_tokens = kPairMinTokensDefault;
+  if (const char* g = getenv("FMMOE_PAIR_ROWS_MIN_TOKENS")) {
+    char* end = nullptr;
+    const long long v = strtoll(g, &end, 10);
+    if (end != g && v >= 0) h->pair_min_tokens = v;
+  }
   h->pipe_ready = false; h->pipe_next = 0; h->ticket_next = 0; h->side_ready = false;
   { const char* dbg = getenv("FMMOE_DEBUG_SYNC"); h->debug_sync = dbg && dbg[0] == '1'; h->debug_seq = 0; }
   if (cudaMalloc(&h->d_status, 256) != cudaSuccess || cudaMemset(h->d_status, 0, 256) != cudaSuccess ||
@@ -268,8 +286,9 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   const RoutePtrs r = bind_route(pl, ws, route);
   // the router clears the scheduler words and (atomic mode) the fp32 accumulator it owns rows of
   // bf16 at small batch: the permutation's scatter pass also writes the expert-grouped copy of x
-  const bool copy_rows = d->dtype == FMMOE_BF16 && !gather_rows_in_gemm(h, T);
-  st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, det ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s,
+  const bool pair = use_pair_rows(h, *d, T, flags);
+  const bool copy_rows = d->dtype == FMMOE_BF16 && (use_small_m(h, T) || !gather_rows_in_gemm(h, T));
+  st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, (det || pair) ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s,
                  copy_rows ? ws + pl.xp_off : nullptr);
   if (st != FMMOE_OK) return st;
   if (after_route) {
@@ -283,11 +302,24 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   fa.tile_counters = r.misc + 1;
   fa.row_token = r.row_token; fa.row_gate = r.row_gate;
   fa.xp = ws + pl.xp_off; fa.act = ws + pl.act_off; fa.act_sh = ws + pl.act_sh_off;
-  fa.acc = det ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off);
+  fa.acc = (det || pair) ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off);
+  fa.pair = pair ? 1 : 0;
+  fa.yb = pair ? ws + pl.acc_off : nullptr;
+  fa.ybsh = pair ? ws + pl.acc_off + (size_t)pl.p_max * d->hidden * 2 : nullptr;
   fa.y = det ? reinterpret_cast<float*>(ws + pl.y_off) : nullptr;
   fa.ysh = det ? reinterpret_cast<float*>(ws + pl.ysh_off) : nullptr;
   fa.deterministic = det; fa.d_status = h->d_status;
-  if (d->dtype == FMMOE_BF16) {
+  fa.test_withhold_stage = -1; fa.grid_override = 0;
+  if (d->dtype == FMMOE_BF16 && use_small_m(h, T)) {
+    const uint64_t budget = h->wait_budget_ns;
+    if (h->test_withhold_stage >= 0) {     // armed self-test: this call only
+      fa.test_withhold_stage = h->test_withhold_stage; fa.grid_override = 1;
+      h->wait_budget_ns = h->test_budget_ns;
+      h->test_withhold_stage = -1;
+    }
+    st = launch_ffn_sm(h, fa, s);
+    h->wait_budget_ns = budget;
+  } else if (d->dtype == FMMOE_BF16) {
     fa.gather_in_gemm = gather_rows_in_gemm(h, T) ? 1 : 0;
     st = launch_ffn_tc(h, fa, s);
   } else {
@@ -299,6 +331,7 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   fin.x = x; fin.out = out; fin.T = T; fin.H = d->hidden; fin.K = d->top_k; fin.n_shared = d->n_shared;
   fin.dtype = d->dtype; fin.add_residual = (flags & FMMOE_FLAG_RESIDUAL) ? 1 : 0; fin.deterministic = det;
   fin.acc = fa.acc; fin.y = fa.y; fin.ysh = fa.ysh; fin.inv_row = r.inv_row; fin.topk_w = r.topk_w;
+  fin.pair = fa.pair; fin.yb = fa.yb; fin.ybsh = fa.ybsh;
   return launch_finalize(h, fin, s);
 }
 
@@ -499,6 +532,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_host_wait(f
 extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_profile_enable(fmmoe_handle* h, int enable) {
   if (!h) return FMMOE_ERR_INVALID_ARG;
   h->profiling = enable != 0;
+  h->prof_repeat = enable > 1 ? enable : 1;
   return FMMOE_OK;
 }
 
@@ -520,10 +554,19 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_profile_rea
     if (r.id != kernel_id) continue;
     float ms = 0.f;
     FMMOE_CUDA_TRY(cudaEventElapsedTime(&ms, h->ev_pool[r.start], h->ev_pool[r.stop]));
-    tot += ms;
+    tot += ms / (r.reps > 0 ? r.reps : 1);
     ++n;
   }
   *total_ms = tot;
   *launches = n;
+  return FMMOE_OK;
+}
+
+// Self-test of the bounded device-side waits: see include/fmmoe.h.
+extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_test_expire_wait(fmmoe_handle* h, uint64_t budget_ns,
+                                                                                       int32_t k_block) {
+  if (!h || k_block < 0 || budget_ns < 1000 || budget_ns > 1000000000ull) return FMMOE_ERR_INVALID_ARG;
+  h->test_withhold_stage = k_block;
+  h->test_budget_ns = budget_ns;
   return FMMOE_OK;
 }

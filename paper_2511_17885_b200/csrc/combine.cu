@@ -13,7 +13,50 @@ namespace fmmoe {
 struct FinalizeDev {
   const void* x; void* out; long long T; int H, K, n_shared, add_residual, deterministic;
   const float* acc; const float* y; const float* ysh; const int32_t* inv_row; const float* topk_w;
+  const __nv_bfloat16* yb; const __nv_bfloat16* ybsh;
 };
+
+__device__ __forceinline__ void add_bf16x8(float (&v)[8], const __nv_bfloat16* p) {
+  const uint4 u = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+    v[2 * i] += f.x; v[2 * i + 1] += f.y;
+  }
+}
+
+// Pair-row mode (bf16 layers, large batches): GEMM-2 wrote every pair's gate-scaled output row once, in bf16.
+// out[t] = sum over the token's slots 0..K-1 (its rows through inv_row), then the shared experts 0..N_s-1,
+// then the residual, in that fixed order in fp32; one rounding to bf16.  No atomics anywhere, so the result is
+// reproducible bit for bit.  A thread owns 8 neighbouring columns of one token: the rows' 16-byte pieces are
+// independent loads.
+__global__ void __launch_bounds__(256) finalize_pair_kernel(const FinalizeDev a) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int hv = a.H / 8;
+  const long long n = a.T * hv;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const long long t = i / hv;
+    const int c = (int)(i - t * hv) * 8;
+    float v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = 0.f;
+    for (int s = 0; s < a.K; ++s) {
+      const int row = a.inv_row[t * a.K + s];
+      if (row >= 0) add_bf16x8(v, a.yb + (long long)row * a.H + c);
+    }
+    for (int s = 0; s < a.n_shared; ++s) add_bf16x8(v, a.ybsh + ((long long)s * a.T + t) * a.H + c);
+    if (a.add_residual) add_bf16x8(v, static_cast<const __nv_bfloat16*>(a.x) + t * a.H + c);
+    uint32_t w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+      w[j] = *reinterpret_cast<const uint32_t*>(&h2);
+    }
+    *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(a.out) + t * a.H + c) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
 
 template <typename T> struct Vec4;
 template <> struct Vec4<float> {
@@ -75,6 +118,23 @@ fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_
   d.x = a.x; d.out = a.out; d.T = a.T; d.H = a.H; d.K = a.K; d.n_shared = a.n_shared;
   d.add_residual = a.add_residual; d.deterministic = a.deterministic;
   d.acc = a.acc; d.y = a.y; d.ysh = a.ysh; d.inv_row = a.inv_row; d.topk_w = a.topk_w;
+  d.yb = static_cast<const __nv_bfloat16*>(a.yb); d.ybsh = static_cast<const __nv_bfloat16*>(a.ybsh);
+  if (a.pair) {
+    if (a.dtype != FMMOE_BF16 || a.H % 8) return FMMOE_ERR_INTERNAL;
+    const long long n8 = a.T * (a.H / 8);
+    long long blocks8 = (n8 + 255) / 256;
+    const long long cap8 = (long long)h->sm_count * 32;
+    if (blocks8 > cap8) blocks8 = cap8;
+    {
+      ProfScope ps(h, FMMOE_KERNEL_FINALIZE, s);
+      for (int rep = 0; rep < ps.reps; ++rep) {
+        FMMOE_CUDA_TRY(launch_pdl(finalize_pair_kernel, dim3((unsigned)blocks8), dim3(256), 0, s, 1, d));
+        h->launches += 1;
+      }
+    }
+    FMMOE_CUDA_TRY(cudaGetLastError());
+    return FMMOE_OK;
+  }
   const long long n = a.T * (a.H / 4);
   const int threads = 256;
   long long blocks = (n + threads - 1) / threads;
@@ -82,11 +142,13 @@ fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_
   if (blocks > cap) blocks = cap;
   {
     ProfScope ps(h, FMMOE_KERNEL_FINALIZE, s);
-    if (a.dtype == FMMOE_BF16) FMMOE_CUDA_TRY(launch_pdl(finalize_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(threads), 0, s, 1, d));
-    else FMMOE_CUDA_TRY(launch_pdl(finalize_kernel<float>, dim3((unsigned)blocks), dim3(threads), 0, s, 1, d));
+    for (int rep = 0; rep < ps.reps; ++rep) {
+      if (a.dtype == FMMOE_BF16) FMMOE_CUDA_TRY(launch_pdl(finalize_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(threads), 0, s, 1, d));
+      else FMMOE_CUDA_TRY(launch_pdl(finalize_kernel<float>, dim3((unsigned)blocks), dim3(threads), 0, s, 1, d));
+      h->launches += 1;
+    }
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
-  h->launches += 1;
   return FMMOE_OK;
 }
 

@@ -34,14 +34,13 @@
 
 #include "internal.h"
 #include "ptx.cuh"
+#include "ffn_common.cuh"
 
 namespace fmmoe {
 
 constexpr int G_BM = TC_BLOCK_M;   // 128
 constexpr int G_BK = 64;           // one 128-byte swizzle atom of bf16
 constexpr int G_STAGES = 4;
-constexpr int G_SCHED = 4;         // slots of the tile ring
-constexpr int G_SLOT_INTS = 8;     // a slot: tile id (-1: no more tiles) + the decoded TileInfo
 constexpr int G_A_BYTES = G_BM * G_BK * 2;          // 16 KB
 constexpr int G_B_BYTES = 2 * 128 * G_BK * 2;       // 32 KB (two 128-row boxes)
 constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;
@@ -52,87 +51,6 @@ constexpr int G_TMEM_COLS = 512;
 constexpr int G_EPI_LD = 33;                                 // padded row of the epilogue transpose buffer
 constexpr int G_EPI_BYTES = 4 * 32 * G_EPI_LD * 4;           // one 32x32 fp32 block per epilogue warp
 constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_EPI_BYTES + 1024 /*align*/ + 384 /*barriers, tile ring*/;
-
-struct Segment {          // routed experts (0) or shared experts (1)
-  int n_nblocks;          // N-blocks per group
-  int k_blocks;           // K / 64
-  int b_rows_per_group;   // rows of the B tensor per group (S_m for GEMM-1, H for GEMM-2)
-  int n_valid;            // valid output columns per group (S_m for GEMM-1, H for GEMM-2)
-  int a_group_stride;     // rows added to the A row per group index (shared experts only)
-  int out_group_stride;   // rows added to the output row per group index
-  int ld_out;             // leading dimension of the output (elements)
-};
-
-struct GemmParams {
-  const MTile* mtiles;        // routed M-tiles
-  const int32_t* n_mtiles;    // device: number of routed M-tiles
-  int max_mtiles;             // capacity of `mtiles` (a corrupt count must not walk past it)
-  int32_t* tile_counter;      // device: next tile to hand out (zero at launch)
-  int shared_mtiles;          // N_s * ceil(T/128), host-known
-  int mt_per_shared;          // ceil(T/128)
-  long long T;
-  Segment seg[2];
-  // epilogue
-  __nv_bfloat16* act[2];      // MODE 0: activation outputs (routed, shared)
-  const __nv_bfloat16* x; int ld_x;   // MODE 0: hidden states [T, H] the routed rows are gathered from
-  const int32_t* row_token;   // grouped row -> token (MODE 0: gather, MODE 1: combine)
-  const float* row_gate;      // MODE 1
-  float* acc;                 // MODE 1 atomic:  [T, H]
-  float* y[2];                // MODE 1 deterministic: routed [P, H], shared [N_s*T, H]
-  int deterministic;
-  int gather;                 // MODE 0: routed rows come from x through the loader warps (else from the tmA_r map)
-  int* status;
-};
-
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-
-struct TileInfo {
-  int seg, group_local, row0, rows, nb;
-  bool single;   // routed: the expert's rows fit this one M-tile
-};
-
-// Position `tile` of the interleaved order -> (segment, M-tile, N-block).
-__device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, int tile, int n_mt_r) {
-  TileInfo ti;
-  const unsigned long long R = (unsigned long long)n_mt_r * p.seg[0].n_nblocks;
-  const unsigned long long S = (unsigned long long)p.shared_mtiles * p.seg[1].n_nblocks;
-  const unsigned long long N = R + S;
-  const unsigned long long sb = (unsigned long long)tile * S / N;          // shared tiles before this position
-  const unsigned long long sb1 = (unsigned long long)(tile + 1) * S / N;
-  if (sb1 == sb) {
-    const int r = tile - (int)sb;
-    const int mt = r / p.seg[0].n_nblocks;
-    ti.seg = 0;
-    ti.nb = r - mt * p.seg[0].n_nblocks;
-    const MTile m = p.mtiles[mt];
-    ti.group_local = m.group; ti.row0 = m.row0; ti.rows = m.rows;
-    ti.single = m.pad != 0;
-  } else {
-    const int t2 = (int)sb;
-    ti.seg = 1;
-    ti.nb = t2 / p.shared_mtiles;
-    const int mt = t2 - ti.nb * p.shared_mtiles;
-    ti.group_local = mt / p.mt_per_shared;
-    const int mb = mt - ti.group_local * p.mt_per_shared;
-    ti.row0 = mb * G_BM;
-    const long long left = p.T - (long long)ti.row0;
-    ti.rows = left < G_BM ? (int)left : G_BM;
-    ti.single = false;
-  }
-  return ti;
-}
-
-// A slot of the tile ring as the producer publishes it and the other roles read it.
-__device__ __forceinline__ void slot_store(volatile int* s, int tile, const TileInfo& ti) {
-  s[0] = tile; s[1] = ti.seg; s[2] = ti.group_local; s[3] = ti.row0; s[4] = ti.rows; s[5] = ti.nb; s[6] = ti.single;
-}
-__device__ __forceinline__ TileInfo slot_load(const volatile int* s) {
-  TileInfo ti;
-  ti.seg = s[1]; ti.group_local = s[2]; ti.row0 = s[3]; ti.rows = s[4]; ti.nb = s[5]; ti.single = s[6] != 0;
-  return ti;
-}
 
 // MODE 0: GEMM-1 + SwiGLU.  MODE 1: GEMM-2 + combine.
 template <int MODE>
@@ -408,6 +326,29 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         }
         if (p.deterministic) gate = 1.f;   // gates are applied by the ordered gather
         float* ybase = p.deterministic ? p.y[ti.seg] + out_row0 * sg.ld_out + ti.nb * 256 : nullptr;
+        if (p.pair) {
+          // Pair-row mode: this thread owns grouped row r; its 32 accumulator columns of a chunk are 64
+          // contiguous bytes of that row of yb, written straight from registers (two full 32-byte sectors).
+          __nv_bfloat16* yrow = p.yb[ti.seg] + (out_row0 + lane) * sg.ld_out + ti.nb * 256;
+#pragma unroll 1
+          for (int c = 0; c < 8; ++c) {
+            if (ti.nb * 256 + c * 32 >= sg.n_valid) break;   // warp-uniform
+            uint32_t v[32];
+            tmem_ld32(taddr + c * 32, v);
+            tmem_ld_wait();
+            if (lane < rows_w) {
+              uint32_t w16[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const __nv_bfloat162 hh = __floats2bfloat162_rn(gate * __uint_as_float(v[2 * i]), gate * __uint_as_float(v[2 * i + 1]));
+                w16[i] = *reinterpret_cast<const uint32_t*>(&hh);
+              }
+              uint4* dst = reinterpret_cast<uint4*>(yrow + c * 32);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w16[4 * i], w16[4 * i + 1], w16[4 * i + 2], w16[4 * i + 3]);
+            }
+          }
+        } else
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
           if (ti.nb * 256 + c * 32 >= sg.n_valid) break;   // warp-uniform
@@ -460,24 +401,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// bf16 row-major [rows, cols] tensor, box = 64 columns x box_rows rows, 128-byte swizzle.
-static bool make_map(fmmoe_handle* h, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-  if (rows == 0) rows = 1;
-  const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {cols * 2};
-  const cuuint32_t box[2] = {G_BK, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = reinterpret_cast<EncodeTiledFn>(h->encode_tiled)(
-      m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
-}
-
 fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   const fmmoe_layer_desc& d = *a.d;
   const int H = d.hidden, I = d.inter, E = d.n_experts, Ns = d.n_shared, Is = d.shared_inter;
@@ -520,6 +443,7 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   p2.seg[1] = Segment{Ns ? (H + 255) / 256 : 0, Ns ? Is / G_BK : 0, H, H, (int)a.T, (int)a.T, H};
   p2.row_token = a.row_token; p2.row_gate = a.row_gate; p2.acc = a.acc;
   p2.y[0] = a.y; p2.y[1] = a.ysh; p2.deterministic = a.deterministic;
+  p2.yb[0] = static_cast<__nv_bfloat16*>(a.yb); p2.yb[1] = static_cast<__nv_bfloat16*>(a.ybsh); p2.pair = a.pair;
   p2.tile_counter = a.tile_counters + 1;
 
   if (!h->tc_attr_set) {

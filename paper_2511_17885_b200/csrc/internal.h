@@ -21,16 +21,22 @@ struct fmmoe_handle {
   void* encode_tiled;   // cuTensorMapEncodeTiled entry point
   bool tc_attr_set;     // dynamic shared memory opt-in done for the tensor-core kernels
   bool route_attr_set;  // ... for the bf16 router
+  bool sm_attr_set;     // ... for the small-M form of the expert GEMMs
+  int64_t small_m_max_tokens;     // below this many tokens the expert GEMMs run in their small-M form
+  int64_t pair_min_tokens;        // from this many tokens on the combine goes through per-pair bf16 rows (no atomics)
+  int test_withhold_stage;        // self-test (fmmoe_test_expire_wait): armed for the next layer call, else -1
+  uint64_t test_budget_ns;
   uint32_t route_f32_attr_mask;   // ... for the fp32 router instantiations (bit = logits per lane)
   int64_t gather_min_tokens;      // from this many tokens on GEMM-1 gathers the routed rows of x itself
   uint64_t wait_budget_ns;        // time budget of every bounded device-side wait
   // optional kernel timeline
   bool profiling;
+  int prof_repeat;      // timeline on: launches of a short idempotent kernel issued back to back inside one event pair
   bool debug_sync;      // FMMOE_DEBUG_SYNC=1: synchronise after every kernel and report the first CUDA error on stderr
   int64_t debug_seq;    // kernels launched so far in debug mode
   std::vector<cudaEvent_t> ev_pool;
   size_t ev_used;
-  struct ProfRec { int id; size_t start, stop; };
+  struct ProfRec { int id; size_t start, stop; int reps; };
   std::vector<ProfRec> prof;
   // pipelined host I/O (created on first use): one stream per copy direction, a ring of events that
   // order them against the caller's compute stream, and a ring of events behind the host tickets
@@ -69,7 +75,8 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 struct WsPlan {
   size_t blk_cnt_off;           // int32 [E][ceil(T/32)] per-block expert counts / offsets (not cleared)
   size_t misc_off;              // int32 [8]: [0] number of routed M-tiles, [1],[2] GEMM tile counters
-  size_t acc_off;               // fp32 [T,H] combine accumulator (atomic mode)
+  size_t acc_off;               // fp32 [T,H] combine accumulator (atomic mode); the same region holds the bf16
+                                // per-pair outputs [P_max + N_s*T, H] in pair-row mode (sized for the larger)
   size_t topk_idx_off, topk_w_off, inv_row_off;
   size_t expert_off_off, row_token_off, row_gate_off, mtiles_off;
   size_t xp_off;                // dtype [P_max,H] rows gathered by expert (bf16 path)
@@ -84,16 +91,25 @@ struct WsPlan {
 bool plan_workspace(const fmmoe_layer_desc& d, int64_t T, uint32_t flags, WsPlan* p);
 
 // Brackets one kernel launch with events when the handle's timeline is on.
+// Kernels that give the same result when run twice in a row on the same arguments: with the timeline's repeat
+// count above 1 their launch is issued that many times inside the event pair (`reps`), so that the launch
+// latency an event pair adds to a 10-30 us kernel is amortised.  The scan / scatter pass works in place and
+// the GEMMs consume a tile counter, so they always run once.
+static inline bool prof_idempotent(int id) {
+  return id == FMMOE_KERNEL_ROUTE || id == FMMOE_KERNEL_FINALIZE || id == FMMOE_KERNEL_PRUNE_INDEX ||
+         id == FMMOE_KERNEL_PRUNE_SCORE || id == FMMOE_KERNEL_PRUNE_SELECT || id == FMMOE_KERNEL_PRUNE_COMPACT;
+}
 struct ProfScope {
-  fmmoe_handle* h; cudaStream_t s; size_t rec; bool on; int kid;
-  ProfScope(fmmoe_handle* h_, int id, cudaStream_t s_) : h(h_), s(s_), rec(0), on(h_->profiling), kid(id) {
+  fmmoe_handle* h; cudaStream_t s; size_t rec; bool on; int kid; int reps;
+  ProfScope(fmmoe_handle* h_, int id, cudaStream_t s_) : h(h_), s(s_), rec(0), on(h_->profiling), kid(id), reps(1) {
     if (!on) return;
+    if (h->prof_repeat > 1 && prof_idempotent(id)) reps = h->prof_repeat;
     while (h->ev_pool.size() < h->ev_used + 2) {
       cudaEvent_t e;
       if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
       h->ev_pool.push_back(e);
     }
-    fmmoe_handle::ProfRec r{id, h->ev_used, h->ev_used + 1};
+    fmmoe_handle::ProfRec r{id, h->ev_used, h->ev_used + 1, reps};
     h->ev_used += 2;
     h->prof.push_back(r);
     rec = h->prof.size() - 1;
@@ -188,9 +204,13 @@ struct FfnArgs {   // both paths
   void* xp; void* act; void* act_sh;
   float* acc;            // atomic mode
   float* y; float* ysh;  // deterministic mode
+  void* yb; void* ybsh;  // pair-row mode (bf16)
   int deterministic;
+  int pair;              // GEMM-2 stores gate-scaled bf16 rows per pair; the finalize pass sums them per token
   int gather_in_gemm;    // bf16: GEMM-1 gathers the routed rows of x itself (xp is not read)
   int* d_status;
+  int test_withhold_stage;   // small-M form, self-test only (-1: off)
+  int grid_override;         // small-M form, self-test only: CTAs to launch (0: one per SM)
 };
 // Large batches: skip the expert-ordered copy of x and let GEMM-1's loader warps gather the rows.
 // Small batches are bound by the weight stream, where the copy + plain TMA boxes are faster.
@@ -198,12 +218,22 @@ struct FfnArgs {   // both paths
 // in fmmoe_create, overrides it so that either path can be exercised at any size).
 constexpr int64_t kGatherMinTokensDefault = 12288;
 static inline bool gather_rows_in_gemm(const fmmoe_handle* h, int64_t T) { return T >= h->gather_min_tokens; }
-fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05
+fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05, token rows as M
+fmmoe_status launch_ffn_sm(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05, token rows as N (reads xp)
+// Which form runs: below small_m_max_tokens (and below the in-GEMM gather threshold) the small-M form.
+// The fp32 accumulator of the atomic combine is T*H*4 bytes; once it no longer fits the L2 cache next to the
+// activations its read-modify-writes page through HBM, and writing every pair's row once in bf16 is cheaper.
+constexpr int64_t kPairMinTokensDefault = 8192;
+static inline bool use_pair_rows(const fmmoe_handle* h, const fmmoe_layer_desc& d, int64_t T, uint32_t flags) {
+  return d.dtype == FMMOE_BF16 && !(flags & FMMOE_FLAG_DETERMINISTIC) && T >= h->pair_min_tokens;
+}
+static inline bool use_small_m(const fmmoe_handle* h, int64_t T) { return T < h->small_m_max_tokens && T < h->gather_min_tokens; }
 fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);   // fp32 FMA
 
 struct FinalizeArgs {
   const void* x; void* out; int64_t T; int H, K, n_shared; int dtype; int add_residual; int deterministic;
   const float* acc; const float* y; const float* ysh; const int32_t* inv_row; const float* topk_w;
+  int pair; const void* yb; const void* ybsh;   // pair-row mode: bf16 [P,H] gate-scaled rows, [N_s*T,H] shared rows
 };
 fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_t s);
 

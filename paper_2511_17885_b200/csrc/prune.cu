@@ -6,8 +6,9 @@
 //                        merge set = m highest C (Eq. 15), drop set = d smallest A_bar among
 //                        the rest (both by an in-CTA bitonic sort of (score, window) keys),
 //                        then the stable compaction map (scan of keep flags)
-//   compact_kernel     : copies kept rows; a merged window becomes mean(rows) rescaled to the
-//                        largest member norm (Eq. 16-18) at its first token's position
+//   compact_kernel     : copies kept rows (a warp per row, eight rows per CTA); a merged window becomes
+//                        mean(rows) rescaled to the largest member norm (Eq. 16-18) at its first token's
+//                        position, formed by the whole CTA
 // Ranks come from sorting unique (value, window index) keys, so the keep-set does not depend
 // on thread order; ties go to the lower window index.
 #include <cuda_bf16.h>
@@ -423,100 +424,131 @@ template <> struct Row8<float> {
   }
 };
 
+// Rows per CTA of compact_kernel: one warp copies one kept row (the common case: with the paper's merge
+// rates about 3 % of the output rows are merged windows), then the whole CTA forms the block's merged rows
+// one after another, so that a merge still has 256 threads behind it.
+constexpr int CP_ROWS = 8;
+
 template <typename T>
 __global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const PruneSeqs sq, long long row_base, long long n_rows) {
   constexpr int N = Row8<T>::N;
   __shared__ float s_red[8][MAXW + 1];
   __shared__ float s_scale;
-  const long long row = row_base + blockIdx.x;
+  __shared__ unsigned s_merged;                  // bit w: row w of this block is a merged window
   pdl_launch_dependents();
-  pdl_wait();
-  if (blockIdx.x >= n_rows) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_merged = 0;
+  __syncthreads();
+  pdl_wait();
   const T* X = static_cast<const T*>(a.x);
-  T* O = static_cast<T*>(a.x_out) + row * a.H;
-  int b = 0;
-  while (b + 1 < sq.n_seq && row >= sq.out_off[b + 1]) ++b;
-  const long long t0 = a.keep_idx_ws[row];
-  const int kd = a.kind_ws[row];
-  if (t0 < sq.seq_off[b] || t0 >= sq.seq_off[b + 1]) {
-    // a slot the selection pass did not fill: only possible when the mask contradicts the host's vision
-    // count (reported through the status word).  Never index x with it.
-    uint4* dst = reinterpret_cast<uint4*>(O);
-    for (int i = tid; i < a.H / N; i += 256) dst[i] = make_uint4(0u, 0u, 0u, 0u);
-    return;
-  }
-  if (kd != 2) {
-    const uint4* src = reinterpret_cast<const uint4*>(X + t0 * a.H);
-    uint4* dst = reinterpret_cast<uint4*>(O);
-    for (int i = tid; i < a.H / N; i += 256) dst[i] = src[i];
-    return;
-  }
-  int v0 = a.vrank[t0];
-  if (v0 < 0 || v0 + a.W > sq.n_vis[b]) v0 = 0;   // inconsistent mask / count (status word set): stay inside the list
-  const long long s_lo = sq.seq_off[b], s_hi = sq.seq_off[b + 1];
-  long long mem[MAXW];
+  const int vec = a.H / N;                       // 16-byte pieces per row
+  const long long blk_row0 = (long long)blockIdx.x * CP_ROWS;
+  // ---- phase 1: warp w copies row blk_row0 + w (all loads of a row in flight before its stores)
+  int my_kind = -1;
+  {
+    const long long rel = blk_row0 + warp;
+    if (rel < n_rows) {
+      const long long row = row_base + rel;
+      int b = 0;
+      while (b + 1 < sq.n_seq && row >= sq.out_off[b + 1]) ++b;
+      const long long t0 = a.keep_idx_ws[row];
+      my_kind = a.kind_ws[row];
+      uint4* dst = reinterpret_cast<uint4*>(static_cast<T*>(a.x_out) + row * a.H);
+      if (t0 < sq.seq_off[b] || t0 >= sq.seq_off[b + 1]) {
+        // a slot the selection pass did not fill: only possible when the mask contradicts the host's vision
+        // count (reported through the status word).  Never index x with it.
+        for (int i = lane; i < vec; i += 32) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        my_kind = -1;
+      } else if (my_kind != 2) {
+        const uint4* src = reinterpret_cast<const uint4*>(X + t0 * a.H);
+        for (int i0 = 0; i0 < vec; i0 += 256) {
+          uint4 v[8];
 #pragma unroll
-  for (int k = 0; k < MAXW; ++k) {
-    long long tkn = k < a.W ? a.vis_list[s_lo + v0 + k] : s_lo;
-    if (tkn < s_lo || tkn >= s_hi) tkn = s_lo;
-    mem[k] = tkn;
-  }
-  const float invW = 1.f / (float)a.W;
-  // pass 1: squared norms of the members and of the mean
-  float part[MAXW + 1];
+          for (int u = 0; u < 8; ++u) { const int i = i0 + u * 32 + lane; if (i < vec) v[u] = src[i]; }
 #pragma unroll
-  for (int k = 0; k <= MAXW; ++k) part[k] = 0.f;
-  for (int i = tid; i < a.H / N; i += 256) {
-    float mean[N];
-#pragma unroll
-    for (int j = 0; j < N; ++j) mean[j] = 0.f;
-#pragma unroll
-    for (int k = 0; k < MAXW; ++k) {
-      if (k < a.W) {
-        float f[N];
-        Row8<T>::load(X + mem[k] * a.H + i * N, f);
-#pragma unroll
-        for (int j = 0; j < N; ++j) { part[k] = fmaf(f[j], f[j], part[k]); mean[j] += f[j]; }
+          for (int u = 0; u < 8; ++u) { const int i = i0 + u * 32 + lane; if (i < vec) dst[i] = v[u]; }
+        }
       }
     }
-#pragma unroll
-    for (int j = 0; j < N; ++j) { const float mv = mean[j] * invW; part[MAXW] = fmaf(mv, mv, part[MAXW]); }
   }
-#pragma unroll
-  for (int k = 0; k <= MAXW; ++k) {
-    float v = part[k];
-#pragma unroll
-    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    if (lane == 0) s_red[warp][k] = v;
-  }
+  // ---- phase 2: the block's merged rows, one at a time, by the whole CTA
+  if (lane == 0 && my_kind == 2) atomicOr(&s_merged, 1u << warp);
   __syncthreads();
-  if (tid == 0) {
-    float tot[MAXW + 1];
-    for (int k = 0; k <= MAXW; ++k) { tot[k] = 0.f; for (int w = 0; w < 8; ++w) tot[k] += s_red[w][k]; }
-    float nmax = 0.f;
-    for (int k = 0; k < a.W; ++k) nmax = fmaxf(nmax, sqrtf(tot[k]));
-    const float nb = sqrtf(tot[MAXW]);
-    s_scale = a.merge_mode == 1 ? 1.f : (nb > 0.f ? nmax / nb : 0.f);   // Eq. 18
-  }
-  __syncthreads();
-  const float scale = s_scale * invW;
-  for (int i = tid; i < a.H / N; i += 256) {
-    float mean[N];
-#pragma unroll
-    for (int j = 0; j < N; ++j) mean[j] = 0.f;
+  const unsigned merged_mask = s_merged;
+  for (int w = 0; w < CP_ROWS; ++w) {
+    if (!((merged_mask >> w) & 1)) continue;
+    const long long row = row_base + blk_row0 + w;
+    T* O = static_cast<T*>(a.x_out) + row * a.H;
+    int b = 0;
+    while (b + 1 < sq.n_seq && row >= sq.out_off[b + 1]) ++b;
+    const long long t0 = a.keep_idx_ws[row];
+    int v0 = a.vrank[t0];
+    if (v0 < 0 || v0 + a.W > sq.n_vis[b]) v0 = 0;   // inconsistent mask / count (status word set): stay inside the list
+    const long long s_lo = sq.seq_off[b], s_hi = sq.seq_off[b + 1];
+    long long mem[MAXW];
 #pragma unroll
     for (int k = 0; k < MAXW; ++k) {
-      if (k < a.W) {
-        float f[N];
-        Row8<T>::load(X + mem[k] * a.H + i * N, f);
+      long long tkn = k < a.W ? a.vis_list[s_lo + v0 + k] : s_lo;
+      if (tkn < s_lo || tkn >= s_hi) tkn = s_lo;
+      mem[k] = tkn;
+    }
+    const float invW = 1.f / (float)a.W;
+    // pass 1: squared norms of the members and of the mean
+    float part[MAXW + 1];
 #pragma unroll
-        for (int j = 0; j < N; ++j) mean[j] += f[j];
+    for (int k = 0; k <= MAXW; ++k) part[k] = 0.f;
+    for (int i = tid; i < vec; i += 256) {
+      float mean[N];
+#pragma unroll
+      for (int j = 0; j < N; ++j) mean[j] = 0.f;
+#pragma unroll
+      for (int k = 0; k < MAXW; ++k) {
+        if (k < a.W) {
+          float f[N];
+          Row8<T>::load(X + mem[k] * a.H + i * N, f);
+#pragma unroll
+          for (int j = 0; j < N; ++j) { part[k] = fmaf(f[j], f[j], part[k]); mean[j] += f[j]; }
+        }
       }
+#pragma unroll
+      for (int j = 0; j < N; ++j) { const float mv = mean[j] * invW; part[MAXW] = fmaf(mv, mv, part[MAXW]); }
     }
 #pragma unroll
-    for (int j = 0; j < N; ++j) mean[j] *= scale;
-    Row8<T>::store(O + i * N, mean);
+    for (int k = 0; k <= MAXW; ++k) {
+      float v = part[k];
+#pragma unroll
+      for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) s_red[warp][k] = v;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      float tot[MAXW + 1];
+      for (int k = 0; k <= MAXW; ++k) { tot[k] = 0.f; for (int ww = 0; ww < 8; ++ww) tot[k] += s_red[ww][k]; }
+      float nmax = 0.f;
+      for (int k = 0; k < a.W; ++k) nmax = fmaxf(nmax, sqrtf(tot[k]));
+      const float nb = sqrtf(tot[MAXW]);
+      s_scale = a.merge_mode == 1 ? 1.f : (nb > 0.f ? nmax / nb : 0.f);   // Eq. 18
+    }
+    __syncthreads();
+    const float scale = s_scale * invW;
+    for (int i = tid; i < vec; i += 256) {
+      float mean[N];
+#pragma unroll
+      for (int j = 0; j < N; ++j) mean[j] = 0.f;
+#pragma unroll
+      for (int k = 0; k < MAXW; ++k) {
+        if (k < a.W) {
+          float f[N];
+          Row8<T>::load(X + mem[k] * a.H + i * N, f);
+#pragma unroll
+          for (int j = 0; j < N; ++j) mean[j] += f[j];
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < N; ++j) mean[j] *= scale;
+      Row8<T>::store(O + i * N, mean);
+    }
+    __syncthreads();   // s_red / s_scale are reused by the block's next merged row
   }
 }
 
@@ -654,28 +686,36 @@ fmmoe_status fmmoe::prune_visual_phases(fmmoe_handle* h, const fmmoe_prune_param
     al.sim = a.sim + win_base; al.asum = a.asum + win_base;
     if (phases & 1) {
       cudaStream_t s = s_select;
-      { ProfScope ps(h, FMMOE_KERNEL_PRUNE_INDEX, s); FMMOE_CUDA_TRY(launch_pdl(vis_index_kernel, dim3(nb), dim3(1024), 0, s, 1, al, rel)); }
-      FMMOE_CUDA_TRY(cudaGetLastError());
-      h->launches += 1;
-      if (n_win > 0) {
-        { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SCORE, s); FMMOE_CUDA_TRY(launch_pdl(window_score_kernel, dim3((n_win + 7) / 8), dim3(256), 0, s, 1, al, rel)); }
-        FMMOE_CUDA_TRY(cudaGetLastError());
-        h->launches += 1;
+      {
+        ProfScope ps(h, FMMOE_KERNEL_PRUNE_INDEX, s);
+        for (int rep = 0; rep < ps.reps; ++rep, ++h->launches)
+          FMMOE_CUDA_TRY(launch_pdl(vis_index_kernel, dim3(nb), dim3(1024), 0, s, 1, al, rel));
       }
-      { ProfScope ps(h, FMMOE_KERNEL_PRUNE_SELECT, s); FMMOE_CUDA_TRY(launch_pdl(select_kernel, dim3(nb), dim3(1024), sel_smem, s, 1, al, rel)); }
       FMMOE_CUDA_TRY(cudaGetLastError());
-      h->launches += 1;
+      if (n_win > 0) {
+        ProfScope ps(h, FMMOE_KERNEL_PRUNE_SCORE, s);
+        for (int rep = 0; rep < ps.reps; ++rep, ++h->launches)
+          FMMOE_CUDA_TRY(launch_pdl(window_score_kernel, dim3((n_win + 7) / 8), dim3(256), 0, s, 1, al, rel));
+      }
+      FMMOE_CUDA_TRY(cudaGetLastError());
+      {
+        ProfScope ps(h, FMMOE_KERNEL_PRUNE_SELECT, s);
+        for (int rep = 0; rep < ps.reps; ++rep, ++h->launches)
+          FMMOE_CUDA_TRY(launch_pdl(select_kernel, dim3(nb), dim3(1024), sel_smem, s, 1, al, rel));
+      }
+      FMMOE_CUDA_TRY(cudaGetLastError());
     }
     const long long rows = rel.out_off[nb] - rel.out_off[0];
     if ((phases & 2) && rows > 0) {
       cudaStream_t s = s_rows;
       ProfScope ps(h, FMMOE_KERNEL_PRUNE_COMPACT, s);
-      if (dtype == FMMOE_BF16)
-        FMMOE_CUDA_TRY(launch_pdl(compact_kernel<__nv_bfloat16>, dim3((unsigned)rows), dim3(256), 0, s, 1, al, rel, (long long)rel.out_off[0], (long long)rows));
-      else
-        FMMOE_CUDA_TRY(launch_pdl(compact_kernel<float>, dim3((unsigned)rows), dim3(256), 0, s, 1, al, rel, (long long)rel.out_off[0], (long long)rows));
+      for (int rep = 0; rep < ps.reps; ++rep, ++h->launches) {
+        if (dtype == FMMOE_BF16)
+          FMMOE_CUDA_TRY(launch_pdl(compact_kernel<__nv_bfloat16>, dim3((unsigned)((rows + CP_ROWS - 1) / CP_ROWS)), dim3(256), 0, s, 1, al, rel, (long long)rel.out_off[0], (long long)rows));
+        else
+          FMMOE_CUDA_TRY(launch_pdl(compact_kernel<float>, dim3((unsigned)((rows + CP_ROWS - 1) / CP_ROWS)), dim3(256), 0, s, 1, al, rel, (long long)rel.out_off[0], (long long)rows));
+      }
       FMMOE_CUDA_TRY(cudaGetLastError());
-      h->launches += 1;
     }
     win_base += n_win;
   }

@@ -561,8 +561,11 @@ static fmmoe_status launch_route_tc(fmmoe_handle* h, RouteDev d, cudaStream_t s)
   const int tiles = (int)((d.T + RT_BM - 1) / RT_BM);
   {
     ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
-    FMMOE_CUDA_TRY(launch_pdl(route_tc_kernel, dim3((unsigned)(tiles * split)), dim3(RT_THREADS), smem, s, (unsigned)split, mx, mw, d,
-                              stages, tmem_cols, (int)tile_bytes, split, h->d_status));
+    for (int rep = 0; rep < ps.reps; ++rep) {
+      FMMOE_CUDA_TRY(launch_pdl(route_tc_kernel, dim3((unsigned)(tiles * split)), dim3(RT_THREADS), smem, s, (unsigned)split, mx, mw, d,
+                                stages, tmem_cols, (int)tile_bytes, split, h->d_status));
+      h->launches += 1;
+    }
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   return FMMOE_OK;
@@ -579,7 +582,10 @@ static fmmoe_status launch_nt(fmmoe_handle* h, const RouteDev& d, int grid, cuda
   }
   {
     ProfScope ps(h, FMMOE_KERNEL_ROUTE, s);
-    FMMOE_CUDA_TRY(launch_pdl(route_f32_kernel<NT>, dim3(grid), dim3(R_THREADS), smem, s, 1, d));
+    for (int rep = 0; rep < ps.reps; ++rep) {
+      FMMOE_CUDA_TRY(launch_pdl(route_f32_kernel<NT>, dim3(grid), dim3(R_THREADS), smem, s, 1, d));
+      h->launches += 1;
+    }
   }
   FMMOE_CUDA_TRY(cudaGetLastError());
   return FMMOE_OK;
@@ -611,7 +617,6 @@ fmmoe_status launch_route(fmmoe_handle* h, const RouteArgs& a, cudaStream_t s) {
       default: return FMMOE_ERR_UNSUPPORTED;
     }
   }
-  if (st == FMMOE_OK) h->launches += 1;
   return st;
 }
 

@@ -144,18 +144,40 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_stack_forwa
     ro.probs = s ? probs : nullptr;
     // the layer writes straight into the caller's buffer when nothing follows it
     void* layer_out = (last && !s) ? x_out : free_buf(cur_x);
-    fmmoe_status st = fmmoe_moe_forward(h, d, &layer_w[l], cur_x, cur_mask, T, lf, layer_out, &ro, ws + pl.layer_ws,
-                                        pl.layer_ws_bytes, cuda_stream);
-    if (st != FMMOE_OK) return st;
-    cur_x = layer_out;
-    if (s) {
-      for (int32_t b = 0; b < n_seq; ++b) eta[b] = (int64_t)floor((double)n_vis[b] * s->retain + 1e-9);
-      void* pruned = last ? x_out : free_buf(cur_x);
-      uint8_t* pmask = (last && is_visual_out) ? is_visual_out : free_mask(cur_mask);
-      st = fmmoe_prune_visual(h, &s->params, probs, d->n_experts, s->attn, cur_x, d->dtype, d->hidden, cur_mask, off.data(),
-                              vis.data(), eta.data(), n_seq, pruned, pmask, nullptr, nullptr, noff.data(), ws + pl.prune_ws,
-                              pl.prune_ws_bytes, cuda_stream);
+    fmmoe_status st;
+    if (!s) {
+      st = fmmoe_moe_forward(h, d, &layer_w[l], cur_x, cur_mask, T, lf, layer_out, &ro, ws + pl.layer_ws,
+                             pl.layer_ws_bytes, cuda_stream);
       if (st != FMMOE_OK) return st;
+      cur_x = layer_out;
+    } else {
+      // A pruning layer: the layer and its stage as the single call, whose scoring and selection kernels run
+      // beside the expert GEMMs instead of after them.  Three activation tensors are involved (the layer's
+      // input, its output, the pruned rows) and the workspace has two buffers: the pruned rows take the place
+      // of the layer's input, which nothing reads after the layer's last kernel.  That needs the input to be
+      // one of this workspace's buffers, i.e. any layer but the first (the caller's x is never written).
+      for (int32_t b = 0; b < n_seq; ++b) eta[b] = (int64_t)floor((double)n_vis[b] * s->retain + 1e-9);
+      const bool in_place_ok = cur_x != x;      // the layer's input is dead once GEMM-1 and the router have read it
+      void* pruned = last ? x_out : (in_place_ok ? const_cast<void*>(cur_x) : nullptr);
+      uint8_t* pmask = (last && is_visual_out) ? is_visual_out : free_mask(cur_mask);
+      if (pruned) {
+        st = fmmoe_moe_forward_prune(h, d, &layer_w[l], cur_x, cur_mask, T, lf, layer_out, &ro, &s->params, s->attn,
+                                     off.data(), vis.data(), eta.data(), n_seq, pruned, pmask, nullptr, nullptr,
+                                     noff.data(), ws + pl.layer_ws, pl.layer_ws_bytes + pl.prune_ws_bytes, cuda_stream);
+        if (st != FMMOE_OK) return st;
+        cur_x = layer_out;
+      } else {
+        // stage right after the first layer: no third buffer is free, so the two calls in sequence
+        st = fmmoe_moe_forward(h, d, &layer_w[l], cur_x, cur_mask, T, lf, layer_out, &ro, ws + pl.layer_ws,
+                               pl.layer_ws_bytes, cuda_stream);
+        if (st != FMMOE_OK) return st;
+        cur_x = layer_out;
+        pruned = free_buf(cur_x);
+        st = fmmoe_prune_visual(h, &s->params, probs, d->n_experts, s->attn, cur_x, d->dtype, d->hidden, cur_mask,
+                                off.data(), vis.data(), eta.data(), n_seq, pruned, pmask, nullptr, nullptr, noff.data(),
+                                ws + pl.prune_ws, pl.prune_ws_bytes, cuda_stream);
+        if (st != FMMOE_OK) return st;
+      }
       for (int32_t b = 0; b < n_seq; ++b) {
         const int64_t n_text = (off[b + 1] - off[b]) - vis[b];
         vis[b] = (noff[b + 1] - noff[b]) - n_text;

@@ -82,9 +82,13 @@ class LayerWorkload:
                                                   self.seq_off, self.n_vis, self.n_retain)
             return self.last
         if self.prune is not None:
-            self.last = self.h.fmmoe_moe_forward_prune(self.desc, self.ws, self.x, self.mask, self.flags, self.out,
-                                                       self.route, self.pp, self.attn, self.seq_off, self.n_vis,
-                                                       self.n_retain)
+            if getattr(self, "_call", None) is None or self._call_route is not self.route:
+                # marshalled once: the timed loop is one C call per step and allocates nothing
+                self._call = self.h.prepare_forward_prune(self.desc, self.ws, self.x, self.mask, self.flags, self.out,
+                                                          self.route, self.pp, self.attn, self.seq_off, self.n_vis,
+                                                          self.n_retain)
+                self._call_route = self.route
+            self.last = self._call.run()
         else:
             self.h.fmmoe_moe_forward(self.desc, self.ws, self.x, self.mask, self.flags, out=self.out, route=self.route)
         return self.last
@@ -122,12 +126,14 @@ class LayerWorkload:
         self.h.fmmoe_upload_async(sl["x_dev"], self.x_host)
         self.h.fmmoe_upload_async(sl["mask_dev"], self.mask_host)
         if self.prune is not None:
-            r = self.h.fmmoe_moe_forward_prune(self.desc, self.ws, sl["x_dev"], sl["mask_dev"], self.flags, sl["out_dev"],
-                                               self.route, self.pp, self.attn, self.seq_off, self.n_vis, self.n_retain,
-                                               want_aux=False)
+            if sl.get("call") is None:                 # marshalled once per slot: own outputs, own workspace
+                sl["call"] = self.h.prepare_forward_prune(self.desc, self.ws, sl["x_dev"], sl["mask_dev"], self.flags,
+                                                          sl["out_dev"], self.route, self.pp, self.attn, self.seq_off,
+                                                          self.n_vis, self.n_retain, want_aux=False)
+            r = sl["call"].run()
             if sl["pruned_host"] is None or sl["pruned_host"].shape != r["x_out"].shape:
                 sl["pruned_host"] = torch.empty(r["x_out"].shape, dtype=r["x_out"].dtype).pin_memory()
-            sl["pruned_dev"] = r["x_out"]              # stays referenced until the slot's ticket has been waited for
+            sl["pruned_dev"] = r["x_out"]              # owned by the slot's call: rewritten only after the ticket wait
             self.h.fmmoe_download_async(sl["out_host"], sl["out_dev"])
             self.h.fmmoe_download_async(sl["pruned_host"], r["x_out"])
             self.pruned_host = sl["pruned_host"]
@@ -152,6 +158,10 @@ class LayerWorkload:
         if self.pruned_host is not None:
             n += self.pruned_host.numel() * self.pruned_host.element_size()
         return n
+
+    def merged_rows(self) -> int:
+        """Merged windows of the last step's pruning stage (each read W rows and wrote one)."""
+        return int((self.last["kind"] == 2).sum()) if self.last is not None and self.last.get("kind") is not None else 0
 
     def routing_stats(self):
         """(routed pairs P, experts with at least one row) of the last step."""

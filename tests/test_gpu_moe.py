@@ -318,18 +318,36 @@ def _rows_per_expert_case(counts, n_text_extra, H=128, I_=192, seed=41):
     return I.round_to_storage(x, "bf16"), mask, w, E
 
 
-@pytest.mark.parametrize("gather_min", ["0", None])
-def test_rows_per_expert_boundaries_on_both_gemm1_row_paths(gather_min, monkeypatch):
-    """Experts holding 0, 1, 16, 17, 64, 65, 128 and 129 rows (and two with several hundred), EVERY output row
-    against the oracle, on both ways GEMM-1 obtains its routed rows: the expert-ordered copy written by the
-    scatter pass (default at this size) and the in-GEMM gather by token (forced through the handle's threshold,
-    which is otherwise only reached from 12,288 tokens on)."""
-    counts = [0, 1, 16, 17, 64, 65, 128, 129]
+ROW_PATHS = {
+    # name: environment read by fmmoe_create -> which kernels the expert GEMMs run as at this size
+    "small_m": {},                                                        # default below 12,288 tokens: rows as the MMA's N
+    "rows_as_m_copy": {"FMMOE_SMALL_M_MAX_TOKENS": "0"},                  # rows as M, expert-ordered copy of x
+    "rows_as_m_gather": {"FMMOE_SMALL_M_MAX_TOKENS": "0", "FMMOE_GATHER_MIN_TOKENS": "0"},   # rows as M, in-GEMM gather
+    # the combine through per-pair bf16 rows (default from 8,192 tokens on), under both forms
+    "small_m_pair_rows": {"FMMOE_PAIR_ROWS_MIN_TOKENS": "0"},
+    "rows_as_m_gather_pair_rows": {"FMMOE_SMALL_M_MAX_TOKENS": "0", "FMMOE_GATHER_MIN_TOKENS": "0",
+                                   "FMMOE_PAIR_ROWS_MIN_TOKENS": "0"},
+}
+
+
+def handle_with_env(monkeypatch, env):
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    h = B.Handle(0)                                  # the thresholds are read once, when the handle is created
+    for k in env:
+        monkeypatch.delenv(k, raising=False)
+    return h
+
+
+@pytest.mark.parametrize("path", list(ROW_PATHS))
+def test_rows_per_expert_boundaries_on_every_gemm_form(path, monkeypatch):
+    """Experts holding 0, 1, 15, 16, 17, 33, 64, 65, 96, 97, 128 and 129 rows (and two with several hundred), EVERY
+    output row against the oracle, on each form of the expert GEMMs: token rows as the MMA's N dimension (the
+    default below 12,288 tokens), rows as M reading the expert-ordered copy written by the scatter pass, and rows
+    as M with the in-GEMM gather by token (otherwise only reached from 12,288 tokens on)."""
+    counts = [0, 1, 15, 16, 17, 33, 64, 65, 96, 97, 128, 129]
     x, mask, w, E = _rows_per_expert_case(counts, n_text_extra=300)
-    if gather_min is not None:
-        monkeypatch.setenv("FMMOE_GATHER_MIN_TOKENS", gather_min)
-    h = B.Handle(0)                                  # the threshold is read once, when the handle is created
-    monkeypatch.delenv("FMMOE_GATHER_MIN_TOKENS", raising=False)
+    h = handle_with_env(monkeypatch, ROW_PATHS[path])
     T, H = x.shape
     I_ = w["w_gate"].shape[1]
     desc = B.make_desc(H, E, I_, 0, 0, 2, 1, torch.bfloat16)
@@ -345,4 +363,82 @@ def test_rows_per_expert_boundaries_on_both_gemm1_row_paths(gather_min, monkeypa
         ref = O.moe_forward(x, mask, w, 2, 1, True, logits32=host(route["logits"]))
         assert np.array_equal(host(route["topk_idx"]), ref["topk_idx"])
         assert row_rel_err(host(out), ref["out"]) < 2e-2
+    h.close()
+
+
+@pytest.mark.parametrize("T", [1, 7, 16, 40])
+def test_decode_sized_batches_with_shared_experts(T):
+    """A handful of tokens (a decode step): every expert holds 0-3 rows, so each routed tile is one 16-row MMA
+    column block; shared experts and odd feature-block counts (S_m = 192 = 128 + 64) included."""
+    check_layer("bf16", T, 256, 16, 192, 4, 2, 1, 192, flags=B.FLAG_REDUCE_ON, seed=50 + T)
+    check_layer("bf16", T, 128, 8, 64, 2, 1, 0, 0, flags=B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC, seed=60 + T)
+
+
+def test_small_m_form_equals_rows_as_m_form_bit_for_bit_in_fixed_order_mode(monkeypatch):
+    """The two forms of the expert GEMMs accumulate every output element over the same k order in fp32, so with the
+    fixed-order combine their layer outputs are identical bit for bit."""
+    r = np.random.default_rng(71)
+    T, H, E, I_ = 900, 256, 16, 320
+    x = I.round_to_storage(r.standard_normal((T, H)), "bf16")
+    mask = (r.random(T) < 0.7).astype(np.uint8)
+    w = random_layer(r, "bf16", H, E, I_, 1, 128)
+    outs = []
+    for env in (ROW_PATHS["small_m"], ROW_PATHS["rows_as_m_copy"]):
+        h = handle_with_env(monkeypatch, env)
+        desc = B.make_desc(H, E, I_, 1, 128, 4, 2, torch.bfloat16)
+        wd = upload_weights(w, "bf16"); ws = B.make_weights(wd)
+        outs.append(h.fmmoe_moe_forward(desc, ws, dev(x, torch.bfloat16), dev(mask),
+                                        B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC).clone())
+        h.check_status()
+        h.close()
+    assert torch.equal(outs[0], outs[1])
+
+
+@pytest.mark.parametrize("k_block", [0, 5])
+def test_bounded_wait_runs_out_and_the_handle_recovers(k_block):
+    """The producer of GEMM-1 (one CTA, tiny shape) stops before it issues k-block `k_block`; the issuing thread's
+    wait for that stage has a 3 ms budget and nothing will ever complete it.  Expected: the call returns, the kernels
+    finish, fmmoe_get_status reports FMMOE_ERR_TIMEOUT exactly once, and the next ordinary call on the same handle
+    passes parity (tensor memory was released, no barrier is left half-way)."""
+    h = B.Handle(0)
+    r = np.random.default_rng(81)
+    T, H, E, I_ = 96, 512, 4, 128            # H = 512: eight k-blocks per GEMM-1 tile
+    x = I.round_to_storage(r.standard_normal((T, H)), "bf16")
+    mask = (r.random(T) < 0.5).astype(np.uint8)
+    w = random_layer(r, "bf16", H, E, I_, 0, 0)
+    desc = B.make_desc(H, E, I_, 0, 0, 2, 1, torch.bfloat16)
+    wd = upload_weights(w, "bf16"); ws = B.make_weights(wd)
+    xd, md = dev(x, torch.bfloat16), dev(mask)
+    h.fmmoe_test_expire_wait(3_000_000, k_block)
+    h.fmmoe_moe_forward(desc, ws, xd, md, B.FLAG_REDUCE_ON)
+    assert h.get_status() == 5                # FMMOE_ERR_TIMEOUT, read and cleared
+    assert h.get_status() == 0
+    route = {"logits": torch.empty(T, E, dtype=torch.float32, device="cuda")}
+    out = h.fmmoe_moe_forward(desc, ws, xd, md, B.FLAG_REDUCE_ON, route=route)
+    h.check_status()
+    ref = O.moe_forward(x, mask, w, 2, 1, True, logits32=host(route["logits"]))
+    assert row_rel_err(host(out), ref["out"]) < 2e-2
+    h.close()
+
+
+@pytest.mark.parametrize("path", ["small_m_pair_rows", "rows_as_m_gather_pair_rows"])
+def test_pair_row_combine_with_shared_experts_residual_and_reproducibility(path, monkeypatch):
+    """The combine through per-pair bf16 rows: shared experts, residual, K_v = 0 tokens, against the oracle within
+    the bf16 tolerance; it sums in a fixed order without atomics, so two runs agree bit for bit."""
+    h = handle_with_env(monkeypatch, ROW_PATHS[path])
+    r = np.random.default_rng(91)
+    T, H, E, I_, Ns, Is, K, Kv = 700, 256, 16, 192, 2, 128, 4, 0
+    x = I.round_to_storage(r.standard_normal((T, H)), "bf16")
+    mask = (r.random(T) < 0.6).astype(np.uint8)
+    w = random_layer(r, "bf16", H, E, I_, Ns, Is)
+    desc = B.make_desc(H, E, I_, Ns, Is, K, Kv, torch.bfloat16)
+    wd = upload_weights(w, "bf16"); ws = B.make_weights(wd)
+    route = {"logits": torch.empty(T, E, dtype=torch.float32, device="cuda")}
+    flags = B.FLAG_REDUCE_ON | B.FLAG_RESIDUAL
+    a = h.fmmoe_moe_forward(desc, ws, dev(x, torch.bfloat16), dev(mask), flags, route=route).clone()
+    b = h.fmmoe_moe_forward(desc, ws, dev(x, torch.bfloat16), dev(mask), flags, route=route)
+    h.check_status()
+    assert torch.equal(a, b)
+    ref = O.moe_forward(x, mask, w, K, Kv, True, add_residual=True, logits32=host(route["logits"]))
+    assert row_rel_err(host(a), ref["out"]) < 2e-2
     h.close()
