@@ -1,7 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the FastMMoE MoE-layer hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload all|C0|C1|C2|C2x4|C3|C4] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload all|C0|C1|C2|C2x4|C3|C4|C1_fp8|C2_fp8|C3_fp8]
+                    [--impl reference]
 
 One "step" = one pass of the whole hot path over one batch of synthetic tokens:
 router + top-k + gates, permute-by-expert, grouped SwiGLU expert GEMMs + shared
@@ -12,7 +13,8 @@ is the whole stack (fmmoe_stack_forward).
 The default (`--workload all`) prints ONE JSON line whose top-level fields are the
 largest single-layer workload (the batch of four Qwen3-MoE-style sequences, 14,336
 tokens) and whose `configs` object holds one record per other workload (C0, C1, C2,
-C3, C4), each with its own timing, clocks, roofline and end-to-end figure.
+C3, C4, and C1-C3 once more with their expert matrices stored as FP8), each with its
+own timing, clocks, roofline and end-to-end figure.
 
 Timing: a block is exactly K steps between two CUDA events, with a barrier and a
 device synchronisation on both sides.  Whatever K is, blocks are repeated until the
@@ -39,7 +41,7 @@ import numpy as np  # noqa: E402
 METRIC = "MoE-layer prefill tokens/s"
 UNIT = "tokens/s"
 LAYER_WORKLOADS = ("C0", "C1", "C2", "C2x4", "C3")
-WORKLOADS = ("all",) + LAYER_WORKLOADS + ("C4",)
+WORKLOADS = ("all",) + LAYER_WORKLOADS + ("C1_fp8", "C2_fp8", "C3_fp8", "C4")
 HEADLINE = "C2x4"
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # the nominal peaks the metric names (8 TB/s, dense bf16)
 
@@ -90,17 +92,18 @@ def weight_bytes(cfg):
 
 
 # ------------------------------------------------------------------ algorithmic work per launch
-def kernel_work(cfg, kernel, P, touched, prune_rows=None):
+def kernel_work(cfg, kernel, P, touched, prune_rows=None, w_elem=None):
     """(bytes, flops) one launch of `kernel` must move / compute for this workload.
     P = routed pairs, touched = experts with at least one row, prune_rows = (rows read, rows written) of the
-    compaction pass."""
+    compaction pass, w_elem = bytes per stored expert-matrix element (1 for the FP8 weight stream)."""
     e = 2 if cfg.dtype == "bf16" else 4
+    we = e if w_elem is None else w_elem
     T, H, E, I_, Ns, Is, K = cfg.n_tokens, cfg.hidden, cfg.n_experts, cfg.inter, cfg.n_shared, cfg.shared_inter, cfg.top_k
     if kernel == "gemm1":
-        b = touched * 2 * H * I_ * e + Ns * 2 * H * Is * e + T * H * e + (P * I_ + Ns * T * Is) * e
+        b = touched * 2 * H * I_ * we + Ns * 2 * H * Is * we + T * H * e + (P * I_ + Ns * T * Is) * e
         f = 4 * H * I_ * P + 4 * H * Is * Ns * T
     elif kernel == "gemm2":
-        b = touched * H * I_ * e + Ns * H * Is * e + (P * I_ + Ns * T * Is) * e + T * H * e
+        b = touched * H * I_ * we + Ns * H * Is * we + (P * I_ + Ns * T * Is) * e + T * H * e
         f = 2 * H * I_ * P + 2 * H * Is * Ns * T
     elif kernel == "route":
         b = T * H * e + E * H * e + T * K * 8 + T * E * 4
@@ -368,15 +371,22 @@ def roofline_of(kernel, b, f, per_launch_s, peaks, traffic):
     return roof
 
 
-def measure_layer(name, args, D, rank, local, world, peaks, with_cpu):
+def measure_layer(name, args, D, rank, local, world, peaks, with_cpu, fp8=False):
     import torch
     from paper_2511_17885_b200 import binding as B
     from paper_2511_17885_b200.workload import LayerWorkload
     dev = f"cuda:{local}"
     cfg, prune = workload_cfg(name)
     h = B.Handle(local)
-    wl = LayerWorkload(cfg, h, device=local, prune=prune, token_seed=D.token_seed_for_rank(cfg.seed, rank))
+    wl = LayerWorkload(cfg, h, device=local, prune=prune, token_seed=D.token_seed_for_rank(cfg.seed, rank),
+                       fp8_weights=fp8)
     K, W = max(args.steps, 1), max(args.warmup, 3)
+    if args.plain:      # for profilers: warm-up and K steps of the device-resident path, nothing else
+        for _ in range(args.warmup + K):
+            wl.step()
+        torch.cuda.synchronize()
+        h.check_status("plain run")
+        return {"value": 0.0, "ms_per_step": 0.0, "dtype": cfg.dtype, "config": describe(name, cfg, prune), "plain": True}
     for _ in range(W):
         wl.step()
     settle_s = settle_clocks(wl.step, local)
@@ -456,6 +466,7 @@ def measure_layer(name, args, D, rank, local, world, peaks, with_cpu):
     clocks.stop()
 
     # ---- rooflines
+    w_elem = 1 if fp8 else None
     t_out = int(wl.last["x_out"].shape[0]) if wl.last is not None else 0
     merged = wl.merged_rows() if wl.last is not None else 0
     prune_rows = (t_out + merged * (prune.window - 1), t_out)
@@ -465,7 +476,7 @@ def measure_layer(name, args, D, rank, local, world, peaks, with_cpu):
         if not v["launches"]:
             continue
         per_launch_s = v["ms"] * 1e-3 / v["launches"]
-        b, f = kernel_work(cfg, k, P, touched, prune_rows)
+        b, f = kernel_work(cfg, k, P, touched, prune_rows, w_elem)
         kernels[k] = {"us_per_launch": per_launch_s * 1e6, "launches_per_step": v["launches"] / kp,
                       "us_per_step": v["ms"] * 1e3 / kp, "share": v["ms"] / tot_ms,
                       "algorithmic_bytes": b, "hbm_gbs": b / per_launch_s / 1e9 if b else None,
@@ -473,17 +484,21 @@ def measure_layer(name, args, D, rank, local, world, peaks, with_cpu):
                       "tensor_tflops": f / per_launch_s / 1e12 if f else None}
     dom = max(prof, key=lambda k: prof[k]["ms"])
     per_launch_s = prof[dom]["ms"] * 1e-3 / max(prof[dom]["launches"], 1)
-    b, f = kernel_work(cfg, dom, P, touched, prune_rows)
+    b, f = kernel_work(cfg, dom, P, touched, prune_rows, w_elem)
     roof = roofline_of(dom, b, f, per_launch_s, peaks, NCU_TRAFFIC_BYTES.get(name, {}).get(dom))
     # whole step against the slower of (activated FLOPs at tensor peak, algorithmic bytes at HBM bandwidth)
     e = 2 if cfg.dtype == "bf16" else 4
-    tot_b = sum(kernel_work(cfg, k, P, touched)[0] for k in ("route", "gemm1", "gemm2")) - 2 * cfg.n_tokens * cfg.hidden * e
+    tot_b = sum(kernel_work(cfg, k, P, touched, None, w_elem)[0] for k in ("route", "gemm1", "gemm2")) - 2 * cfg.n_tokens * cfg.hidden * e
     tot_f = sum(kernel_work(cfg, k, P, touched)[1] for k in ("route", "gemm1", "gemm2"))
     t_hbm, t_tc = tot_b / (peaks["hbm_gbs"] * 1e9), tot_f / (peaks["tf_sustained"] * 1e12)
     t_step = max(t_hbm, t_tc)
     t_step_nom = max(tot_b / (NOMINAL["hbm_gbs"] * 1e9), tot_f / (NOMINAL["bf16_tflops"] * 1e12))
 
     conf = describe(name, cfg, prune)
+    if fp8:
+        conf["workload"] += ("; expert matrices stored as FP8 E4M3 bytes with one power-of-two scale per 128x128 block "
+                             "(activations, accumulation and outputs as in the bf16 layer)")
+        conf["l2"] = conf["l2"].replace(f"({weight_bytes(cfg) / 1e6:.0f} MB)", f"({weight_bytes(cfg) / 2e6:.0f} MB as FP8)")
     conf.update({"routed_pairs": P, "experts_touched": touched, "parallelism": f"replicas x{world} (no collective)"})
     rec = {"value": value, "unit": UNIT, "ms_per_step": step_s * 1e3, "timing": stats, "dtype": cfg.dtype,
            "config": conf,
@@ -568,6 +583,12 @@ def measure_stack(args, D, rank, local, world, peaks, with_cpu):
     h = B.Handle(local)
     wl = StackWorkload(sc, h, device=local, token_seed=D.token_seed_for_rank(sc.layer.seed, rank), n_layers=n_layers)
     K, W = max(1, min(args.steps, 10)), max(args.warmup, 3)      # a stack step is 24 layers: at most 10 per block
+    if args.plain:      # for profilers
+        for _ in range(args.warmup + K):
+            wl.step()
+        torch.cuda.synchronize()
+        h.check_status("plain run")
+        return {"value": 0.0, "ms_per_step": 0.0, "dtype": sc.layer.dtype, "config": stack_describe(sc, n_layers), "plain": True}
     for _ in range(min(W, 5)):
         wl.step()
     settle_s = settle_clocks(wl.step, local, min_s=0.2)
@@ -719,15 +740,19 @@ def run_ours(args):
     peaks = load_peaks()
     head = HEADLINE if args.workload == "all" else args.workload
     others = [w for w in ("C0", "C1", "C2", "C3", "C4") if w != head] if args.workload == "all" else []
-    with_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
+    with_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline and not args.plain
 
     def measure(name, cpu):
         if name == "C4":
             return measure_stack(args, D, rank, local, world, peaks, cpu)
+        if name.endswith("_fp8"):
+            return measure_layer(name[:-4], args, D, rank, local, world, peaks, cpu, fp8=True)
         return measure_layer(name, args, D, rank, local, world, peaks, cpu)
 
     rec = measure(head, with_cpu)
     configs = {}
+    if args.workload == "all":     # the weight-stream-bound workloads once more with FP8 expert weights
+        others = others[:-1] + ["C1_fp8", "C2_fp8", "C3_fp8"] + others[-1:]
     for name in others:
         configs[name] = measure(name, False)
     if rank == 0:
@@ -755,6 +780,8 @@ def main():
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="timed GPU work per workload and per region: blocks of --steps steps are repeated until it is reached")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--plain", action="store_true",
+                    help="run --warmup + --steps steps of the device-resident path and exit (what a profiler is pointed at)")
     ap.add_argument("--layers", type=int, default=0, help="C4 only: run the first N layers of the stack")
     ap.add_argument("--no-dense", action="store_true", help="C4 only: skip the unreduced, unpruned comparison run")
     args = ap.parse_args()

@@ -45,6 +45,19 @@ typedef enum {
 
 typedef enum { FMMOE_F32 = 0, FMMOE_BF16 = 1 } fmmoe_dtype;
 
+/* Storage format of the expert matrices (w_gate, w_up, w_down and the shared experts').
+ * FMMOE_WEIGHTS_FP8_BLOCK128 halves the weight stream that bounds a prefill at small batch
+ * (Section 3.1 leaves a few dozen rows per expert; Appendix E: the compressed prefill is
+ * memory-bound): every matrix element is one FP8 E4M3 byte (1 sign, 4 exponent bits with
+ * bias 7, 3 mantissa bits, subnormals, largest magnitude 448; the NaN encodings 0x7f / 0xff
+ * must not occur), and every block of 128 x 128 elements of a matrix [rows, cols] (the last
+ * block of a dimension may be partial) shares one power-of-two scale, stored as its exponent:
+ *   value(r, c) = e4m3(byte[r][c]) * 2^scale_exp[r / 128][c / 128],   -100 <= scale_exp <= 7.
+ * A power of two keeps the conversion to bf16 exact (an E4M3 value has 4 significant bits),
+ * so the layer computes with exactly these values: activations, accumulation and outputs are
+ * as in the bf16 layer.  Requires dtype == FMMOE_BF16; the router matrix stays bf16. */
+typedef enum { FMMOE_WEIGHTS_AS_DTYPE = 0, FMMOE_WEIGHTS_FP8_BLOCK128 = 1 } fmmoe_weight_format;
+
 /* Limits of the kernels. */
 #define FMMOE_MAX_EXPERTS 256
 #define FMMOE_MAX_TOPK 16
@@ -66,6 +79,7 @@ typedef struct {
   int32_t top_k;         /* K, 1..FMMOE_MAX_TOPK                                 */
   int32_t top_k_vis;     /* K_v = pK, 0..K; 0 only if n_shared > 0 (Section 3.1) */
   int32_t dtype;         /* fmmoe_dtype of x, out and all expert/router weights  */
+  int32_t weight_format; /* fmmoe_weight_format of the expert matrices           */
 } fmmoe_layer_desc;
 
 /* Layer parameters (device, read-only).  nn.Linear layout: [out_features, in_features]. */
@@ -78,6 +92,15 @@ typedef struct {
   const void  *ws_gate;   /* [N_s, S_s, H] or NULL                                          */
   const void  *ws_up;     /* [N_s, S_s, H] or NULL                                          */
   const void  *ws_down;   /* [N_s, H, S_s] or NULL                                          */
+  /* FMMOE_WEIGHTS_FP8_BLOCK128 only (else ignored): the matrices above hold one byte per element
+   * and these hold the block scale exponents, int8, row-major, per expert
+   * [ceil(rows/128), ceil(cols/128)] of that expert's [rows, cols] matrix:                      */
+  const int8_t *w_gate_scale;   /* [E, ceil(S_m/128), ceil(H/128)]                                */
+  const int8_t *w_up_scale;     /* [E, ceil(S_m/128), ceil(H/128)]                                */
+  const int8_t *w_down_scale;   /* [E, ceil(H/128), ceil(S_m/128)]                                */
+  const int8_t *ws_gate_scale;  /* [N_s, ceil(S_s/128), ceil(H/128)] or NULL                      */
+  const int8_t *ws_up_scale;    /* [N_s, ceil(S_s/128), ceil(H/128)] or NULL                      */
+  const int8_t *ws_down_scale;  /* [N_s, ceil(H/128), ceil(S_s/128)] or NULL                      */
 } fmmoe_weights;
 
 /* Optional routing outputs (device).  Any pointer may be NULL = not wanted. */
@@ -138,7 +161,9 @@ fmmoe_status fmmoe_route(fmmoe_handle *handle, const fmmoe_layer_desc *desc, con
  * SwiGLU activations once to bf16; fp32 layers use fp32 FMA throughout.
  * out: [T, H] dtype, must not alias x.  `route` (may be NULL) receives the
  * routing record of the call.  bf16 requires H % 64 == 0, S_m % 64 == 0,
- * S_s % 64 == 0. */
+ * S_s % 64 == 0.  With FMMOE_WEIGHTS_FP8_BLOCK128 the expert matrices are streamed as FP8 bytes,
+ * expanded to bf16 in shared memory (exactly) and fed to the same tensor-core contraction; it
+ * additionally requires H % 128 == 0, S_m % 128 == 0 and S_s % 128 == 0. */
 fmmoe_status fmmoe_moe_forward(fmmoe_handle *handle, const fmmoe_layer_desc *desc, const fmmoe_weights *w,
                                const void *x, const uint8_t *is_visual, int64_t n_tokens, uint32_t flags,
                                void *out, const fmmoe_route_out *route, void *workspace,

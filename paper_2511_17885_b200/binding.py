@@ -26,12 +26,14 @@ STATIC_PRUNE_MAX_TOKENS = 32768
 
 class LayerDesc(C.Structure):
     _fields_ = [("hidden", C.c_int32), ("n_experts", C.c_int32), ("inter", C.c_int32), ("n_shared", C.c_int32),
-                ("shared_inter", C.c_int32), ("top_k", C.c_int32), ("top_k_vis", C.c_int32), ("dtype", C.c_int32)]
+                ("shared_inter", C.c_int32), ("top_k", C.c_int32), ("top_k_vis", C.c_int32), ("dtype", C.c_int32),
+                ("weight_format", C.c_int32)]
 
 
 class Weights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
-                ("router_w", "router_b", "w_gate", "w_up", "w_down", "ws_gate", "ws_up", "ws_down")]
+                ("router_w", "router_b", "w_gate", "w_up", "w_down", "ws_gate", "ws_up", "ws_down",
+                 "w_gate_scale", "w_up_scale", "w_down_scale", "ws_gate_scale", "ws_up_scale", "ws_down_scale")]
 
 
 class RouteOut(C.Structure):
@@ -159,8 +161,13 @@ def fmmoe_workspace_bytes(desc: LayerDesc, n_tokens: int, flags: int = 0) -> int
     return int(lib().fmmoe_workspace_bytes(C.byref(desc), n_tokens, flags))
 
 
-def make_desc(hidden, n_experts, inter, n_shared, shared_inter, top_k, top_k_vis, dtype: torch.dtype) -> LayerDesc:
-    return LayerDesc(hidden, n_experts, inter, n_shared, shared_inter, top_k, top_k_vis, _dtype_code(dtype))
+WEIGHTS_AS_DTYPE, WEIGHTS_FP8_BLOCK128 = 0, 1
+
+
+def make_desc(hidden, n_experts, inter, n_shared, shared_inter, top_k, top_k_vis, dtype: torch.dtype,
+              weight_format: int = WEIGHTS_AS_DTYPE) -> LayerDesc:
+    return LayerDesc(hidden, n_experts, inter, n_shared, shared_inter, top_k, top_k_vis, _dtype_code(dtype),
+                     weight_format)
 
 
 def make_stages(stages) -> "C.Array":

@@ -18,6 +18,8 @@ static bool desc_ok(const fmmoe_layer_desc* d) {
   if (d->top_k_vis < 0 || d->top_k_vis > d->top_k) return false;
   if (d->top_k_vis == 0 && d->n_shared == 0) return false;   // p = 0 needs shared experts (Section 3.1)
   if (d->dtype != FMMOE_F32 && d->dtype != FMMOE_BF16) return false;
+  if (d->weight_format != FMMOE_WEIGHTS_AS_DTYPE && d->weight_format != FMMOE_WEIGHTS_FP8_BLOCK128) return false;
+  if (d->weight_format == FMMOE_WEIGHTS_FP8_BLOCK128 && d->dtype != FMMOE_BF16) return false;
   return true;
 }
 
@@ -27,6 +29,9 @@ static fmmoe_status shape_supported(const fmmoe_layer_desc& d, bool forward) {
   if (d.dtype == FMMOE_BF16) {
     if (d.hidden % 64) return FMMOE_ERR_UNSUPPORTED;
     if (forward && (d.inter % 64 || (d.n_shared && d.shared_inter % 64))) return FMMOE_ERR_UNSUPPORTED;
+    if (forward && d.weight_format == FMMOE_WEIGHTS_FP8_BLOCK128 &&
+        (d.hidden % 128 || d.inter % 128 || (d.n_shared && d.shared_inter % 128)))
+      return FMMOE_ERR_UNSUPPORTED;
   } else if (forward && (d.hidden % 4 || d.inter % 4 || (d.n_shared && d.shared_inter % 4))) {
     return FMMOE_ERR_UNSUPPORTED;
   }
@@ -105,6 +110,10 @@ static fmmoe_status check_common(fmmoe_handle* h, const fmmoe_layer_desc* d, con
       if (!w->ws_gate || !w->ws_up || !w->ws_down) return FMMOE_ERR_INVALID_ARG;
       if (!aligned16(w->ws_gate) || !aligned16(w->ws_up) || !aligned16(w->ws_down)) return FMMOE_ERR_INVALID_ARG;
     }
+    if (d->weight_format == FMMOE_WEIGHTS_FP8_BLOCK128) {
+      if (!w->w_gate_scale || !w->w_up_scale || !w->w_down_scale) return FMMOE_ERR_INVALID_ARG;
+      if (d->n_shared && (!w->ws_gate_scale || !w->ws_up_scale || !w->ws_down_scale)) return FMMOE_ERR_INVALID_ARG;
+    }
   }
   return FMMOE_OK;
 }
@@ -174,7 +183,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
     if (end != g && v >= 0) h->gather_min_tokens = v;
   }
   h->wait_budget_ns = 2000000000ull;
-  h->sm_attr_set = false;
+  h->sm_attr_set = false; h->smq_attr_set = false;
   h->small_m_max_tokens = kGatherMinTokensDefault;
   if (const char* g = getenv("FMMOE_SMALL_M_MAX_TOKENS")) {
     char* end = nullptr;
@@ -287,7 +296,7 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   // the router clears the scheduler words and (atomic mode) the fp32 accumulator it owns rows of
   // bf16 at small batch: the permutation's scatter pass also writes the expert-grouped copy of x
   const bool pair = use_pair_rows(h, *d, T, flags);
-  const bool copy_rows = d->dtype == FMMOE_BF16 && (use_small_m(h, T) || !gather_rows_in_gemm(h, T));
+  const bool copy_rows = d->dtype == FMMOE_BF16 && (use_small_m(h, *d, T) || !gather_rows_in_gemm(h, T));
   st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, (det || pair) ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s,
                  copy_rows ? ws + pl.xp_off : nullptr);
   if (st != FMMOE_OK) return st;
@@ -310,7 +319,7 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   fa.ysh = det ? reinterpret_cast<float*>(ws + pl.ysh_off) : nullptr;
   fa.deterministic = det; fa.d_status = h->d_status;
   fa.test_withhold_stage = -1; fa.grid_override = 0;
-  if (d->dtype == FMMOE_BF16 && use_small_m(h, T)) {
+  if (use_small_m(h, *d, T)) {
     const uint64_t budget = h->wait_budget_ns;
     if (h->test_withhold_stage >= 0) {     // armed self-test: this call only
       fa.test_withhold_stage = h->test_withhold_stage; fa.grid_override = 1;

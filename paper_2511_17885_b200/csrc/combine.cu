@@ -16,8 +16,7 @@ struct FinalizeDev {
   const __nv_bfloat16* yb; const __nv_bfloat16* ybsh;
 };
 
-__device__ __forceinline__ void add_bf16x8(float (&v)[8], const __nv_bfloat16* p) {
-  const uint4 u = *reinterpret_cast<const uint4*>(p);
+__device__ __forceinline__ void add_bf16x8(float (&v)[8], const uint4 u) {
   const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -36,18 +35,27 @@ __global__ void __launch_bounds__(256) finalize_pair_kernel(const FinalizeDev a)
   pdl_wait();
   const int hv = a.H / 8;
   const long long n = a.T * hv;
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);    // eight bf16 zeros
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
     const long long t = i / hv;
     const int c = (int)(i - t * hv) * 8;
+    // every row index first, then every row piece (independent 16-byte loads in flight together), then the sum
+    int rows[FMMOE_MAX_TOPK];
+#pragma unroll
+    for (int s = 0; s < FMMOE_MAX_TOPK; ++s) rows[s] = s < a.K ? a.inv_row[t * a.K + s] : -1;
+    uint4 q[FMMOE_MAX_TOPK];
+#pragma unroll
+    for (int s = 0; s < FMMOE_MAX_TOPK; ++s)
+      q[s] = rows[s] >= 0 ? *reinterpret_cast<const uint4*>(a.yb + (long long)rows[s] * a.H + c) : zero;
     float v[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) v[j] = 0.f;
-    for (int s = 0; s < a.K; ++s) {
-      const int row = a.inv_row[t * a.K + s];
-      if (row >= 0) add_bf16x8(v, a.yb + (long long)row * a.H + c);
-    }
-    for (int s = 0; s < a.n_shared; ++s) add_bf16x8(v, a.ybsh + ((long long)s * a.T + t) * a.H + c);
-    if (a.add_residual) add_bf16x8(v, static_cast<const __nv_bfloat16*>(a.x) + t * a.H + c);
+#pragma unroll
+    for (int s = 0; s < FMMOE_MAX_TOPK; ++s)
+      if (s < a.K) add_bf16x8(v, q[s]);          // adding the zeros of an unused slot changes nothing
+    for (int s = 0; s < a.n_shared; ++s)
+      add_bf16x8(v, *reinterpret_cast<const uint4*>(a.ybsh + ((long long)s * a.T + t) * a.H + c));
+    if (a.add_residual) add_bf16x8(v, *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(a.x) + t * a.H + c));
     uint32_t w[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {

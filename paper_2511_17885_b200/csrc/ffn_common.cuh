@@ -43,6 +43,7 @@ struct GemmParams {
   int pair;                   // MODE 1: write yb instead of reducing into acc
   int gather;                 // MODE 0: routed rows come from x through the loader warps (else from the tmA_r map)
   int* status;
+  const int8_t* wscale[2][2];          // FP8 weight stream: block scale exponents, [segment][weight box of the stage]
   unsigned long long wait_budget_ns;   // time budget of every bounded wait (ffn_sm.cu)
   int test_withhold_stage;             // self-test: the producer stops before this k-block (-1: never)
 };
@@ -116,5 +117,19 @@ static inline bool make_map(fmmoe_handle* h, CUtensorMap* m, const void* base, u
   return r == CUDA_SUCCESS;
 }
 
+
+// FP8 bytes, row-major [rows, cols], box = 64 bytes x box_rows rows, no swizzle (read by threads, not by the MMA).
+static inline bool make_map_u8(fmmoe_handle* h, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  if (rows == 0) rows = 1;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(h->encode_tiled)(
+      m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
 
 }  // namespace fmmoe

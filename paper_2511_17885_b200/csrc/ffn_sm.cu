@@ -18,6 +18,12 @@
 //           token to the fp32 accumulator with one 128-byte reduction (or stores them, fixed-order mode).
 // The transposed accumulator needs no shared-memory staging: for a fixed token the lanes of a warp already
 // hold consecutive output features.
+// FP8 weight stream (WQ = 1): the expert matrices arrive as FP8 E4M3 bytes with one power-of-two scale per
+// 128 x 128 block.  TMA brings the bytes (half the HBM traffic of bf16) into a ring of raw stages; eight more
+// warps expand every weight box to bf16 in the 128-byte-swizzled layout the MMA reads (exactly: an E4M3 value
+// has 4 significant bits and the scale is a power of two) into a second, two-deep ring; the activations stay
+// bf16 and go from the raw stage straight to the MMA.  The contraction, the accumulators and the epilogues are
+// those of the bf16 stream.
 // Every wait is bounded; on expiry the CTA records FMMOE_ERR_TIMEOUT and leaves.
 #include <cuda_bf16.h>
 
@@ -29,12 +35,37 @@ namespace fmmoe {
 
 constexpr int S_BK = 64;                              // one 128-byte swizzle atom of bf16
 constexpr int S_STAGES = 4;
-constexpr int S_W_BYTES = 128 * S_BK * 2;             // one 128-feature weight box: 16 KB
+constexpr int S_W_BYTES = 128 * S_BK * 2;             // one 128-feature weight box as bf16: 16 KB
+constexpr int S_WQ_BYTES = 128 * S_BK;                // the same box as FP8 bytes: 8 KB
 constexpr int S_X_BYTES = 128 * S_BK * 2;             // room for up to 128 token rows: 16 KB
-constexpr int S_STAGE_BYTES = 2 * S_W_BYTES + S_X_BYTES;
 constexpr int S_THREADS = 192;                        // scheduler/producer warp, issuer warp, four epilogue warps
+constexpr int S_CONVERTERS = 256;                     // FP8 stream: eight more warps that expand the weight boxes
+constexpr int S_CVT_PIECES = 512 / S_CONVERTERS;      // 16-byte pieces of a weight box per converter thread
+constexpr int S_CVT_STAGES = 2;
 constexpr int S_TMEM_COLS = 512;                      // 2 accumulator stages x (2 x 128 columns)
-constexpr int S_SMEM_BYTES = S_STAGES * S_STAGE_BYTES + 1024 /*align*/ + 512 /*barriers, tile ring*/;
+// bf16 stream: a stage is [W0 16K][W1 16K][X 16K].  FP8 stream: a raw stage is [W0 8K][W1 8K][X 16K] and the
+// expanded weights live in S_CVT_STAGES buffers of [W0 16K][W1 16K].
+template <int WQ> struct SmLayout {
+  static constexpr int W_RAW = WQ ? S_WQ_BYTES : S_W_BYTES;
+  static constexpr int X_OFF = 2 * W_RAW;
+  static constexpr int STAGE_BYTES = X_OFF + S_X_BYTES;
+  static constexpr int CVT_OFF = S_STAGES * STAGE_BYTES;
+  static constexpr int CVT_BYTES = WQ ? S_CVT_STAGES * 2 * S_W_BYTES : 0;
+  static constexpr int BAR_OFF = CVT_OFF + CVT_BYTES;
+  static constexpr int SMEM_BYTES = BAR_OFF + 1024 /*align*/ + 512 /*barriers, tile ring*/;
+  static constexpr int THREADS = WQ ? S_THREADS + S_CONVERTERS : S_THREADS;
+};
+
+// Two E4M3 bytes (bytes 2*sel and 2*sel+1 of w) -> two bf16 in one word, times `mul` (a power of two in both
+// halves).  An E4M3 byte s.eeee.mmm placed as s.0000eeee.mmm0000 is the bf16 number 2^(e-127) (1 + m/8), or the
+// bf16 subnormal 2^-126 (m/8) for e = 0: in both cases the E4M3 value times 2^-120, so one exact bf16 multiply
+// by 2^(120 + scale exponent) finishes the conversion.
+__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t w, int sel, __nv_bfloat162 mul) {
+  const uint32_t y = __byte_perm(w, 0u, sel ? 0x3424u : 0x1404u);     // [b_lo << 8 | b_hi << 24]
+  const uint32_t bits = (y & 0x80008000u) | ((y >> 4) & 0x07f007f0u);
+  const __nv_bfloat162 v = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&bits), mul);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
 
 __device__ __forceinline__ void red_add_f32(float* addr, float v) {
   asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
@@ -44,8 +75,8 @@ __device__ __forceinline__ void red_add_f32(float* addr, float v) {
 __device__ __forceinline__ int n_pad_of(int rows) { return rows <= 16 ? 16 : (rows + 15) & ~15; }
 
 // MODE 0: GEMM-1 + SwiGLU.  MODE 1: GEMM-2 + combine.
-template <int MODE>
-__global__ void __launch_bounds__(S_THREADS, 1)
+template <int MODE, int WQ>
+__global__ void __launch_bounds__(SmLayout<WQ>::THREADS, 1)
 ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__ CUtensorMap tmX64,
               const __grid_constant__ CUtensorMap tmX96, const __grid_constant__ CUtensorMap tmX128,
               const __grid_constant__ CUtensorMap tmXs,
@@ -55,14 +86,18 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   unsigned char* smem = smem_raw + ((1024 - (raw & 1023)) & 1023);   // 1024-byte aligned tiles (128B swizzle)
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S_STAGES * S_STAGE_BYTES);
+  using L = SmLayout<WQ>;
+  constexpr int S_STAGE_BYTES = L::STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
   uint64_t* full_bar = bars;                   // [S_STAGES]
   uint64_t* empty_bar = bars + S_STAGES;       // [S_STAGES]
   uint64_t* tfull_bar = bars + 2 * S_STAGES;   // [2]
   uint64_t* tempty_bar = tfull_bar + 2;        // [2]
   uint64_t* sfull_bar = tempty_bar + 2;        // [G_SCHED]
   uint64_t* sempty_bar = sfull_bar + G_SCHED;  // [G_SCHED]
-  volatile int* ring = reinterpret_cast<volatile int*>(sempty_bar + G_SCHED);   // [G_SCHED][G_SLOT_INTS]
+  uint64_t* cfull_bar = sempty_bar + G_SCHED;  // [S_CVT_STAGES]  FP8 stream: expanded weights ready
+  uint64_t* cempty_bar = cfull_bar + S_CVT_STAGES;   // [S_CVT_STAGES]
+  volatile int* ring = reinterpret_cast<volatile int*>(cempty_bar + S_CVT_STAGES);   // [G_SCHED][G_SLOT_INTS]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(ring) + G_SCHED * G_SLOT_INTS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -71,9 +106,13 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
   pdl_launch_dependents();
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < S_STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
+    // a raw stage is free again once the MMAs have read its activations and (FP8 stream) every converter
+    // thread has read its weight bytes
+    for (int i = 0; i < S_STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], WQ ? 1 + S_CONVERTERS : 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&tfull_bar[i], 1); mbar_init(&tempty_bar[i], 128); }
-    for (int i = 0; i < G_SCHED; ++i) { mbar_init(&sfull_bar[i], 1); mbar_init(&sempty_bar[i], 5); }   // issuer + 4 epilogue warps
+    // readers of a tile id: issuer + 4 epilogue warps (+ the converter warps)
+    for (int i = 0; i < G_SCHED; ++i) { mbar_init(&sfull_bar[i], 1); mbar_init(&sempty_bar[i], WQ ? 5 + S_CONVERTERS / 32 : 5); }
+    for (int i = 0; i < S_CVT_STAGES; ++i) { mbar_init(&cfull_bar[i], S_CONVERTERS); mbar_init(&cempty_bar[i], 1); }
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -149,15 +188,16 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
           }
           ++issued;
           unsigned char* sW = smem + stage * S_STAGE_BYTES;
-          mbar_arrive_expect_tx(&full_bar[stage], 2u * S_W_BYTES + x_bytes);
+          mbar_arrive_expect_tx(&full_bar[stage], 2u * L::W_RAW + x_bytes);
+          // the weight maps count columns in elements: bf16 elements, or FP8 bytes
           if (stream_w) {
             tma_load_2d_hint(sW, mW0, &full_bar[stage], kb * S_BK, w_y0, pol_stream);
-            tma_load_2d_hint(sW + S_W_BYTES, mW1, &full_bar[stage], kb * S_BK, w_y1, pol_stream);
+            tma_load_2d_hint(sW + L::W_RAW, mW1, &full_bar[stage], kb * S_BK, w_y1, pol_stream);
           } else {
             tma_load_2d(sW, mW0, &full_bar[stage], kb * S_BK, w_y0);
-            tma_load_2d(sW + S_W_BYTES, mW1, &full_bar[stage], kb * S_BK, w_y1);
+            tma_load_2d(sW + L::W_RAW, mW1, &full_bar[stage], kb * S_BK, w_y1);
           }
-          tma_load_2d(sW + 2 * S_W_BYTES, mX, &full_bar[stage], kb * S_BK, x_row);
+          tma_load_2d(sW + L::X_OFF, mX, &full_bar[stage], kb * S_BK, x_row);
           if (++stage == S_STAGES) { stage = 0; phase ^= 1; }
         }
         if (!ok || stop) break;
@@ -170,6 +210,7 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       int as = 0; uint32_t aphase = 0;
+      int cs = 0; uint32_t cphase = 0;
       bool ok = true;
       for (uint32_t it = 0; ok; ++it) {
         const int slot = it % G_SCHED;
@@ -187,11 +228,13 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
         const uint32_t d0 = tmem_base + as * 256, d1 = d0 + 128;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(&full_bar[stage], phase, abort_flag, budget)) { ok = false; break; }
+          if (WQ && !mbar_wait(&cfull_bar[cs], cphase, abort_flag, budget)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sW = smem_u32(smem + stage * S_STAGE_BYTES);
+          const uint32_t sS = smem_u32(smem + stage * S_STAGE_BYTES);
+          const uint32_t sW = WQ ? smem_u32(smem + L::CVT_OFF + cs * 2 * S_W_BYTES) : sS;
           const uint64_t dw0 = umma_desc_sw128(sW);
           const uint64_t dw1 = umma_desc_sw128(sW + S_W_BYTES);
-          const uint64_t dx = umma_desc_sw128(sW + 2 * S_W_BYTES);
+          const uint64_t dx = umma_desc_sw128(sS + L::X_OFF);
 #pragma unroll
           for (int k = 0; k < S_BK / 16; ++k) {     // +32 bytes per K = 16 step inside the swizzle atom
             umma_bf16(d0, dw0 + 2 * k, dx + 2 * k, idesc, (kb | k) != 0);
@@ -199,6 +242,10 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
           }
           umma_commit(&empty_bar[stage]);   // stage reusable once these MMAs have read it
           if (++stage == S_STAGES) { stage = 0; phase ^= 1; }
+          if (WQ) {
+            umma_commit(&cempty_bar[cs]);   // and so is the buffer of expanded weights
+            if (++cs == S_CVT_STAGES) { cs = 0; cphase ^= 1; }
+          }
         }
         if (!ok) break;
         umma_commit(&tfull_bar[as]);        // both accumulators complete
@@ -206,7 +253,72 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
       }
       if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
-  } else {
+  } else if (WQ && warp >= 6) {
+    // ------------------------------------------------------------ weight converters (FP8 stream, warps 6..13)
+    // Per k-block: two boxes of 128 rows x 64 FP8 bytes (row-major, 64-byte rows) -> two boxes of 128 rows x 64
+    // bf16 in the 128-byte swizzle (16-byte chunk c of row r at r*128 + ((c ^ (r & 7)) * 16)).  A thread takes
+    // 16 bytes (row p/4, bytes 16*(p%4) ..) at a time: one 16-byte load, two 16-byte stores; consecutive
+    // threads read consecutive pieces and the eight lanes of a quarter-warp write eight different chunks.
+    const int ct = threadIdx.x - S_THREADS;      // 0 .. S_CONVERTERS-1
+    int stage = 0; uint32_t phase = 0;
+    int cs = 0; uint32_t cphase = 0;
+    bool ok = true;
+    for (uint32_t it = 0; ok; ++it) {
+      const int slot = it % G_SCHED;
+      const uint32_t sph = (it / G_SCHED) & 1;
+      if (!mbar_wait(&sfull_bar[slot], sph, abort_flag, budget)) { ok = false; break; }
+      const int tile = ring[slot * G_SLOT_INTS];
+      const TileInfo ti = slot_load(ring + slot * G_SLOT_INTS);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sempty_bar[slot]);
+      if (tile < 0) break;
+      const Segment& sg = p.seg[ti.seg];
+      // block scales of the tile's two weight boxes: lane l holds the exponent of 128-column block l
+      const int n_kb128 = (sg.k_blocks + 1) >> 1;
+      const int rb0 = MODE == 0 ? ti.nb : 2 * ti.nb, rb1 = MODE == 0 ? ti.nb : 2 * ti.nb + 1;
+      const int rb_per_group = (sg.b_rows_per_group + 127) >> 7;
+      const long long sc_base = (long long)ti.group_local * rb_per_group;
+      int se0 = 0, se1 = 0;
+      if (lane < n_kb128) {
+        se0 = p.wscale[ti.seg][0][(sc_base + rb0) * n_kb128 + lane];
+        if (rb1 < rb_per_group) se1 = p.wscale[ti.seg][1][(sc_base + rb1) * n_kb128 + lane];
+      }
+      for (int kb = 0; kb < sg.k_blocks; ++kb) {
+        if (!mbar_wait(&full_bar[stage], phase, abort_flag, budget)) { ok = false; break; }
+        if (!mbar_wait(&cempty_bar[cs], cphase ^ 1, abort_flag, budget)) { ok = false; break; }
+        const int e0 = __shfl_sync(0xffffffffu, se0, kb >> 1), e1 = __shfl_sync(0xffffffffu, se1, kb >> 1);
+        const unsigned char* raw_w = smem + stage * S_STAGE_BYTES;
+        unsigned char* out_w = smem + L::CVT_OFF + cs * 2 * S_W_BYTES;
+#pragma unroll
+        for (int box = 0; box < 2; ++box) {
+          const uint32_t mbits = (uint32_t)(247 + (box ? e1 : e0)) << 7;      // bf16 2^(120 + scale exponent)
+          const uint32_t m2 = mbits | (mbits << 16);
+          const __nv_bfloat162 mul = *reinterpret_cast<const __nv_bfloat162*>(&m2);
+          uint4 q[S_CVT_PIECES];
+#pragma unroll
+          for (int i = 0; i < S_CVT_PIECES; ++i)
+            q[i] = *reinterpret_cast<const uint4*>(raw_w + box * S_WQ_BYTES + (i * S_CONVERTERS + ct) * 16);
+#pragma unroll
+          for (int i = 0; i < S_CVT_PIECES; ++i) {
+            const int pce = i * S_CONVERTERS + ct, r = pce >> 2, c = pce & 3;
+            const uint32_t w4[4] = {q[i].x, q[i].y, q[i].z, q[i].w};
+            uint32_t o[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { o[2 * j] = e4m3x2_to_bf16x2(w4[j], 0, mul); o[2 * j + 1] = e4m3x2_to_bf16x2(w4[j], 1, mul); }
+            unsigned char* row = out_w + box * S_W_BYTES + r * 128;
+            *reinterpret_cast<uint4*>(row + (((2 * c) ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ (r & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+          }
+        }
+        fence_proxy_async_smem();            // the MMA reads these generic-proxy writes through the async proxy
+        mbar_arrive(&cfull_bar[cs]);
+        mbar_arrive(&empty_bar[stage]);      // this thread is done with the stage's weight bytes
+        if (++stage == S_STAGES) { stage = 0; phase ^= 1; }
+        if (++cs == S_CVT_STAGES) { cs = 0; cphase ^= 1; }
+      }
+    }
+    if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+  } else if (warp >= 2 && warp < 6) {
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int q = warp & 3;                 // TMEM lane quarter this warp may access = features 32q .. 32q+31
     int as = 0; uint32_t aphase = 0;
@@ -323,7 +435,9 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
 }
 
 // ---------------------------------------------------------------- host side
-fmmoe_status launch_ffn_sm(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
+template <int WQ>
+static fmmoe_status launch_ffn_sm_impl(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
+  using L = SmLayout<WQ>;
   const fmmoe_layer_desc& d = *a.d;
   const int H = d.hidden, I = d.inter, E = d.n_experts, Ns = d.n_shared, Is = d.shared_inter;
   if (!h->encode_tiled) return FMMOE_ERR_CUDA;
@@ -337,15 +451,18 @@ fmmoe_status launch_ffn_sm(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
     ok &= make_map(h, &X1r[i], a.xp, p_rows, H, 32 * (i + 1));
     ok &= make_map(h, &X2r[i], a.act, p_rows, I, 32 * (i + 1));
   }
-  ok &= make_map(h, &G1r, a.w->w_gate, (uint64_t)E * I, H, 128);
-  ok &= make_map(h, &U1r, a.w->w_up, (uint64_t)E * I, H, 128);
-  ok &= make_map(h, &D2r, a.w->w_down, (uint64_t)E * H, I, 128);
+  auto wmap = [&](CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols) {
+    return WQ ? make_map_u8(h, m, base, rows, cols, 128) : make_map(h, m, base, rows, cols, 128);
+  };
+  ok &= wmap(&G1r, a.w->w_gate, (uint64_t)E * I, H);
+  ok &= wmap(&U1r, a.w->w_up, (uint64_t)E * I, H);
+  ok &= wmap(&D2r, a.w->w_down, (uint64_t)E * H, I);
   if (Ns) {
     ok &= make_map(h, &X1s, a.x, (uint64_t)a.T, H, 128);
-    ok &= make_map(h, &G1s, a.w->ws_gate, (uint64_t)Ns * Is, H, 128);
-    ok &= make_map(h, &U1s, a.w->ws_up, (uint64_t)Ns * Is, H, 128);
+    ok &= wmap(&G1s, a.w->ws_gate, (uint64_t)Ns * Is, H);
+    ok &= wmap(&U1s, a.w->ws_up, (uint64_t)Ns * Is, H);
     ok &= make_map(h, &X2s, a.act_sh, (uint64_t)Ns * a.T, Is, 128);
-    ok &= make_map(h, &D2s, a.w->ws_down, (uint64_t)Ns * H, Is, 128);
+    ok &= wmap(&D2s, a.w->ws_down, (uint64_t)Ns * H, Is);
   } else {
     X1s = X1r[3]; G1s = G1r; U1s = U1r; X2s = X2r[3]; D2s = D2r;   // never dereferenced without shared experts
   }
@@ -361,6 +478,8 @@ fmmoe_status launch_ffn_sm(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   p1.x = static_cast<const __nv_bfloat16*>(a.x); p1.ld_x = H; p1.row_token = a.row_token; p1.gather = 0;
   p1.tile_counter = a.tile_counters;
   p1.wait_budget_ns = h->wait_budget_ns; p1.test_withhold_stage = a.test_withhold_stage;
+  p1.wscale[0][0] = a.w->w_gate_scale; p1.wscale[0][1] = a.w->w_up_scale;
+  p1.wscale[1][0] = a.w->ws_gate_scale; p1.wscale[1][1] = a.w->ws_up_scale;
 
   GemmParams p2 = p1;
   p2.seg[0] = Segment{(H + 255) / 256, I / S_BK, H, H, 0, 0, H};
@@ -370,19 +489,26 @@ fmmoe_status launch_ffn_sm(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
   p2.yb[0] = static_cast<__nv_bfloat16*>(a.yb); p2.yb[1] = static_cast<__nv_bfloat16*>(a.ybsh); p2.pair = a.pair;
   p2.tile_counter = a.tile_counters + 1;
   p2.test_withhold_stage = -1;
+  p2.wscale[0][0] = p2.wscale[0][1] = a.w->w_down_scale;
+  p2.wscale[1][0] = p2.wscale[1][1] = a.w->ws_down_scale;
 
-  if (!h->sm_attr_set) {
-    FMMOE_CUDA_TRY(cudaFuncSetAttribute(ffn_sm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES));
-    FMMOE_CUDA_TRY(cudaFuncSetAttribute(ffn_sm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM_BYTES));
-    h->sm_attr_set = true;
+  bool& attr_set = WQ ? h->smq_attr_set : h->sm_attr_set;
+  if (!attr_set) {
+    FMMOE_CUDA_TRY(cudaFuncSetAttribute(ffn_sm_kernel<0, WQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES));
+    FMMOE_CUDA_TRY(cudaFuncSetAttribute(ffn_sm_kernel<1, WQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES));
+    attr_set = true;
   }
   const int grid = a.grid_override > 0 ? a.grid_override : h->sm_count;
-  { ProfScope ps(h, FMMOE_KERNEL_GEMM1, s); FMMOE_CUDA_TRY(launch_pdl(ffn_sm_kernel<0>, dim3(grid), dim3(S_THREADS), S_SMEM_BYTES, s, 1, X1r[0], X1r[1], X1r[2], X1r[3], X1s, G1r, U1r, G1s, U1s, p1)); }
+  { ProfScope ps(h, FMMOE_KERNEL_GEMM1, s); FMMOE_CUDA_TRY(launch_pdl(ffn_sm_kernel<0, WQ>, dim3(grid), dim3(L::THREADS), L::SMEM_BYTES, s, 1, X1r[0], X1r[1], X1r[2], X1r[3], X1s, G1r, U1r, G1s, U1s, p1)); }
   FMMOE_CUDA_TRY(cudaGetLastError());
-  { ProfScope ps(h, FMMOE_KERNEL_GEMM2, s); FMMOE_CUDA_TRY(launch_pdl(ffn_sm_kernel<1>, dim3(grid), dim3(S_THREADS), S_SMEM_BYTES, s, 1, X2r[0], X2r[1], X2r[2], X2r[3], X2s, D2r, D2r, D2s, D2s, p2)); }
+  { ProfScope ps(h, FMMOE_KERNEL_GEMM2, s); FMMOE_CUDA_TRY(launch_pdl(ffn_sm_kernel<1, WQ>, dim3(grid), dim3(L::THREADS), L::SMEM_BYTES, s, 1, X2r[0], X2r[1], X2r[2], X2r[3], X2s, D2r, D2r, D2s, D2s, p2)); }
   FMMOE_CUDA_TRY(cudaGetLastError());
   h->launches += 2;
   return FMMOE_OK;
+}
+
+fmmoe_status launch_ffn_sm(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
+  return a.d->weight_format == FMMOE_WEIGHTS_FP8_BLOCK128 ? launch_ffn_sm_impl<1>(h, a, s) : launch_ffn_sm_impl<0>(h, a, s);
 }
 
 }  // namespace fmmoe

@@ -22,6 +22,7 @@ struct fmmoe_handle {
   bool tc_attr_set;     // dynamic shared memory opt-in done for the tensor-core kernels
   bool route_attr_set;  // ... for the bf16 router
   bool sm_attr_set;     // ... for the small-M form of the expert GEMMs
+  bool smq_attr_set;    // ... and its FP8 weight stream
   int64_t small_m_max_tokens;     // below this many tokens the expert GEMMs run in their small-M form
   int64_t pair_min_tokens;        // from this many tokens on the combine goes through per-pair bf16 rows (no atomics)
   int test_withhold_stage;        // self-test (fmmoe_test_expire_wait): armed for the next layer call, else -1
@@ -227,7 +228,12 @@ constexpr int64_t kPairMinTokensDefault = 8192;
 static inline bool use_pair_rows(const fmmoe_handle* h, const fmmoe_layer_desc& d, int64_t T, uint32_t flags) {
   return d.dtype == FMMOE_BF16 && !(flags & FMMOE_FLAG_DETERMINISTIC) && T >= h->pair_min_tokens;
 }
-static inline bool use_small_m(const fmmoe_handle* h, int64_t T) { return T < h->small_m_max_tokens && T < h->gather_min_tokens; }
+// FP8 weights exist only in that form (the weight boxes are expanded in shared memory there).
+static inline bool use_small_m(const fmmoe_handle* h, const fmmoe_layer_desc& d, int64_t T) {
+  if (d.dtype != FMMOE_BF16) return false;
+  if (d.weight_format == FMMOE_WEIGHTS_FP8_BLOCK128) return true;
+  return T < h->small_m_max_tokens && T < h->gather_min_tokens;
+}
 fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);   // fp32 FMA
 
 struct FinalizeArgs {

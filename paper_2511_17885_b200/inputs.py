@@ -295,3 +295,48 @@ def stack_layer_weights_torch(cfg: StackCfg, layer: int, device: str):
         w["ws_up"] = draw((lc.n_shared, Is, H))
         w["ws_down"] = draw((lc.n_shared, H, Is), down_std)
     return w
+
+
+# ----------------------------------------------------------------------------
+# FP8 storage of the expert matrices (a storage format, not part of the method)
+# ----------------------------------------------------------------------------
+EXPERT_MATRICES = ("w_gate", "w_up", "w_down", "ws_gate", "ws_up", "ws_down")
+
+
+def to_fp8_block128(w: np.ndarray):
+    """Store a stack of matrices [G, R, C] as FP8 E4M3 bytes with one power-of-two scale per 128 x 128 block.
+
+    Per block: the smallest exponent s in [-100, 7] with max|w| / 2^s <= 448 (the largest E4M3 magnitude), then
+    each element w / 2^s rounded to E4M3 (torch's float8_e4m3fn cast: round to nearest even).
+    Returns (bytes uint8 [G, R, C], exponents int8 [G, ceil(R/128), ceil(C/128)], stored values float32 [G, R, C]);
+    the stored values are what the bytes and exponents represent, decoded with torch's own float8 type, so that a
+    CPU reference can consume them by value."""
+    import torch
+    G, R, C = w.shape
+    rb, cb = (R + 127) // 128, (C + 127) // 128
+    t = torch.from_numpy(np.ascontiguousarray(w, dtype=np.float32))
+    pad = torch.zeros((G, rb * 128, cb * 128), dtype=torch.float32)
+    pad[:, :R, :C] = t
+    blocks = pad.view(G, rb, 128, cb, 128)
+    amax = blocks.abs().amax(dim=(2, 4))                                    # [G, rb, cb]
+    exps = torch.where(amax > 0, torch.ceil(torch.log2(amax / 448.0)), torch.zeros_like(amax)).clamp_(-100, 7)
+    scale = torch.exp2(exps)[:, :, None, :, None]
+    q = (blocks / scale).to(torch.float8_e4m3fn)
+    stored = (q.to(torch.float32) * scale).reshape(G, rb * 128, cb * 128)[:, :R, :C].contiguous()
+    qbytes = q.view(torch.uint8).reshape(G, rb * 128, cb * 128)[:, :R, :C].contiguous()
+    return qbytes.numpy(), exps.to(torch.int8).numpy(), stored.numpy()
+
+
+def weights_to_fp8(w: Dict[str, Optional[np.ndarray]]):
+    """Expert matrices of a layer in FP8 block storage.  Returns (stored, packed): `stored` is the weight dict with
+    every expert matrix replaced by the values its FP8 form represents (float32; router untouched) and `packed`
+    maps name -> uint8 bytes and name + "_scale" -> int8 exponents."""
+    stored, packed = dict(w), {}
+    for k in EXPERT_MATRICES:
+        if w.get(k) is None:
+            continue
+        qb, ex, val = to_fp8_block128(w[k])
+        stored[k] = val
+        packed[k] = qb
+        packed[k + "_scale"] = ex
+    return stored, packed

@@ -26,6 +26,17 @@ def upload_weights(w: Dict[str, Optional[np.ndarray]], dtype: str, device: str) 
     return out
 
 
+def upload_weights_fp8(w: Dict[str, Optional[np.ndarray]], packed: Dict[str, np.ndarray], dtype: str,
+                       device: str) -> Dict[str, Optional[torch.Tensor]]:
+    """Router parameters as usual; expert matrices as FP8 bytes plus their int8 block-scale exponents."""
+    out = upload_weights({k: v for k, v in w.items() if k not in I.EXPERT_MATRICES}, dtype, device)
+    for k in I.EXPERT_MATRICES:
+        out[k] = None
+    for k, v in packed.items():
+        out[k] = torch.from_numpy(np.ascontiguousarray(v)).to(device)
+    return out
+
+
 class LayerWorkload:
     """One MoE layer over one batch of sequences, followed by one pruning stage.
 
@@ -36,20 +47,26 @@ class LayerWorkload:
 
     def __init__(self, cfg: I.LayerCfg, handle: B.Handle, device: int = 0, prune: Optional[I.PruneCfg] = None,
                  use_attn: bool = False, flags: int = B.FLAG_REDUCE_ON, token_seed: Optional[int] = None,
-                 keep_host: bool = False):
+                 keep_host: bool = False, fp8_weights: bool = False):
         self.cfg, self.h = cfg, handle
         dev = f"cuda:{device}"
         td = TDT[cfg.dtype]
         x, mask, seq_off, n_vis = I.make_tokens(cfg, seed=token_seed)
         w = I.make_weights(cfg)
+        self.fp8_weights = fp8_weights
+        if fp8_weights:
+            # the layer's expert matrices stored as FP8 bytes + block scales; `w` becomes the values they represent
+            w, packed = I.weights_to_fp8(w)
+            self.wd = upload_weights_fp8(w, packed, cfg.dtype, dev)
+        else:
+            self.wd = upload_weights(w, cfg.dtype, dev)
         self.host = {"x": x, "mask": mask, "w": w} if keep_host else None
         self.seq_off, self.n_vis = seq_off, n_vis
         self.x = torch.from_numpy(x).to(dev).to(td).contiguous()
         self.mask = torch.from_numpy(mask).to(dev)
-        self.wd = upload_weights(w, cfg.dtype, dev)
         self.ws = B.make_weights(self.wd)
         self.desc = B.make_desc(cfg.hidden, cfg.n_experts, cfg.inter, cfg.n_shared, cfg.shared_inter, cfg.top_k,
-                                cfg.top_k_vis, td)
+                                cfg.top_k_vis, td, B.WEIGHTS_FP8_BLOCK128 if fp8_weights else B.WEIGHTS_AS_DTYPE)
         self.flags = flags
         T, E, K = cfg.n_tokens, cfg.n_experts, cfg.top_k
         self.out = torch.empty_like(self.x)

@@ -28,9 +28,9 @@ def oracle_layer(x, mask, w, K, Kv, reduce_on, logits32, add_residual=False):
     return r, out
 
 
-def check_layer_workload(cfg, handle_=None):
+def check_layer_workload(cfg, handle_=None, fp8_weights=False):
     h = handle_ or handle()
-    wl = LayerWorkload(cfg, h, device=0, prune=None, keep_host=True)
+    wl = LayerWorkload(cfg, h, device=0, prune=None, keep_host=True, fp8_weights=fp8_weights)
     T, E, K = cfg.n_tokens, cfg.n_experts, cfg.top_k
     wl.route = {"logits": torch.empty(T, E, dtype=torch.float32, device="cuda"),
                 "probs": torch.empty(T, E, dtype=torch.float32, device="cuda"),
@@ -65,6 +65,13 @@ def check_layer_workload(cfg, handle_=None):
 def test_c1_full():
     wl, g = check_layer_workload(I.C1)
     assert int(g["expert_off"][-1]) == 2304 * 3 + 128 * 6
+
+
+def test_c1_and_c2_full_with_fp8_expert_weights():
+    """The full-size DeepSeekMoE-style and Qwen3-MoE-style layers with their expert matrices stored as FP8 bytes +
+    block scales: every output row against the oracle fed the values that storage represents."""
+    check_layer_workload(I.C1, fp8_weights=True)
+    check_layer_workload(I.C2, fp8_weights=True)
 
 
 def test_c2_full_and_batch_of_four():
