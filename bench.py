@@ -13,8 +13,9 @@ is the whole stack (fmmoe_stack_forward).
 The default (`--workload all`) prints ONE JSON line whose top-level fields are the
 largest single-layer workload (the batch of four Qwen3-MoE-style sequences, 14,336
 tokens) and whose `configs` object holds one record per other workload (C0, C1, C2,
-C3, C4, and C1-C3 once more with their expert matrices stored as FP8), each with its
-own timing, clocks, roofline and end-to-end figure.
+C3, C4, C1-C3 once more with their expert matrices stored as FP8, and the paper's two
+three-stage pruning schedules on stacks of the matching layer shape), each with its own
+timing, clocks, roofline and end-to-end figure.
 
 Timing: a block is exactly K steps between two CUDA events, with a barrier and a
 device synchronisation on both sides.  Whatever K is, blocks are repeated until the
@@ -41,7 +42,10 @@ import numpy as np  # noqa: E402
 METRIC = "MoE-layer prefill tokens/s"
 UNIT = "tokens/s"
 LAYER_WORKLOADS = ("C0", "C1", "C2", "C2x4", "C3")
-WORKLOADS = ("all",) + LAYER_WORKLOADS + ("C1_fp8", "C2_fp8", "C3_fp8", "C4")
+# the paper's own three-stage schedules (Appendix A) at 50 % overall retention, attention-guided, on a stack of the
+# matching layer shape: name -> (backbone family, overall retention)
+PAPER_STACKS = {"S_internvl_50": ("internvl3.5", 0.5), "S_deepseek_50": ("deepseek-vl2", 0.5)}
+WORKLOADS = ("all",) + LAYER_WORKLOADS + ("C1_fp8", "C2_fp8", "C3_fp8", "C4") + tuple(PAPER_STACKS)
 HEADLINE = "C2x4"
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # the nominal peaks the metric names (8 TB/s, dense bf16)
 
@@ -264,11 +268,13 @@ def block_stats(secs, mhz, K):
 
 
 # ------------------------------------------------------------------ oracle timing
-def oracle_sample(name, cfg, prune, frac):
+def oracle_sample(name, cfg, prune, frac, fp8=False):
     """Inputs of a bounded sample: the first `frac` of every sequence's visual and text tokens."""
     from paper_2511_17885_b200 import inputs as I
     x, mask, seq_off, n_vis = I.make_tokens(cfg)
     w = I.make_weights(cfg)
+    if fp8:      # the values the FP8 bytes and block scales represent
+        w, _ = I.weights_to_fp8(w)
     idx = []
     for b in range(cfg.batch):
         lo = int(seq_off[b])
@@ -302,8 +308,8 @@ def blas_threads():
     return 1
 
 
-def time_oracle(name, cfg, prune, frac, steps, warmup, one_thread_frac=None):
-    xs, ms, so, nvs, w = oracle_sample(name, cfg, prune, frac)
+def time_oracle(name, cfg, prune, frac, steps, warmup, one_thread_frac=None, fp8=False):
+    xs, ms, so, nvs, w = oracle_sample(name, cfg, prune, frac, fp8)
     for _ in range(warmup):
         oracle_step(cfg, prune, xs, ms, so, nvs, w)
     t0 = time.perf_counter()
@@ -339,9 +345,11 @@ def run_reference(args):
     if rank != 0:
         return 0
     name = HEADLINE if args.workload == "all" else args.workload
+    fp8 = name.endswith("_fp8")
+    name = name[:-4] if fp8 else name
     cfg, prune = workload_cfg(name)
     frac = 1.0 if cfg.n_tokens <= 4096 else 4096.0 / cfg.n_tokens
-    value, spp, cores, sample, _ = time_oracle(name, cfg, prune, frac, max(args.steps, 1), min(args.warmup, 1))
+    value, spp, cores, sample, _ = time_oracle(name, cfg, prune, frac, max(args.steps, 1), min(args.warmup, 1), fp8=fp8)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": spp * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -521,14 +529,17 @@ def measure_layer(name, args, D, rank, local, world, peaks, with_cpu, fp8=False)
 
 
 # ------------------------------------------------------------------ the 24-layer stack (C4)
-def stack_describe(sc, n_layers):
+def stack_describe(sc, n_layers, label="C4", attention=False):
     lc = sc.layer
-    st = ", ".join(f"after layer {l}: to {int(pc.retain * 100)}% (W={pc.window}, gamma={pc.gamma})"
+    st = ", ".join(f"after layer {l}: to {pc.retain * 100:.1f}% (W={pc.window}, gamma={pc.gamma}"
+                   + (f", alpha={pc.alpha}" if attention else "") + ")"
                    for l, pc in sorted(sc.prune_after.items()))
-    return {"workload": f"C4: {n_layers} MoE layers of the C1 shape with residual adds (attention omitted), "
+    score = ("attention-guided score, A_hat of Eq. 7 from fmmoe_attention_importance on stand-in queries / keys inside "
+             "the step" if attention else "attention-free score")
+    return {"workload": f"{label}: {n_layers} MoE layers of the {lc.name} shape with residual adds (attention layers omitted), "
                         f"{lc.batch} x ({lc.n_vis} visual + {lc.n_text} text) tokens, H={lc.hidden} E={lc.n_experts} "
                         f"I={lc.inter} shared={lc.n_shared} K={lc.top_k}, K_v={lc.top_k_vis} from layer {sc.reduce_from}; "
-                        f"pruning {st}; attention-free score",
+                        f"pruning {st}; {score}",
             "tokens_per_step": lc.n_tokens,
             "l2": f"inputs larger than L2: {n_layers} x {weight_bytes(lc) / 1e6:.0f} MB of distinct layer weights"}
 
@@ -572,23 +583,25 @@ def stack_cpu_baseline(sc, n_layers):
     return {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample}
 
 
-def measure_stack(args, D, rank, local, world, peaks, with_cpu):
+def measure_stack(args, D, rank, local, world, peaks, with_cpu, sc=None, label="C4", attention=False):
     import torch
     from paper_2511_17885_b200 import binding as B
     from paper_2511_17885_b200 import inputs as I
     from paper_2511_17885_b200.workload import StackWorkload
     dev = f"cuda:{local}"
-    sc = I.C4
-    n_layers = args.layers or sc.n_layers
+    paper = sc is not None
+    sc = I.C4 if sc is None else sc
+    n_layers = sc.n_layers if paper else (args.layers or sc.n_layers)
     h = B.Handle(local)
-    wl = StackWorkload(sc, h, device=local, token_seed=D.token_seed_for_rank(sc.layer.seed, rank), n_layers=n_layers)
+    wl = StackWorkload(sc, h, device=local, token_seed=D.token_seed_for_rank(sc.layer.seed, rank), n_layers=n_layers,
+                       attention=attention)
     K, W = max(1, min(args.steps, 10)), max(args.warmup, 3)      # a stack step is 24 layers: at most 10 per block
     if args.plain:      # for profilers
         for _ in range(args.warmup + K):
             wl.step()
         torch.cuda.synchronize()
         h.check_status("plain run")
-        return {"value": 0.0, "ms_per_step": 0.0, "dtype": sc.layer.dtype, "config": stack_describe(sc, n_layers), "plain": True}
+        return {"value": 0.0, "ms_per_step": 0.0, "dtype": sc.layer.dtype, "config": stack_describe(sc, n_layers, label, attention), "plain": True}
     for _ in range(min(W, 5)):
         wl.step()
     settle_s = settle_clocks(wl.step, local, min_s=0.2)
@@ -652,7 +665,7 @@ def measure_stack(args, D, rank, local, world, peaks, with_cpu):
     flops_per_launch = {"gemm1": g1, "gemm2": g2, "route": rt}.get(dom, 0.0) / n_layers
     roof = {"bound": "tensor", "achieved": flops_per_launch / per_launch_s / 1e12, "peak": peaks["tf_sustained"],
             "peak_nominal": NOMINAL["bf16_tflops"], "unit": "TFLOP/s", "kernel": dom, "us_per_launch": per_launch_s * 1e6,
-            "algorithmic_flops": flops_per_launch, "traffic": NCU_TRAFFIC_BYTES.get("C4", {}).get(dom),
+            "algorithmic_flops": flops_per_launch, "traffic": NCU_TRAFFIC_BYTES.get(label, {}).get(dom),
             "peak_source": peaks["source"] + " (sustained bf16)",
             "note": "per-launch figures are the mean over the stack's layers (three different token counts)"}
     roof["frac"] = roof["achieved"] / roof["peak"]
@@ -665,7 +678,7 @@ def measure_stack(args, D, rank, local, world, peaks, with_cpu):
 
     # the unreduced, unpruned comparison run (K experts for every token, all tokens in every layer)
     dense = None
-    if not args.no_dense:
+    if not args.no_dense and not paper:
         del wl.x_out
         wd = StackWorkload.__new__(StackWorkload)
         wd.__dict__.update(wl.__dict__)
@@ -690,7 +703,7 @@ def measure_stack(args, D, rank, local, world, peaks, with_cpu):
         h.check_status("dense-k run")
         del wd
 
-    conf = stack_describe(sc, n_layers)
+    conf = stack_describe(sc, n_layers, label, attention)
     conf.update({"parallelism": f"replicas x{world} (no collective)", "tokens_per_layer": [t for t, _ in shapes],
                  "final_tokens": wl.out_off[-1], "output_std": out_std,
                  "weights": "N(0, 0.02^2); down-projections N(0, (0.02/sqrt(2*layers))^2) so that the norm-free "
@@ -716,13 +729,14 @@ def run_stack_reference(args):
     if int(os.environ.get("RANK", 0)) != 0:
         return 0
     from paper_2511_17885_b200 import inputs as I
-    sc = I.C4
-    n_layers = args.layers or sc.n_layers
+    paper = args.workload in PAPER_STACKS
+    sc = I.paper_stack(*PAPER_STACKS[args.workload]) if paper else I.C4
+    n_layers = sc.n_layers if paper else (args.layers or sc.n_layers)
     cb = stack_cpu_baseline(sc, n_layers)
     line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sc.layer.n_tokens / cb["value"] * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": stack_describe(sc, n_layers), "cpu_baseline": cb,
+            "config": stack_describe(sc, n_layers, args.workload, paper), "cpu_baseline": cb,
             "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -745,6 +759,11 @@ def run_ours(args):
     def measure(name, cpu):
         if name == "C4":
             return measure_stack(args, D, rank, local, world, peaks, cpu)
+        if name in PAPER_STACKS:
+            from paper_2511_17885_b200 import inputs as I
+            model, retain = PAPER_STACKS[name]
+            return measure_stack(args, D, rank, local, world, peaks, False, sc=I.paper_stack(model, retain), label=name,
+                                 attention=True)
         if name.endswith("_fp8"):
             return measure_layer(name[:-4], args, D, rank, local, world, peaks, cpu, fp8=True)
         return measure_layer(name, args, D, rank, local, world, peaks, cpu)
@@ -752,7 +771,7 @@ def run_ours(args):
     rec = measure(head, with_cpu)
     configs = {}
     if args.workload == "all":     # the weight-stream-bound workloads once more with FP8 expert weights
-        others = others[:-1] + ["C1_fp8", "C2_fp8", "C3_fp8"] + others[-1:]
+        others = others[:-1] + ["C1_fp8", "C2_fp8", "C3_fp8"] + others[-1:] + list(PAPER_STACKS)
     for name in others:
         configs[name] = measure(name, False)
     if rank == 0:
@@ -786,7 +805,7 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="C4 only: skip the unreduced, unpruned comparison run")
     args = ap.parse_args()
     if args.impl == "reference":
-        sys.exit(run_stack_reference(args) if args.workload == "C4" else run_reference(args))
+        sys.exit(run_stack_reference(args) if (args.workload == "C4" or args.workload in PAPER_STACKS) else run_reference(args))
     sys.exit(run_ours(args))
 
 

@@ -7,7 +7,7 @@
 //   D[128 output features, N token rows] (+)= W[128 features, 64] * X[N rows, 64]^T,   N = 16, 32, ... 128
 // so that the tensor work of a tile and the activation box both shrink with the expert's rows, in steps
 // of 16 and 32 rows.  Everything else is the persistent kernel of ffn_tc.cu: the same tile list and
-// interleaved order, a warp that schedules tiles and feeds a 4-stage TMA ring, one thread that issues
+// interleaved order, a warp that schedules tiles, one that feeds a 4-stage TMA ring, one thread that issues
 // the MMAs into two tensor-memory accumulator stages, four epilogue warps.
 //   GEMM-1: a tile is (M-tile of one expert) x (128 intermediate features); two MMAs per k-step (gate
 //           rows, up rows) share the activation operand; accumulators D_gate, D_up hold feature f in
@@ -38,7 +38,7 @@ constexpr int S_STAGES = 4;
 constexpr int S_W_BYTES = 128 * S_BK * 2;             // one 128-feature weight box as bf16: 16 KB
 constexpr int S_WQ_BYTES = 128 * S_BK;                // the same box as FP8 bytes: 8 KB
 constexpr int S_X_BYTES = 128 * S_BK * 2;             // room for up to 128 token rows: 16 KB
-constexpr int S_THREADS = 192;                        // scheduler/producer warp, issuer warp, four epilogue warps
+constexpr int S_THREADS = 224;                        // producer warp, issuer warp, four epilogue warps, tile-scheduler warp
 constexpr int S_CONVERTERS = 256;                     // FP8 stream: eight more warps that expand the weight boxes
 constexpr int S_CVT_PIECES = 512 / S_CONVERTERS;      // 16-byte pieces of a weight box per converter thread
 constexpr int S_CVT_STAGES = 2;
@@ -100,6 +100,7 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
   volatile int* ring = reinterpret_cast<volatile int*>(cempty_bar + S_CVT_STAGES);   // [G_SCHED][G_SLOT_INTS]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(ring) + G_SCHED * G_SLOT_INTS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* prod_half = abort_flag + 1;    // tiles the producer has taken half-way (paces the tile scheduler)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint64_t budget = p.wait_budget_ns;
@@ -107,13 +108,15 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
 
   if (threadIdx.x == 0) {
     // a raw stage is free again once the MMAs have read its activations and (FP8 stream) every converter
-    // thread has read its weight bytes
-    for (int i = 0; i < S_STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], WQ ? 1 + S_CONVERTERS : 1); }
+    // warp has read its weight bytes (one arrival per warp: hundreds of per-thread arrivals on one barrier
+    // would cost more than the conversion itself)
+    for (int i = 0; i < S_STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], WQ ? 1 + S_CONVERTERS / 32 : 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&tfull_bar[i], 1); mbar_init(&tempty_bar[i], 128); }
-    // readers of a tile id: issuer + 4 epilogue warps (+ the converter warps)
-    for (int i = 0; i < G_SCHED; ++i) { mbar_init(&sfull_bar[i], 1); mbar_init(&sempty_bar[i], WQ ? 5 + S_CONVERTERS / 32 : 5); }
-    for (int i = 0; i < S_CVT_STAGES; ++i) { mbar_init(&cfull_bar[i], S_CONVERTERS); mbar_init(&cempty_bar[i], 1); }
+    // readers of a tile id: producer + issuer + 4 epilogue warps (+ the converter warps)
+    for (int i = 0; i < G_SCHED; ++i) { mbar_init(&sfull_bar[i], 1); mbar_init(&sempty_bar[i], WQ ? 6 + S_CONVERTERS / 32 : 6); }
+    for (int i = 0; i < S_CVT_STAGES; ++i) { mbar_init(&cfull_bar[i], S_CONVERTERS / 32); mbar_init(&cempty_bar[i], 1); }
     *abort_flag = 0;
+    *prod_half = 0;
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -140,23 +143,17 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
       const uint64_t pol_stream = l2_policy_evict_first();
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      // Publishes the tile claimed as `raw` under sequence number `seq`, decoded.  1: a tile, 0: no tiles
-      // left, -1: timeout.
-      auto publish = [&](uint32_t seq, int raw_id, TileInfo& ti) -> int {
-        const int slot = seq % G_SCHED;
-        const uint32_t sph = (seq / G_SCHED) & 1;
-        if (!mbar_wait(&sempty_bar[slot], sph ^ 1, abort_flag, budget)) return -1;
-        const int tile = raw_id < total_tiles ? raw_id : -1;
-        if (tile >= 0) ti = decode_tile(p, tile, n_mt_r);
-        slot_store(ring + slot * G_SLOT_INTS, tile, ti);
-        mbar_arrive(&sfull_bar[slot]);
-        return tile >= 0;
-      };
-      TileInfo ti = {}, ti_next = {};
-      int have = publish(0, atomicAdd(p.tile_counter, 1), ti);
       int issued = 0;        // k-blocks handed to the TMA engine so far
       bool stop = false;
-      for (uint32_t it = 0; have == 1; ++it) {
+      for (uint32_t it = 0; ok && !stop; ++it) {
+        // the tile comes decoded from the scheduler warp: the producer touches no global memory but the TMA maps
+        const int slot = it % G_SCHED;
+        const uint32_t sph = (it / G_SCHED) & 1;
+        if (!mbar_wait(&sfull_bar[slot], sph, abort_flag, budget)) { ok = false; break; }
+        const int tile = ring[slot * G_SLOT_INTS];
+        const TileInfo ti = slot_load(ring + slot * G_SLOT_INTS);
+        mbar_arrive(&sempty_bar[slot]);
+        if (tile < 0) break;
         const Segment& sg = p.seg[ti.seg];
         // activation box: the smallest of 32 / 64 / 96 / 128 rows that covers the tile's (padded) rows
         const int npad = n_pad_of(ti.rows);
@@ -170,14 +167,9 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
         const int x_row = ti.row0 + ti.group_local * sg.a_group_stride;
         const int w_y0 = ti.group_local * sg.b_rows_per_group + ti.nb * (MODE == 0 ? 128 : 256);
         const int w_y1 = MODE == 0 ? w_y0 : w_y0 + 128;
-        const int kb_claim = sg.k_blocks >> 1, kb_publish = sg.k_blocks - 1;
-        int raw_next = 0, have_next = 0;
+        const int kb_half = sg.k_blocks >> 1;
         for (int kb = 0; kb < sg.k_blocks; ++kb) {
-          if (kb == kb_claim) raw_next = atomicAdd(p.tile_counter, 1);
-          if (kb == kb_publish) {
-            have_next = publish(it + 1, raw_next, ti_next);
-            if (have_next < 0) { ok = false; break; }
-          }
+          if (kb == kb_half) *prod_half = (int)it + 1;     // the scheduler may now claim the next tile
           if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, budget)) { ok = false; break; }
           if (issued == p.test_withhold_stage) {
             // Self-test hook (fmmoe_test_expire_wait): the producer stops here, before it has issued any copy
@@ -200,10 +192,39 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
           tma_load_2d(sW + L::X_OFF, mX, &full_bar[stage], kb * S_BK, x_row);
           if (++stage == S_STAGES) { stage = 0; phase ^= 1; }
         }
-        if (!ok || stop) break;
-        ti = ti_next; have = have_next;
       }
-      if (!ok || have < 0) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+      if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+    }
+  } else if (warp == 6) {
+    // ------------------------------------------------------------ tile scheduler
+    // Claims tiles from the global counter, decodes them (a global read of the M-tile list and a few
+    // divisions) and publishes them through the slot ring: tile n+1 is claimed when the producer is half-way
+    // through tile n.  Keeping this off the producer matters: its ring holds about as much work as a load takes
+    // to arrive, so any pause of the producer starves the MMAs.
+    if (lane == 0) {
+      bool ok = true;
+      for (uint32_t seq = 0; ok; ++seq) {
+        if (seq >= 1) {
+          const uint64_t t0 = global_timer_ns();
+          while (*prod_half < (int)seq) {
+            __nanosleep(64);
+            if (*abort_flag || global_timer_ns() - t0 > budget) { ok = false; break; }
+          }
+          if (!ok) break;
+        }
+        const int raw_id = atomicAdd(p.tile_counter, 1);
+        const int tile = raw_id < total_tiles ? raw_id : -1;
+        TileInfo ti = {};
+        if (tile >= 0) ti = decode_tile(p, tile, n_mt_r);
+        const int slot = seq % G_SCHED;
+        const uint32_t sph = (seq / G_SCHED) & 1;
+        if (!mbar_wait(&sempty_bar[slot], sph ^ 1, abort_flag, budget)) { ok = false; break; }
+        slot_store(ring + slot * G_SLOT_INTS, tile, ti);
+        mbar_arrive(&sfull_bar[slot]);
+        if (tile < 0) break;
+      }
+      // a scheduler that gave up because another role aborted records nothing: the status word has the cause
+      if (!ok && !*abort_flag) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ UMMA issuer
@@ -253,8 +274,8 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
       }
       if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
-  } else if (WQ && warp >= 6) {
-    // ------------------------------------------------------------ weight converters (FP8 stream, warps 6..13)
+  } else if (WQ && warp >= 7) {
+    // ------------------------------------------------------------ weight converters (FP8 stream, warps 7..14)
     // Per k-block: two boxes of 128 rows x 64 FP8 bytes (row-major, 64-byte rows) -> two boxes of 128 rows x 64
     // bf16 in the 128-byte swizzle (16-byte chunk c of row r at r*128 + ((c ^ (r & 7)) * 16)).  A thread takes
     // 16 bytes (row p/4, bytes 16*(p%4) ..) at a time: one 16-byte load, two 16-byte stores; consecutive
@@ -284,8 +305,9 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
         if (rb1 < rb_per_group) se1 = p.wscale[ti.seg][1][(sc_base + rb1) * n_kb128 + lane];
       }
       for (int kb = 0; kb < sg.k_blocks; ++kb) {
-        if (!mbar_wait(&full_bar[stage], phase, abort_flag, budget)) { ok = false; break; }
-        if (!mbar_wait(&cempty_bar[cs], cphase ^ 1, abort_flag, budget)) { ok = false; break; }
+        // warp-uniform outcome: the arrivals below are made by one lane on behalf of the warp
+        if (!__all_sync(0xffffffffu, mbar_wait(&full_bar[stage], phase, abort_flag, budget) &&
+                                     mbar_wait(&cempty_bar[cs], cphase ^ 1, abort_flag, budget))) { ok = false; break; }
         const int e0 = __shfl_sync(0xffffffffu, se0, kb >> 1), e1 = __shfl_sync(0xffffffffu, se1, kb >> 1);
         const unsigned char* raw_w = smem + stage * S_STAGE_BYTES;
         unsigned char* out_w = smem + L::CVT_OFF + cs * 2 * S_W_BYTES;
@@ -311,8 +333,11 @@ ffn_sm_kernel(const __grid_constant__ CUtensorMap tmX32, const __grid_constant__
           }
         }
         fence_proxy_async_smem();            // the MMA reads these generic-proxy writes through the async proxy
-        mbar_arrive(&cfull_bar[cs]);
-        mbar_arrive(&empty_bar[stage]);      // this thread is done with the stage's weight bytes
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(&cfull_bar[cs]);
+          mbar_arrive(&empty_bar[stage]);    // this warp is done with the stage's weight bytes
+        }
         if (++stage == S_STAGES) { stage = 0; phase ^= 1; }
         if (++cs == S_CVT_STAGES) { cs = 0; cphase ^= 1; }
       }

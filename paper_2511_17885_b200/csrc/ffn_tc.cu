@@ -6,9 +6,9 @@
 //   GEMM-1  [rows_e, H] x [H, 2*S_m]  -> SwiGLU in the epilogue -> act [rows, S_m] bf16
 //   GEMM-2  [rows_e, S_m] x [S_m, H]  -> gate-weighted combine in the epilogue
 // Both run in one persistent, warp-specialised kernel template:
-//   warp 0    : tile scheduler + TMA producer (A tile 128x64 + two B boxes 128x64 per stage,
-//               128B swizzle, L2 eviction hints)
-//   warps 6-9 : GEMM-1 at large batch only: gather the rows of a routed M-tile straight from x by
+//   warp 0    : TMA producer (A tile 128x64 + two B boxes 128x64 per stage, 128B swizzle, L2 eviction hints)
+//   warp 6    : tile scheduler (claims and decodes tiles one ahead of the producer)
+//   warps 7-10: GEMM-1 at large batch only: gather the rows of a routed M-tile straight from x by
 //               token with cp.async into the same swizzled layout, so that no expert-ordered copy
 //               of x is written and read back (at small batch that copy plus plain TMA boxes is
 //               faster: the kernel is then launched without these warps)
@@ -17,8 +17,8 @@
 //               global stores / reductions), overlapped with the next tile's main loop
 //               through two TMEM accumulator stages (2 x 256 columns).
 // A tile is (M-tile of 128 grouped rows) x (N-block).  Tiles are handed out dynamically (an
-// atomic counter; the producer publishes each tile id to the other roles through a small
-// shared-memory ring), in an order that
+// atomic counter; the scheduler warp publishes each tile, decoded, to the other roles through a
+// small shared-memory ring), in an order that
 //   - walks the routed tiles M-tile-major, so the 128 activation rows of an M-tile are
 //     re-read from L2 by CTAs running at the same time while every weight tile streams
 //     from HBM once,
@@ -44,7 +44,7 @@ constexpr int G_STAGES = 4;
 constexpr int G_A_BYTES = G_BM * G_BK * 2;          // 16 KB
 constexpr int G_B_BYTES = 2 * 128 * G_BK * 2;       // 32 KB (two 128-row boxes)
 constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;
-constexpr int G_THREADS = 192;          // scheduler/producer warp, issuer warp, four epilogue warps
+constexpr int G_THREADS = 224;          // producer warp, issuer warp, four epilogue warps, tile-scheduler warp
 constexpr int G_LOADERS = 128;          // GEMM-1 only: four more warps that gather the routed rows of x
 constexpr int G_THREADS_G1 = G_THREADS + G_LOADERS;
 constexpr int G_TMEM_COLS = 512;
@@ -73,6 +73,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
   volatile int* ring = reinterpret_cast<volatile int*>(sempty_bar + G_SCHED);   // [G_SCHED][G_SLOT_INTS]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(ring) + G_SCHED * G_SLOT_INTS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* prod_half = abort_flag + 1;    // tiles the producer has taken half-way (paces the tile scheduler)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   pdl_launch_dependents();
@@ -81,9 +82,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
     // GEMM-1: a stage is full when the producer's TMA bytes have landed AND every loader thread's copies have
     for (int i = 0; i < G_STAGES; ++i) { mbar_init(&full_bar[i], (MODE == 0 && p.gather) ? 1 + G_LOADERS : 1); mbar_init(&empty_bar[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&tfull_bar[i], 1); mbar_init(&tempty_bar[i], 128); }
-    // readers of a tile id: issuer + 4 epilogue warps (+ 4 loader warps in GEMM-1)
-    for (int i = 0; i < G_SCHED; ++i) { mbar_init(&sfull_bar[i], 1); mbar_init(&sempty_bar[i], (MODE == 0 && p.gather) ? 9 : 5); }
+    // readers of a tile id: producer + issuer + 4 epilogue warps (+ 4 loader warps in GEMM-1)
+    for (int i = 0; i < G_SCHED; ++i) { mbar_init(&sfull_bar[i], 1); mbar_init(&sempty_bar[i], (MODE == 0 && p.gather) ? 10 : 6); }
     *abort_flag = 0;
+    *prod_half = 0;
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -110,21 +112,15 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
       const uint64_t pol_stream = l2_policy_evict_first();
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      // Publishes the tile claimed as `raw` under sequence number `seq` (decoded, so that no other
-      // role touches global memory to learn what it is).  1: a tile, 0: no tiles left, -1: timeout.
-      auto publish = [&](uint32_t seq, int raw, TileInfo& ti) -> int {
-        const int slot = seq % G_SCHED;
-        const uint32_t sph = (seq / G_SCHED) & 1;
-        if (!mbar_wait(&sempty_bar[slot], sph ^ 1, abort_flag)) return -1;
-        const int tile = raw < total_tiles ? raw : -1;
-        if (tile >= 0) ti = decode_tile(p, tile, n_mt_r);
-        slot_store(ring + slot * G_SLOT_INTS, tile, ti);
-        mbar_arrive(&sfull_bar[slot]);
-        return tile >= 0;
-      };
-      TileInfo ti = {}, ti_next = {};
-      int have = publish(0, atomicAdd(p.tile_counter, 1), ti);
-      for (uint32_t it = 0; have == 1; ++it) {
+      for (uint32_t it = 0; ok; ++it) {
+        // the tile comes decoded from the scheduler warp: the producer touches no global memory but the TMA maps
+        const int slot = it % G_SCHED;
+        const uint32_t sph = (it / G_SCHED) & 1;
+        if (!mbar_wait(&sfull_bar[slot], sph, abort_flag)) { ok = false; break; }
+        const int tile = ring[slot * G_SLOT_INTS];
+        const TileInfo ti = slot_load(ring + slot * G_SLOT_INTS);
+        mbar_arrive(&sempty_bar[slot]);
+        if (tile < 0) break;
         const Segment& sg = p.seg[ti.seg];
         const CUtensorMap* mA = ti.seg ? &tmA_s : &tmA_r;
         const CUtensorMap* mB0 = ti.seg ? &tmB0_s : &tmB0_r;
@@ -140,16 +136,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
         const int a_row = ti.row0 + ti.group_local * sg.a_group_stride;
         const int b_y0 = ti.group_local * sg.b_rows_per_group + ti.nb * (MODE == 0 ? 128 : 256);
         const int b_y1 = MODE == 0 ? b_y0 : b_y0 + 128;
-        // The next tile is claimed half-way through this one and decoded while the last stages of
-        // this one are still in flight, so the ring never drains between tiles.
-        const int kb_claim = sg.k_blocks >> 1, kb_publish = sg.k_blocks - 1;
-        int raw_next = 0, have_next = 0;
+        const int kb_half = sg.k_blocks >> 1;
         for (int kb = 0; kb < sg.k_blocks; ++kb) {
-          if (kb == kb_claim) raw_next = atomicAdd(p.tile_counter, 1);
-          if (kb == kb_publish) {
-            have_next = publish(it + 1, raw_next, ti_next);
-            if (have_next < 0) { ok = false; break; }
-          }
+          if (kb == kb_half) *prod_half = (int)it + 1;     // the scheduler may now claim the next tile
           if (!mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           unsigned char* sA = smem + stage * G_STAGE_BYTES;
           mbar_arrive_expect_tx(&full_bar[stage], gather_a ? G_B_BYTES : G_STAGE_BYTES);
@@ -163,10 +152,39 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
           }
           if (++stage == G_STAGES) { stage = 0; phase ^= 1; }
         }
-        if (!ok) break;
-        ti = ti_next; have = have_next;
       }
-      if (!ok || have < 0) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+      if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
+    }
+  } else if (warp == 6) {
+    // ------------------------------------------------------------ tile scheduler
+    // Claims tiles from the global counter, decodes them (a global read of the M-tile list and a few
+    // divisions) and publishes them through the slot ring, one tile ahead of the producer: tile n+1 is
+    // claimed when the producer is half-way through tile n.  Keeping this off the producer matters: its
+    // ring holds about as much work as a load takes to arrive, so any pause of the producer starves the MMAs.
+    if (lane == 0) {
+      bool ok = true;
+      for (uint32_t seq = 0; ok; ++seq) {
+        if (seq >= 1) {     // tile n+1 is claimed once the producer is half-way through tile n
+          const uint64_t t0 = global_timer_ns();
+          while (*prod_half < (int)seq) {
+            __nanosleep(64);
+            if (*abort_flag || global_timer_ns() - t0 > 2000000000ull) { ok = false; break; }
+          }
+          if (!ok) break;
+        }
+        const int raw_id = atomicAdd(p.tile_counter, 1);
+        const int tile = raw_id < total_tiles ? raw_id : -1;
+        TileInfo ti = {};
+        if (tile >= 0) ti = decode_tile(p, tile, n_mt_r);
+        const int slot = seq % G_SCHED;
+        const uint32_t sph = (seq / G_SCHED) & 1;
+        if (!mbar_wait(&sempty_bar[slot], sph ^ 1, abort_flag)) { ok = false; break; }
+        slot_store(ring + slot * G_SLOT_INTS, tile, ti);
+        mbar_arrive(&sfull_bar[slot]);
+        if (tile < 0) break;
+      }
+      // a scheduler that gave up because another role aborted records nothing: the status word has the cause
+      if (!ok && !*abort_flag) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ UMMA issuer
@@ -209,8 +227,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
       }
       if (!ok) { atomicCAS(p.status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
-  } else if (warp >= 6) {
-    // ------------------------------------------------------------ row loaders (GEMM-1 only, warps 6..9)
+  } else if (warp >= 7) {
+    // ------------------------------------------------------------ row loaders (GEMM-1 only, warps 7..10)
     // Every stage of a routed tile: 128 rows x 128 bytes of x, row r = token row_token[row0 + r],
     // written where a TMA box with the 128-byte swizzle would put them (16-byte chunk c of row r at
     // r*128 + ((c ^ (r & 7)) * 16)).  Eight lanes cover one row, a thread serves rows q, q+16, ...

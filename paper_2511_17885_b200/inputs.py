@@ -249,6 +249,28 @@ def paper_schedule(model: str, overall_retain: float) -> Dict[int, PruneCfg]:
             for t, layer in enumerate(sc["layers"])}
 
 
+def paper_stack(model: str, overall_retain: float) -> StackCfg:
+    """A stack that carries the paper's three-stage schedule of one backbone family (Appendix A): the layer shape of
+    the matching single-layer workload, one sequence, as many layers as the schedule needs plus one more (so that
+    the last stage's output is consumed by a layer), expert reduction from layer 2 on."""
+    layer = {"internvl3.5": C2, "deepseek-vl2": C1}[model]
+    sched = paper_schedule(model, overall_retain)
+    return StackCfg(name=f"paper-{model}-{int(overall_retain * 100)}", layer=replace(layer, name=f"{model}-layer", prune=()),
+                    n_layers=max(sched) + 2, reduce_from=2, prune_after=sched, seed=50 + int(overall_retain * 100))
+
+
+def make_stage_qk(cfg: StackCfg, layer: int, n_tokens: int, n_seq: int, n_heads: int = 16, n_kv_heads: int = 4,
+                  head_dim: int = 64):
+    """Stand-in for the attention layer's tensors that Eq. 7 reads at a pruning layer: the last tokens' queries
+    [n_seq, n_heads, d] and the keys [n_tokens, n_kv_heads, d] of the sequence as it is at that layer.  Keys are a
+    smooth random walk over the tokens plus noise (neighbouring vision tokens attend alike), bf16 values."""
+    rq, rk = _spawn(cfg.seed * 1000 + 61 + layer, 2)
+    q = rq.standard_normal((n_seq, n_heads, head_dim))
+    walk = np.cumsum(0.15 * rk.standard_normal((n_tokens, n_kv_heads, head_dim)), axis=0)
+    k = walk / (np.abs(walk).max() + 1e-9) * 3.0 + 0.3 * rk.standard_normal((n_tokens, n_kv_heads, head_dim))
+    return round_to_storage(q, "bf16"), round_to_storage(k, "bf16")
+
+
 def interleaved_mask(n_tokens: int, rng: np.random.Generator, p_vis: float = 0.7) -> np.ndarray:
     """A modality mask with text and vision runs interleaved (edge-case tests)."""
     m = np.zeros(n_tokens, dtype=np.uint8)

@@ -196,7 +196,7 @@ class StackWorkload:
     dense=True  : the unreduced, unpruned comparison run (K experts for every token, no stages)."""
 
     def __init__(self, cfg: I.StackCfg, handle: B.Handle, device: int = 0, token_seed: Optional[int] = None,
-                 dense: bool = False, n_layers: Optional[int] = None):
+                 dense: bool = False, n_layers: Optional[int] = None, attention: bool = False):
         self.cfg, self.h = cfg, handle
         lc = cfg.layer
         dev = f"cuda:{device}"
@@ -214,6 +214,19 @@ class StackWorkload:
         self.reduce_from = self.n_layers + 1 if dense else cfg.reduce_from
         self.stages = [] if dense else [(l, pc.retain, B.prune_params(pc.window, pc.gamma, pc.alpha), None)
                                         for l, pc in sorted(cfg.prune_after.items()) if l < self.n_layers]
+        # attention-guided scoring (Eq. 7, 11-13): every stage gets the attention-importance vector of the sequence
+        # as it is at that layer, computed by fmmoe_attention_importance from stand-in queries and keys at every step
+        self.attention = attention and not dense
+        self.qk = {}
+        if self.attention:
+            done = []
+            for i, (l, r, pp, _) in enumerate(self.stages):
+                off_here, _ = B.fmmoe_stack_output_layout(done, l + 1, seq_off, n_vis)
+                q, k = I.make_stage_qk(cfg, l, off_here[-1], len(n_vis))
+                a = torch.empty(off_here[-1], dtype=torch.float32, device=dev)
+                self.qk[l] = (torch.from_numpy(q).to(dev).to(td), torch.from_numpy(k).to(dev).to(td), off_here, a)
+                self.stages[i] = (l, r, pp, a)
+                done.append(self.stages[i])
         self.out_off, self.out_vis = B.fmmoe_stack_output_layout(self.stages, self.n_layers, seq_off, n_vis)
         self.x_out = torch.empty((self.out_off[-1], lc.hidden), dtype=td, device=dev)
         self.mask_out = torch.empty(self.out_off[-1], dtype=torch.uint8, device=dev)
@@ -226,6 +239,8 @@ class StackWorkload:
         return self.cfg.layer.n_tokens
 
     def step(self):
+        for l, (q, k, off_here, a) in self.qk.items():      # Eq. 7 for every pruning layer of this step
+            self.h.fmmoe_attention_importance(q, k, off_here, out=a)
         self.h.fmmoe_stack_forward(self.desc, self.wstructs, self.reduce_from, self.stages, self.x, self.mask,
                                    self.seq_off, self.n_vis, 0, x_out=self.x_out, is_visual_out=self.mask_out)
         return self.x_out
@@ -254,6 +269,8 @@ class StackWorkload:
             self.h.fmmoe_host_wait(sl["ticket"])
         self.h.fmmoe_upload_async(sl["x"], self.x_host)
         self.h.fmmoe_upload_async(sl["mask"], self.mask_host)
+        for l, (q, k, off_here, a) in self.qk.items():
+            self.h.fmmoe_attention_importance(q, k, off_here, out=a)
         self.h.fmmoe_stack_forward(self.desc, self.wstructs, self.reduce_from, self.stages, sl["x"], sl["mask"],
                                    self.seq_off, self.n_vis, 0, x_out=sl["x_out"], is_visual_out=sl["mask_out"])
         self.h.fmmoe_download_async(sl["out_host"], sl["x_out"])

@@ -173,3 +173,68 @@ def test_c4_stack_full():
     h.check_status("layerwise")
     assert cur_off == out_off
     assert torch.equal(cur_x, y) and torch.equal(cur_m, vis_out)
+
+
+@pytest.mark.parametrize("retain", [0.75, 0.5, 0.25])
+@pytest.mark.parametrize("model", ["internvl3.5", "deepseek-vl2"])
+def test_paper_three_stage_schedules_at_full_size(model, retain):
+    """The paper's two schedules (Appendix A: pruning after layers 5/8/12 with W = 5 on the Qwen3-MoE-style layer,
+    after layers 2/5/8 with W = 3 on the DeepSeekMoE-style layer) at 75 / 50 / 25 % overall retention with the
+    per-stage ratio r^(1/3) (Appendix D) and the (alpha, gamma) of that retention, attention-guided: A_hat comes
+    from fmmoe_attention_importance on stand-in queries and keys of each pruning layer.  At every stage the keep-set
+    and the kinds are bit-exact against the oracle (fed the kernel's fp32 probabilities and A_hat), A_hat itself is
+    within 1e-5 of the oracle's Eq. 7, the kept count is in [eta, eta + W), and the stack driver equals the
+    layer-by-layer calls bit for bit (fixed-order combine)."""
+    sc = I.paper_stack(model, retain)
+    lc = sc.layer
+    h = handle()
+    dev_, td = "cuda:0", torch.bfloat16
+    x, mask, seq_off, n_vis = I.make_tokens(lc)
+    xd = torch.from_numpy(x).to(dev_).to(td).contiguous()
+    md = torch.from_numpy(mask).to(dev_)
+    layers = [I.stack_layer_weights_torch(sc, l, dev_) for l in range(sc.n_layers)]
+    wstructs = [B.make_weights(w) for w in layers]
+    desc = B.make_desc(lc.hidden, lc.n_experts, lc.inter, lc.n_shared, lc.shared_inter, lc.top_k, lc.top_k_vis, td)
+    E = lc.n_experts
+    stages, attn_of, done = [], {}, []
+    for layer, pc in sorted(sc.prune_after.items()):
+        off_here, _ = B.fmmoe_stack_output_layout(done, layer + 1, seq_off, n_vis)
+        q, k = I.make_stage_qk(sc, layer, off_here[-1], len(n_vis))
+        a = h.fmmoe_attention_importance(torch.from_numpy(q).to(dev_).to(td), torch.from_numpy(k).to(dev_).to(td), off_here)
+        ref_a = O.attention_importance(q, k, off_here)
+        assert np.abs(host(a) - ref_a).max() <= 1e-5 * max(ref_a.max(), 1e-30) + 1e-9
+        attn_of[layer] = a
+        st = (layer, pc.retain, B.prune_params(pc.window, pc.gamma, pc.alpha), a)
+        stages.append(st); done.append(st)
+    flags = B.FLAG_DETERMINISTIC
+    y, vis_out, out_off = h.fmmoe_stack_forward(desc, wstructs, sc.reduce_from, stages, xd, md, seq_off, n_vis, flags)
+    h.check_status("stack")
+    cur_x, cur_m, cur_off, cur_vis = xd, md, list(seq_off), [int(v) for v in n_vis]
+    n_v0 = int(n_vis[0])
+    for l in range(sc.n_layers):
+        T = cur_x.shape[0]
+        lf = flags | B.FLAG_RESIDUAL | (B.FLAG_REDUCE_ON if l >= sc.reduce_from else 0)
+        route = {"probs": torch.empty(T, E, dtype=torch.float32, device=dev_)}
+        out = h.fmmoe_moe_forward(desc, wstructs[l], cur_x, cur_m, lf, route=route)
+        if l in sc.prune_after:
+            pc = sc.prune_after[l]
+            eta = I.retain_counts(n_vis, pc.retain)
+            pr = h.fmmoe_prune_visual(B.prune_params(pc.window, pc.gamma, pc.alpha), route["probs"], attn_of[l], out,
+                                      cur_m, cur_off, cur_vis, eta)
+            ref = O.prune_visual(host(out), host(cur_m), host(route["probs"]), host(attn_of[l]), cur_off, eta, pc.window,
+                                 pc.alpha, pc.gamma)
+            assert np.array_equal(host(pr["keep_idx"]), ref["keep_idx"]), f"stage after layer {l}"
+            assert np.array_equal(host(pr["kind"]), ref["kind"])
+            assert row_rel_err(host(pr["x_out"]), ref["x_out"]) < TOL
+            n_text = [cur_off[b + 1] - cur_off[b] - cur_vis[b] for b in range(len(cur_vis))]
+            cur_off = pr["out_seq_off"]
+            cur_vis = [cur_off[b + 1] - cur_off[b] - n_text[b] for b in range(len(n_text))]
+            assert int(eta[0]) <= cur_vis[0] < int(eta[0]) + pc.window
+            assert abs(pc.retain - retain ** ((sorted(sc.prune_after).index(l) + 1) / 3.0)) < 1e-12   # beta^t of the original
+            cur_x, cur_m = pr["x_out"], pr["is_visual_out"]
+        else:
+            cur_x = out
+    h.check_status("layerwise")
+    assert cur_off == out_off and torch.equal(cur_x, y) and torch.equal(cur_m, vis_out)
+    assert n_v0 * retain <= cur_vis[0] < n_v0 * retain + 3 * sc.prune_after[max(sc.prune_after)].window
+    assert bool(torch.isfinite(y.float()).all())
