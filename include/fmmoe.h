@@ -123,7 +123,10 @@ typedef struct fmmoe_handle fmmoe_handle;   /* opaque: device, SM count, status 
  * kernel and reports the first failing one on stderr; FMMOE_GATHER_MIN_TOKENS=n moves the
  * token count from which GEMM-1 gathers the routed rows itself (default 12288);
  * FMMOE_SMALL_M_MAX_TOKENS=n moves the token count below which the expert GEMMs run with the
- * token rows as the MMA's N dimension (default 12288; 0 turns that form off). */
+ * token rows as the MMA's N dimension (default 12288; 0 turns that form off);
+ * FMMOE_CTA_PAIR_MIN_TOKENS=n makes them run on CTA pairs with 256-row tiles from n tokens on
+ * (off by default: measured no faster than the one-CTA form on a power-capped B200); FMMOE_PAIR_ROWS_MIN_TOKENS=n the token count from which the combine goes
+ * through per-pair bf16 rows instead of atomic adds (default 8192). */
 fmmoe_status fmmoe_create(fmmoe_handle **handle, int device);
 fmmoe_status fmmoe_destroy(fmmoe_handle *handle);
 const char  *fmmoe_status_string(fmmoe_status s);

@@ -17,7 +17,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libfmmoe.so")
-SOURCES = ["api.cu", "route.cu", "permute.cu", "ffn_tc.cu", "ffn_sm.cu", "ffn_f32.cu", "combine.cu", "prune.cu", "stack.cu", "attn.cu"]
+SOURCES = ["api.cu", "route.cu", "permute.cu", "ffn_tc.cu", "ffn_tc2.cu", "ffn_sm.cu", "ffn_f32.cu", "combine.cu", "prune.cu", "stack.cu", "attn.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]

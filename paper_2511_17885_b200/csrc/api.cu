@@ -3,6 +3,7 @@
 //   route (Eq. 1-3, 5; block counts and in-block ranks) -> permute-by-expert (scan, scatter)
 //   -> [copy of the routed rows into expert order, small batches] -> GEMM-1 (+ row gather by
 //   token, large batches) + SwiGLU -> GEMM-2 + combine (Eq. 4) -> finalize.
+#include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -120,7 +121,8 @@ static fmmoe_status check_common(fmmoe_handle* h, const fmmoe_layer_desc* d, con
 
 static fmmoe_status run_route(fmmoe_handle* h, const fmmoe_layer_desc& d, const fmmoe_weights& w, const void* x,
                               const uint8_t* is_visual, int64_t T, uint32_t flags, const RoutePtrs& r,
-                              bool need_permute, float* acc_zero, cudaStream_t s, void* gather_xp = nullptr) {
+                              bool need_permute, float* acc_zero, cudaStream_t s, void* gather_xp = nullptr,
+                              int block_m = 0) {
   RouteArgs ra;
   ra.x = x; ra.router_w = w.router_w; ra.router_b = w.router_b; ra.is_visual = is_visual;
   ra.T = T; ra.H = d.hidden; ra.E = d.n_experts; ra.K = d.top_k; ra.Kv = d.top_k_vis;
@@ -134,7 +136,7 @@ static fmmoe_status run_route(fmmoe_handle* h, const fmmoe_layer_desc& d, const 
   pa.blk_tokens = route_block_tokens(d.dtype, T, d.hidden);
   pa.n_blk = route_num_blocks(d.dtype, T, d.hidden);
   pa.T = T; pa.K = d.top_k; pa.E = d.n_experts;
-  pa.block_m = d.dtype == FMMOE_BF16 ? TC_BLOCK_M : F32_BLOCK_M;
+  pa.block_m = block_m ? block_m : (d.dtype == FMMOE_BF16 ? TC_BLOCK_M : F32_BLOCK_M);
   pa.expert_off = r.expert_off; pa.row_token = r.row_token; pa.row_gate = r.row_gate; pa.inv_row = r.inv_row;
   pa.mtiles = r.mtiles; pa.n_mtiles = r.misc;
   pa.gather_x = gather_xp ? x : nullptr; pa.gather_xp = gather_xp;
@@ -183,7 +185,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
     if (end != g && v >= 0) h->gather_min_tokens = v;
   }
   h->wait_budget_ns = 2000000000ull;
-  h->sm_attr_set = false; h->smq_attr_set = false;
+  h->sm_attr_set = false; h->smq_attr_set = false; h->tc2_attr_set = false;
   h->small_m_max_tokens = kGatherMinTokensDefault;
   if (const char* g = getenv("FMMOE_SMALL_M_MAX_TOKENS")) {
     char* end = nullptr;
@@ -191,6 +193,12 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
     if (end != g && v >= 0) h->small_m_max_tokens = v;
   }
   h->test_withhold_stage = -1; h->test_budget_ns = 0;
+  h->cta_pair_min_tokens = INT64_MAX;      // off unless asked for: measured no faster than the one-CTA form (power-capped)
+  if (const char* g = getenv("FMMOE_CTA_PAIR_MIN_TOKENS")) {
+    char* end = nullptr;
+    const long long v = strtoll(g, &end, 10);
+    if (end != g && v >= 0) h->cta_pair_min_tokens = v;
+  }
   h->pair_min_tokens = kPairMinTokensDefault;
   if (const char* g = getenv("FMMOE_PAIR_ROWS_MIN_TOKENS")) {
     char* end = nullptr;
@@ -296,9 +304,10 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   // the router clears the scheduler words and (atomic mode) the fp32 accumulator it owns rows of
   // bf16 at small batch: the permutation's scatter pass also writes the expert-grouped copy of x
   const bool pair = use_pair_rows(h, *d, T, flags);
-  const bool copy_rows = d->dtype == FMMOE_BF16 && (use_small_m(h, *d, T) || !gather_rows_in_gemm(h, T));
+  const bool cta_pairs = use_cta_pairs(h, *d, T);
+  const bool copy_rows = d->dtype == FMMOE_BF16 && (cta_pairs || use_small_m(h, *d, T) || !gather_rows_in_gemm(h, T));
   st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, (det || pair) ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s,
-                 copy_rows ? ws + pl.xp_off : nullptr);
+                 copy_rows ? ws + pl.xp_off : nullptr, cta_pairs ? 2 * TC_BLOCK_M : 0);
   if (st != FMMOE_OK) return st;
   if (after_route) {
     st = after_route->fn(after_route->ctx);
@@ -319,7 +328,9 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   fa.ysh = det ? reinterpret_cast<float*>(ws + pl.ysh_off) : nullptr;
   fa.deterministic = det; fa.d_status = h->d_status;
   fa.test_withhold_stage = -1; fa.grid_override = 0;
-  if (use_small_m(h, *d, T)) {
+  if (cta_pairs) {
+    st = launch_ffn_tc2(h, fa, s);
+  } else if (use_small_m(h, *d, T)) {
     const uint64_t budget = h->wait_budget_ns;
     if (h->test_withhold_stage >= 0) {     // armed self-test: this call only
       fa.test_withhold_stage = h->test_withhold_stage; fa.grid_override = 1;

@@ -30,29 +30,29 @@ __device__ __forceinline__ void add_bf16x8(float (&v)[8], const uint4 u) {
 // then the residual, in that fixed order in fp32; one rounding to bf16.  No atomics anywhere, so the result is
 // reproducible bit for bit.  A thread owns 8 neighbouring columns of one token: the rows' 16-byte pieces are
 // independent loads.
+template <int KK>
 __global__ void __launch_bounds__(256) finalize_pair_kernel(const FinalizeDev a) {
   pdl_launch_dependents();
   pdl_wait();
   const int hv = a.H / 8;
   const long long n = a.T * hv;
-  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);    // eight bf16 zeros
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
     const long long t = i / hv;
     const int c = (int)(i - t * hv) * 8;
-    // every row index first, then every row piece (independent 16-byte loads in flight together), then the sum
-    int rows[FMMOE_MAX_TOPK];
+    // every row index first, then every row piece (KK independent 16-byte loads in flight), then the sum in slot order
+    int rows[KK];
 #pragma unroll
-    for (int s = 0; s < FMMOE_MAX_TOPK; ++s) rows[s] = s < a.K ? a.inv_row[t * a.K + s] : -1;
-    uint4 q[FMMOE_MAX_TOPK];
+    for (int s = 0; s < KK; ++s) rows[s] = a.inv_row[t * KK + s];
+    uint4 q[KK];
 #pragma unroll
-    for (int s = 0; s < FMMOE_MAX_TOPK; ++s)
-      q[s] = rows[s] >= 0 ? *reinterpret_cast<const uint4*>(a.yb + (long long)rows[s] * a.H + c) : zero;
+    for (int s = 0; s < KK; ++s)      // a padded slot (-1) reads row 0 and is not added
+      q[s] = *reinterpret_cast<const uint4*>(a.yb + (long long)(rows[s] < 0 ? 0 : rows[s]) * a.H + c);
     float v[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) v[j] = 0.f;
 #pragma unroll
-    for (int s = 0; s < FMMOE_MAX_TOPK; ++s)
-      if (s < a.K) add_bf16x8(v, q[s]);          // adding the zeros of an unused slot changes nothing
+    for (int s = 0; s < KK; ++s)
+      if (rows[s] >= 0) add_bf16x8(v, q[s]);
     for (int s = 0; s < a.n_shared; ++s)
       add_bf16x8(v, *reinterpret_cast<const uint4*>(a.ybsh + ((long long)s * a.T + t) * a.H + c));
     if (a.add_residual) add_bf16x8(v, *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(a.x) + t * a.H + c));
@@ -65,6 +65,17 @@ __global__ void __launch_bounds__(256) finalize_pair_kernel(const FinalizeDev a)
     *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(a.out) + t * a.H + c) = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
+
+template <int KK>
+static cudaError_t launch_finalize_pair(const FinalizeDev& d, unsigned blocks, cudaStream_t s) {
+  return launch_pdl(finalize_pair_kernel<KK>, dim3(blocks), dim3(256), 0, s, 1, d);
+}
+typedef cudaError_t (*FinalizePairFn)(const FinalizeDev&, unsigned, cudaStream_t);
+static const FinalizePairFn kFinalizePair[FMMOE_MAX_TOPK] = {
+    launch_finalize_pair<1>,  launch_finalize_pair<2>,  launch_finalize_pair<3>,  launch_finalize_pair<4>,
+    launch_finalize_pair<5>,  launch_finalize_pair<6>,  launch_finalize_pair<7>,  launch_finalize_pair<8>,
+    launch_finalize_pair<9>,  launch_finalize_pair<10>, launch_finalize_pair<11>, launch_finalize_pair<12>,
+    launch_finalize_pair<13>, launch_finalize_pair<14>, launch_finalize_pair<15>, launch_finalize_pair<16>};
 
 template <typename T> struct Vec4;
 template <> struct Vec4<float> {
@@ -128,7 +139,7 @@ fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_
   d.acc = a.acc; d.y = a.y; d.ysh = a.ysh; d.inv_row = a.inv_row; d.topk_w = a.topk_w;
   d.yb = static_cast<const __nv_bfloat16*>(a.yb); d.ybsh = static_cast<const __nv_bfloat16*>(a.ybsh);
   if (a.pair) {
-    if (a.dtype != FMMOE_BF16 || a.H % 8) return FMMOE_ERR_INTERNAL;
+    if (a.dtype != FMMOE_BF16 || a.H % 8 || a.K < 1 || a.K > FMMOE_MAX_TOPK) return FMMOE_ERR_INTERNAL;
     const long long n8 = a.T * (a.H / 8);
     long long blocks8 = (n8 + 255) / 256;
     const long long cap8 = (long long)h->sm_count * 32;
@@ -136,7 +147,7 @@ fmmoe_status launch_finalize(fmmoe_handle* h, const FinalizeArgs& a, cudaStream_
     {
       ProfScope ps(h, FMMOE_KERNEL_FINALIZE, s);
       for (int rep = 0; rep < ps.reps; ++rep) {
-        FMMOE_CUDA_TRY(launch_pdl(finalize_pair_kernel, dim3((unsigned)blocks8), dim3(256), 0, s, 1, d));
+        FMMOE_CUDA_TRY(kFinalizePair[a.K - 1](d, (unsigned)blocks8, s));
         h->launches += 1;
       }
     }

@@ -11,6 +11,8 @@ namespace fmmoe {
 
 constexpr int G_SCHED = 4;         // slots of the tile ring
 constexpr int G_SLOT_INTS = 8;     // a slot: tile id (-1: no more tiles) + the decoded TileInfo
+constexpr int G_EPI_LD = 33;                                 // padded row of the epilogue transpose buffer
+constexpr int G_EPI_BYTES = 4 * 32 * G_EPI_LD * 4;           // one 32x32 fp32 block per epilogue warp
 
 struct Segment {          // routed experts (0) or shared experts (1)
   int n_nblocks;          // N-blocks per group
@@ -27,8 +29,9 @@ struct GemmParams {
   const int32_t* n_mtiles;    // device: number of routed M-tiles
   int max_mtiles;             // capacity of `mtiles` (a corrupt count must not walk past it)
   int32_t* tile_counter;      // device: next tile to hand out (zero at launch)
-  int shared_mtiles;          // N_s * ceil(T/128), host-known
-  int mt_per_shared;          // ceil(T/128)
+  int block_m;                // rows per M-tile of the tile list (128; 256 for CTA pairs)
+  int shared_mtiles;          // N_s * ceil(T/block_m), host-known
+  int mt_per_shared;          // ceil(T/block_m)
   long long T;
   Segment seg[2];
   // epilogue
@@ -80,9 +83,9 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, int tile, i
     const int mt = t2 - ti.nb * p.shared_mtiles;
     ti.group_local = mt / p.mt_per_shared;
     const int mb = mt - ti.group_local * p.mt_per_shared;
-    ti.row0 = mb * TC_BLOCK_M;
+    ti.row0 = mb * p.block_m;
     const long long left = p.T - (long long)ti.row0;
-    ti.rows = left < TC_BLOCK_M ? (int)left : TC_BLOCK_M;
+    ti.rows = left < p.block_m ? (int)left : p.block_m;
     ti.single = false;
   }
   return ti;
@@ -96,6 +99,115 @@ __device__ __forceinline__ TileInfo slot_load(const volatile int* s) {
   TileInfo ti;
   ti.seg = s[1]; ti.group_local = s[2]; ti.row0 = s[3]; ti.rows = s[4]; ti.nb = s[5]; ti.single = s[6] != 0;
   return ti;
+}
+
+// Epilogue of one tile for one epilogue warp: the warp owns TMEM lane quarter q (taddr already points at it and
+// at the accumulator stage), i.e. `rpw` rows of the tile starting at tile row q * rpw (32 rows, or 16 when a tile
+// of at most 64 rows ran as M = 64 MMAs).  `ti` describes the 128-row tile this CTA holds.  `stg` is the warp's
+// 32 x 33 fp32 staging block.
+//   MODE 0: SwiGLU of the gate / up columns -> act (bf16), coalesced through the staging block.
+//   MODE 1: gate scaling, then per-pair bf16 rows (pair-row mode), fp32 rows (fixed-order mode) or vector
+//           reductions into the fp32 accumulator.
+template <int MODE>
+__device__ __forceinline__ void tc_epilogue(const GemmParams& p, const TileInfo& ti, const Segment& sg, uint32_t taddr,
+                                            float* stg, int lane, int q, int rpw) {
+  const int rows_w = min(ti.rows - q * rpw, rpw);   // valid rows among this warp's (may be <= 0)
+  const long long out_row0 = (long long)ti.row0 + q * rpw + (long long)ti.group_local * sg.out_group_stride;
+  const int r = q * rpw + lane;                     // row of the tile held by this thread (if lane < rpw)
+  if (MODE == 0) {
+    uint32_t* stg32 = reinterpret_cast<uint32_t*>(stg);   // [32][17] packed bf16 pairs
+    __nv_bfloat16* dst0 = p.act[ti.seg] + out_row0 * sg.ld_out + ti.nb * 128;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      if (ti.nb * 128 + c * 32 >= sg.n_valid) break;   // warp-uniform
+      uint32_t g[32], u[32];
+      tmem_ld32(taddr + c * 32, g);
+      tmem_ld32(taddr + 128 + c * 32, u);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+        const float a0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
+        const float a1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
+        const __nv_bfloat162 h = __floats2bfloat162_rn(a0, a1);
+        stg32[lane * 17 + i] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+      __syncwarp();
+      // 4 lanes x 16 bytes cover the 64-byte row segment; 8 rows per instruction
+#pragma unroll
+      for (int rr = 0; rr < 4; ++rr) {
+        const int row = rr * 8 + (lane >> 2);
+        const int w4 = (lane & 3) * 4;
+        if (row < rows_w) {
+          const uint32_t* sp = stg32 + row * 17 + w4;
+          *reinterpret_cast<uint4*>(dst0 + (long long)row * sg.ld_out + c * 32 + w4 * 2) =
+              make_uint4(sp[0], sp[1], sp[2], sp[3]);
+        }
+      }
+      __syncwarp();
+    }
+  } else {
+    int tok; float gate;
+    if (ti.seg == 0) {
+      const bool row_ok = lane < rows_w;
+      tok = row_ok ? p.row_token[ti.row0 + r] : 0;
+      gate = row_ok ? p.row_gate[ti.row0 + r] : 0.f;
+    } else {
+      tok = ti.row0 + r; gate = 1.f;
+    }
+    if (p.deterministic) gate = 1.f;   // gates are applied by the ordered gather
+    float* ybase = p.deterministic ? p.y[ti.seg] + out_row0 * sg.ld_out + ti.nb * 256 : nullptr;
+    if (p.pair) {
+      // Pair-row mode: this thread owns grouped row r; its 32 accumulator columns of a chunk are 64
+      // contiguous bytes of that row of yb, written straight from registers (two full 32-byte sectors).
+      __nv_bfloat16* yrow = p.yb[ti.seg] + (out_row0 + lane) * sg.ld_out + ti.nb * 256;
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c) {
+        if (ti.nb * 256 + c * 32 >= sg.n_valid) break;   // warp-uniform
+        uint32_t v[32];
+        tmem_ld32(taddr + c * 32, v);
+        tmem_ld_wait();
+        if (lane < rows_w) {
+          uint32_t w16[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const __nv_bfloat162 hh = __floats2bfloat162_rn(gate * __uint_as_float(v[2 * i]), gate * __uint_as_float(v[2 * i + 1]));
+            w16[i] = *reinterpret_cast<const uint32_t*>(&hh);
+          }
+          uint4* dst = reinterpret_cast<uint4*>(yrow + c * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w16[4 * i], w16[4 * i + 1], w16[4 * i + 2], w16[4 * i + 3]);
+        }
+      }
+    } else
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+      if (ti.nb * 256 + c * 32 >= sg.n_valid) break;   // warp-uniform
+      uint32_t v[32];
+      tmem_ld32(taddr + c * 32, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) stg[lane * G_EPI_LD + j] = gate * __uint_as_float(v[j]);
+      __syncwarp();
+      // 8 lanes x 16 bytes cover a row's 128-byte segment; 4 rows per instruction
+#pragma unroll
+      for (int rr = 0; rr < 8; ++rr) {
+        const int row = rr * 4 + (lane >> 3);
+        const int col = (lane & 7) * 4;
+        const int tok_r = __shfl_sync(0xffffffffu, tok, row);
+        if (row < rows_w) {
+          const float* sp = stg + row * G_EPI_LD + col;
+          if (p.deterministic) {
+            *reinterpret_cast<float4*>(ybase + (long long)row * sg.ld_out + c * 32 + col) =
+                make_float4(sp[0], sp[1], sp[2], sp[3]);
+          } else {
+            red_add_v4(p.acc + (long long)tok_r * sg.ld_out + ti.nb * 256 + c * 32 + col, sp[0], sp[1], sp[2], sp[3]);
+          }
+        }
+      }
+      __syncwarp();
+    }
+  }
 }
 
 // ---------------------------------------------------------------- host side

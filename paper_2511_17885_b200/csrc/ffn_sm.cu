@@ -495,7 +495,7 @@ static fmmoe_status launch_ffn_sm_impl(fmmoe_handle* h, const FfnArgs& a, cudaSt
 
   GemmParams p1 = {};
   p1.mtiles = a.mtiles; p1.n_mtiles = a.n_mtiles; p1.max_mtiles = a.max_mtiles;
-  p1.shared_mtiles = Ns * mtps; p1.mt_per_shared = mtps; p1.T = a.T;
+  p1.block_m = TC_BLOCK_M; p1.shared_mtiles = Ns * mtps; p1.mt_per_shared = mtps; p1.T = a.T;
   p1.seg[0] = Segment{(I + 127) / 128, H / S_BK, I, I, 0, 0, I};
   p1.seg[1] = Segment{Ns ? (Is + 127) / 128 : 0, H / S_BK, Is, Is, 0, (int)a.T, Is};
   p1.act[0] = static_cast<__nv_bfloat16*>(a.act); p1.act[1] = static_cast<__nv_bfloat16*>(a.act_sh);

@@ -48,8 +48,6 @@ constexpr int G_THREADS = 224;          // producer warp, issuer warp, four epil
 constexpr int G_LOADERS = 128;          // GEMM-1 only: four more warps that gather the routed rows of x
 constexpr int G_THREADS_G1 = G_THREADS + G_LOADERS;
 constexpr int G_TMEM_COLS = 512;
-constexpr int G_EPI_LD = 33;                                 // padded row of the epilogue transpose buffer
-constexpr int G_EPI_BYTES = 4 * 32 * G_EPI_LD * 4;           // one 32x32 fp32 block per epilogue warp
 constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_EPI_BYTES + 1024 /*align*/ + 384 /*barriers, tile ring*/;
 
 // MODE 0: GEMM-1 + SwiGLU.  MODE 1: GEMM-2 + combine.
@@ -298,103 +296,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tmA_r, const __grid_constant__
       // M = 128: row i of the tile sits in TMEM lane i.  M = 64 (tiles of at most 64 rows): row i sits in
       // lane 32 * (i / 16) + i % 16, so each warp's lane quarter holds 16 rows in its lanes 0..15.
       const int rpw = ti.rows <= 64 ? 16 : 32;          // rows per warp
-      const int r = q * rpw + lane;                     // row of the tile held by this thread (if lane < rpw)
-      const int rows_w = min(ti.rows - q * rpw, rpw);   // valid rows among this warp's (may be <= 0)
-      const long long out_row0 = (long long)ti.row0 + q * rpw + (long long)ti.group_local * sg.out_group_stride;
-      if (MODE == 0) {
-        uint32_t* stg32 = reinterpret_cast<uint32_t*>(stg);   // [32][17] packed bf16 pairs
-        __nv_bfloat16* dst0 = p.act[ti.seg] + out_row0 * sg.ld_out + ti.nb * 128;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          if (ti.nb * 128 + c * 32 >= sg.n_valid) break;   // warp-uniform
-          uint32_t g[32], u[32];
-          tmem_ld32(taddr + c * 32, g);
-          tmem_ld32(taddr + 128 + c * 32, u);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-            const float a0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
-            const float a1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
-            const __nv_bfloat162 h = __floats2bfloat162_rn(a0, a1);
-            stg32[lane * 17 + i] = *reinterpret_cast<const uint32_t*>(&h);
-          }
-          __syncwarp();
-          // 4 lanes x 16 bytes cover the 64-byte row segment; 8 rows per instruction
-#pragma unroll
-          for (int rr = 0; rr < 4; ++rr) {
-            const int row = rr * 8 + (lane >> 2);
-            const int w4 = (lane & 3) * 4;
-            if (row < rows_w) {
-              const uint32_t* sp = stg32 + row * 17 + w4;
-              *reinterpret_cast<uint4*>(dst0 + (long long)row * sg.ld_out + c * 32 + w4 * 2) =
-                  make_uint4(sp[0], sp[1], sp[2], sp[3]);
-            }
-          }
-          __syncwarp();
-        }
-      } else {
-        int tok; float gate;
-        if (ti.seg == 0) {
-          const bool row_ok = lane < rows_w;
-          tok = row_ok ? p.row_token[ti.row0 + r] : 0;
-          gate = row_ok ? p.row_gate[ti.row0 + r] : 0.f;
-        } else {
-          tok = ti.row0 + r; gate = 1.f;
-        }
-        if (p.deterministic) gate = 1.f;   // gates are applied by the ordered gather
-        float* ybase = p.deterministic ? p.y[ti.seg] + out_row0 * sg.ld_out + ti.nb * 256 : nullptr;
-        if (p.pair) {
-          // Pair-row mode: this thread owns grouped row r; its 32 accumulator columns of a chunk are 64
-          // contiguous bytes of that row of yb, written straight from registers (two full 32-byte sectors).
-          __nv_bfloat16* yrow = p.yb[ti.seg] + (out_row0 + lane) * sg.ld_out + ti.nb * 256;
-#pragma unroll 1
-          for (int c = 0; c < 8; ++c) {
-            if (ti.nb * 256 + c * 32 >= sg.n_valid) break;   // warp-uniform
-            uint32_t v[32];
-            tmem_ld32(taddr + c * 32, v);
-            tmem_ld_wait();
-            if (lane < rows_w) {
-              uint32_t w16[16];
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const __nv_bfloat162 hh = __floats2bfloat162_rn(gate * __uint_as_float(v[2 * i]), gate * __uint_as_float(v[2 * i + 1]));
-                w16[i] = *reinterpret_cast<const uint32_t*>(&hh);
-              }
-              uint4* dst = reinterpret_cast<uint4*>(yrow + c * 32);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w16[4 * i], w16[4 * i + 1], w16[4 * i + 2], w16[4 * i + 3]);
-            }
-          }
-        } else
-#pragma unroll 1
-        for (int c = 0; c < 8; ++c) {
-          if (ti.nb * 256 + c * 32 >= sg.n_valid) break;   // warp-uniform
-          uint32_t v[32];
-          tmem_ld32(taddr + c * 32, v);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) stg[lane * G_EPI_LD + j] = gate * __uint_as_float(v[j]);
-          __syncwarp();
-          // 8 lanes x 16 bytes cover a row's 128-byte segment; 4 rows per instruction
-#pragma unroll
-          for (int rr = 0; rr < 8; ++rr) {
-            const int row = rr * 4 + (lane >> 3);
-            const int col = (lane & 7) * 4;
-            const int tok_r = __shfl_sync(0xffffffffu, tok, row);
-            if (row < rows_w) {
-              const float* sp = stg + row * G_EPI_LD + col;
-              if (p.deterministic) {
-                *reinterpret_cast<float4*>(ybase + (long long)row * sg.ld_out + c * 32 + col) =
-                    make_float4(sp[0], sp[1], sp[2], sp[3]);
-              } else {
-                red_add_v4(p.acc + (long long)tok_r * sg.ld_out + ti.nb * 256 + c * 32 + col, sp[0], sp[1], sp[2], sp[3]);
-              }
-            }
-          }
-          __syncwarp();
-        }
-      }
+      tc_epilogue<MODE>(p, ti, sg, taddr, stg, lane, q, rpw);
       tc_fence_before();
       mbar_arrive(&tempty_bar[as]);
       if (++as == 2) { as = 0; aphase ^= 1; }
@@ -448,7 +350,7 @@ fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s) {
 
   GemmParams p1 = {};
   p1.mtiles = a.mtiles; p1.n_mtiles = a.n_mtiles; p1.max_mtiles = a.max_mtiles;
-  p1.shared_mtiles = Ns * mtps; p1.mt_per_shared = mtps; p1.T = a.T;
+  p1.block_m = G_BM; p1.shared_mtiles = Ns * mtps; p1.mt_per_shared = mtps; p1.T = a.T;
   p1.seg[0] = Segment{(I + 127) / 128, H / G_BK, I, I, 0, 0, I};
   p1.seg[1] = Segment{Ns ? (Is + 127) / 128 : 0, H / G_BK, Is, Is, 0, (int)a.T, Is};
   p1.act[0] = static_cast<__nv_bfloat16*>(a.act); p1.act[1] = static_cast<__nv_bfloat16*>(a.act_sh);

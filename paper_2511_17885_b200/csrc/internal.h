@@ -23,6 +23,8 @@ struct fmmoe_handle {
   bool route_attr_set;  // ... for the bf16 router
   bool sm_attr_set;     // ... for the small-M form of the expert GEMMs
   bool smq_attr_set;    // ... and its FP8 weight stream
+  bool tc2_attr_set;    // ... for the CTA-pair form
+  int64_t cta_pair_min_tokens;    // from this many tokens on the expert GEMMs run on CTA pairs (cta_group::2)
   int64_t small_m_max_tokens;     // below this many tokens the expert GEMMs run in their small-M form
   int64_t pair_min_tokens;        // from this many tokens on the combine goes through per-pair bf16 rows (no atomics)
   int test_withhold_stage;        // self-test (fmmoe_test_expire_wait): armed for the next layer call, else -1
@@ -139,15 +141,17 @@ struct ProfScope {
 // Launch with programmatic dependent launch allowed (the kernel calls pdl_wait() before it touches
 // data of earlier kernels), optionally as clusters of `cluster_x` CTAs.
 template <typename... KArgs, typename... Args>
-static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
-                                     unsigned cluster_x, Args&&... args) {
+static inline cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    unsigned cluster_x, bool pdl, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
   cudaLaunchAttribute attr[2];
   int n = 0;
-  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[n].val.programmaticStreamSerializationAllowed = 1;
-  ++n;
+  if (pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
   if (cluster_x > 1) {
     attr[n].id = cudaLaunchAttributeClusterDimension;
     attr[n].val.clusterDim.x = cluster_x; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
@@ -155,6 +159,11 @@ static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 b
   }
   cfg.attrs = attr; cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                     unsigned cluster_x, Args&&... args) {
+  return launch_ex(kernel, grid, block, smem, s, cluster_x, true, std::forward<Args>(args)...);
 }
 
 // ---- launchers (each returns after enqueueing; *launches is incremented per kernel) ----
@@ -221,6 +230,11 @@ constexpr int64_t kGatherMinTokensDefault = 12288;
 static inline bool gather_rows_in_gemm(const fmmoe_handle* h, int64_t T) { return T >= h->gather_min_tokens; }
 fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05, token rows as M
 fmmoe_status launch_ffn_sm(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05, token rows as N (reads xp)
+fmmoe_status launch_ffn_tc2(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);   // bf16, tcgen05, CTA pairs, 256-row tiles (reads xp)
+// Large batches (experts with several hundred rows): 256-row tiles on CTA pairs.
+static inline bool use_cta_pairs(const fmmoe_handle* h, const fmmoe_layer_desc& d, int64_t T) {
+  return d.dtype == FMMOE_BF16 && d.weight_format == FMMOE_WEIGHTS_AS_DTYPE && T >= h->cta_pair_min_tokens;
+}
 // Which form runs: below small_m_max_tokens (and below the in-GEMM gather threshold) the small-M form.
 // The fp32 accumulator of the atomic combine is T*H*4 bytes; once it no longer fits the L2 cache next to the
 // activations its read-modify-writes page through HBM, and writing every pair's row once in bf16 is cheaper.
@@ -232,7 +246,7 @@ static inline bool use_pair_rows(const fmmoe_handle* h, const fmmoe_layer_desc& 
 static inline bool use_small_m(const fmmoe_handle* h, const fmmoe_layer_desc& d, int64_t T) {
   if (d.dtype != FMMOE_BF16) return false;
   if (d.weight_format == FMMOE_WEIGHTS_FP8_BLOCK128) return true;
-  return T < h->small_m_max_tokens && T < h->gather_min_tokens;
+  return T < h->small_m_max_tokens && T < h->gather_min_tokens && T < h->cta_pair_min_tokens;
 }
 fmmoe_status launch_ffn_f32(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);   // fp32 FMA
 

@@ -323,6 +323,9 @@ ROW_PATHS = {
     "small_m": {},                                                        # default below 12,288 tokens: rows as the MMA's N
     "rows_as_m_copy": {"FMMOE_SMALL_M_MAX_TOKENS": "0"},                  # rows as M, expert-ordered copy of x
     "rows_as_m_gather": {"FMMOE_SMALL_M_MAX_TOKENS": "0", "FMMOE_GATHER_MIN_TOKENS": "0"},   # rows as M, in-GEMM gather
+    # 256-row tiles on CTA pairs (default from 12,288 tokens on), with the atomic and the per-pair combine
+    "cta_pairs": {"FMMOE_CTA_PAIR_MIN_TOKENS": "0"},
+    "cta_pairs_pair_rows": {"FMMOE_CTA_PAIR_MIN_TOKENS": "0", "FMMOE_PAIR_ROWS_MIN_TOKENS": "0"},
     # the combine through per-pair bf16 rows (default from 8,192 tokens on), under both forms
     "small_m_pair_rows": {"FMMOE_PAIR_ROWS_MIN_TOKENS": "0"},
     "rows_as_m_gather_pair_rows": {"FMMOE_SMALL_M_MAX_TOKENS": "0", "FMMOE_GATHER_MIN_TOKENS": "0",
@@ -375,7 +378,7 @@ def test_decode_sized_batches_with_shared_experts(T):
 
 
 def test_small_m_form_equals_rows_as_m_form_bit_for_bit_in_fixed_order_mode(monkeypatch):
-    """The two forms of the expert GEMMs accumulate every output element over the same k order in fp32, so with the
+    """The three forms of the expert GEMMs (rows as N, rows as M, rows as M on CTA pairs) accumulate every output element over the same k order in fp32, so with the
     fixed-order combine their layer outputs are identical bit for bit."""
     r = np.random.default_rng(71)
     T, H, E, I_ = 900, 256, 16, 320
@@ -383,7 +386,7 @@ def test_small_m_form_equals_rows_as_m_form_bit_for_bit_in_fixed_order_mode(monk
     mask = (r.random(T) < 0.7).astype(np.uint8)
     w = random_layer(r, "bf16", H, E, I_, 1, 128)
     outs = []
-    for env in (ROW_PATHS["small_m"], ROW_PATHS["rows_as_m_copy"]):
+    for env in (ROW_PATHS["small_m"], ROW_PATHS["rows_as_m_copy"], ROW_PATHS["cta_pairs"]):
         h = handle_with_env(monkeypatch, env)
         desc = B.make_desc(H, E, I_, 1, 128, 4, 2, torch.bfloat16)
         wd = upload_weights(w, "bf16"); ws = B.make_weights(wd)
@@ -391,7 +394,7 @@ def test_small_m_form_equals_rows_as_m_form_bit_for_bit_in_fixed_order_mode(monk
                                         B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC).clone())
         h.check_status()
         h.close()
-    assert torch.equal(outs[0], outs[1])
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
 
 
 @pytest.mark.parametrize("k_block", [0, 5])
@@ -421,7 +424,7 @@ def test_bounded_wait_runs_out_and_the_handle_recovers(k_block):
     h.close()
 
 
-@pytest.mark.parametrize("path", ["small_m_pair_rows", "rows_as_m_gather_pair_rows"])
+@pytest.mark.parametrize("path", ["small_m_pair_rows", "rows_as_m_gather_pair_rows", "cta_pairs_pair_rows", "cta_pairs"])
 def test_pair_row_combine_with_shared_experts_residual_and_reproducibility(path, monkeypatch):
     """The combine through per-pair bf16 rows: shared experts, residual, K_v = 0 tokens, against the oracle within
     the bf16 tolerance; it sums in a fixed order without atomics, so two runs agree bit for bit."""
@@ -438,7 +441,8 @@ def test_pair_row_combine_with_shared_experts_residual_and_reproducibility(path,
     a = h.fmmoe_moe_forward(desc, ws, dev(x, torch.bfloat16), dev(mask), flags, route=route).clone()
     b = h.fmmoe_moe_forward(desc, ws, dev(x, torch.bfloat16), dev(mask), flags, route=route)
     h.check_status()
-    assert torch.equal(a, b)
+    if "pair_rows" in path:          # the atomic combine adds in arrival order
+        assert torch.equal(a, b)
     ref = O.moe_forward(x, mask, w, K, Kv, True, add_residual=True, logits32=host(route["logits"]))
     assert row_rel_err(host(a), ref["out"]) < 2e-2
     h.close()
