@@ -158,26 +158,33 @@ __device__ __forceinline__ void tc_epilogue(const GemmParams& p, const TileInfo&
     if (p.deterministic) gate = 1.f;   // gates are applied by the ordered gather
     float* ybase = p.deterministic ? p.y[ti.seg] + out_row0 * sg.ld_out + ti.nb * 256 : nullptr;
     if (p.pair) {
-      // Pair-row mode: this thread owns grouped row r; its 32 accumulator columns of a chunk are 64
-      // contiguous bytes of that row of yb, written straight from registers (two full 32-byte sectors).
-      __nv_bfloat16* yrow = p.yb[ti.seg] + (out_row0 + lane) * sg.ld_out + ti.nb * 256;
+      // Pair-row mode: gate-scaled bf16 rows per pair.  As in GEMM-1's epilogue the 32 x 32 block goes through
+      // the staging block so that every store instruction writes whole 64-byte row segments (4 lanes x 16
+      // bytes per row, 8 rows per instruction) instead of 32 quarter-segments of 32 different rows.
+      uint32_t* stg32 = reinterpret_cast<uint32_t*>(stg);   // [32][17] packed bf16 pairs
+      __nv_bfloat16* y0 = p.yb[ti.seg] + out_row0 * sg.ld_out + ti.nb * 256;
 #pragma unroll 1
       for (int c = 0; c < 8; ++c) {
         if (ti.nb * 256 + c * 32 >= sg.n_valid) break;   // warp-uniform
         uint32_t v[32];
         tmem_ld32(taddr + c * 32, v);
         tmem_ld_wait();
-        if (lane < rows_w) {
-          uint32_t w16[16];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const __nv_bfloat162 hh = __floats2bfloat162_rn(gate * __uint_as_float(v[2 * i]), gate * __uint_as_float(v[2 * i + 1]));
-            w16[i] = *reinterpret_cast<const uint32_t*>(&hh);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(yrow + c * 32);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w16[4 * i], w16[4 * i + 1], w16[4 * i + 2], w16[4 * i + 3]);
+        for (int i = 0; i < 16; ++i) {
+          const __nv_bfloat162 hh = __floats2bfloat162_rn(gate * __uint_as_float(v[2 * i]), gate * __uint_as_float(v[2 * i + 1]));
+          stg32[lane * 17 + i] = *reinterpret_cast<const uint32_t*>(&hh);
         }
+        __syncwarp();
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr) {
+          const int row = rr * 8 + (lane >> 2);
+          const int w4 = (lane & 3) * 4;
+          if (row < rows_w) {
+            const uint32_t* sp = stg32 + row * 17 + w4;
+            *reinterpret_cast<uint4*>(y0 + (long long)row * sg.ld_out + c * 32 + w4 * 2) = make_uint4(sp[0], sp[1], sp[2], sp[3]);
+          }
+        }
+        __syncwarp();
       }
     } else
 #pragma unroll 1

@@ -493,10 +493,55 @@ __global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const Pr
       mem[k] = tkn;
     }
     const float invW = 1.f / (float)a.W;
-    // pass 1: squared norms of the members and of the mean
     float part[MAXW + 1];
 #pragma unroll
     for (int k = 0; k <= MAXW; ++k) part[k] = 0.f;
+    if (vec <= 256) {
+      // One 16-byte piece per thread and member row: the W pieces stay in registers between the norm pass and
+      // the store, so the member rows are read once (the same sums in the same order as the two-pass form below).
+      float mean[N];
+#pragma unroll
+      for (int j = 0; j < N; ++j) mean[j] = 0.f;
+      if (tid < vec) {
+#pragma unroll
+        for (int k = 0; k < MAXW; ++k) {
+          if (k < a.W) {
+            float f[N];
+            Row8<T>::load(X + mem[k] * a.H + tid * N, f);
+#pragma unroll
+            for (int j = 0; j < N; ++j) { part[k] = fmaf(f[j], f[j], part[k]); mean[j] += f[j]; }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < N; ++j) { const float mv = mean[j] * invW; part[MAXW] = fmaf(mv, mv, part[MAXW]); }
+      }
+#pragma unroll
+      for (int k = 0; k <= MAXW; ++k) {
+        float v = part[k];
+#pragma unroll
+        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) s_red[warp][k] = v;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        float tot[MAXW + 1];
+        for (int k = 0; k <= MAXW; ++k) { tot[k] = 0.f; for (int ww = 0; ww < 8; ++ww) tot[k] += s_red[ww][k]; }
+        float nmax = 0.f;
+        for (int k = 0; k < a.W; ++k) nmax = fmaxf(nmax, sqrtf(tot[k]));
+        const float nb = sqrtf(tot[MAXW]);
+        s_scale = a.merge_mode == 1 ? 1.f : (nb > 0.f ? nmax / nb : 0.f);   // Eq. 18
+      }
+      __syncthreads();
+      if (tid < vec) {
+        const float scale = s_scale * invW;
+#pragma unroll
+        for (int j = 0; j < N; ++j) mean[j] *= scale;
+        Row8<T>::store(O + tid * N, mean);
+      }
+      __syncthreads();   // s_red / s_scale are reused by the block's next merged row
+      continue;
+    }
+    // pass 1: squared norms of the members and of the mean
     for (int i = tid; i < vec; i += 256) {
       float mean[N];
 #pragma unroll
