@@ -52,7 +52,11 @@ NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # the nominal peaks the m
 # DRAM bytes (read + written) one launch of a kernel moved under the profiler, per workload.
 # Each figure comes from one capture of that kernel on that workload; an entry is removed (null in
 # the output) when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    "C2x4": {"gemm1": 1101.6e6, "gemm2": 723.2e6, "route": 60.1e6, "finalize": 296.1e6},   # ffn_tc_kernel<0/1>, route_tc, finalize_pair
+    "C1": {"gemm1": 872.3e6, "gemm2": 493.8e6},                                             # ffn_sm_kernel<0/1, 0>
+    "C1_fp8": {"gemm1": 501.7e6, "gemm2": 293.8e6},                                         # ffn_sm_kernel<0/1, 1>
+}
 
 
 def load_peaks():
@@ -663,13 +667,18 @@ def measure_stack(args, D, rank, local, world, peaks, with_cpu, sc=None, label="
     dom = max(prof, key=lambda k: prof[k]["ms"])
     per_launch_s = prof[dom]["ms"] * 1e-3 / max(prof[dom]["launches"], 1)
     flops_per_launch = {"gemm1": g1, "gemm2": g2, "route": rt}.get(dom, 0.0) / n_layers
-    roof = {"bound": "tensor", "achieved": flops_per_launch / per_launch_s / 1e12, "peak": peaks["tf_sustained"],
-            "peak_nominal": NOMINAL["bf16_tflops"], "unit": "TFLOP/s", "kernel": dom, "us_per_launch": per_launch_s * 1e6,
-            "algorithmic_flops": flops_per_launch, "traffic": NCU_TRAFFIC_BYTES.get(label, {}).get(dom),
-            "peak_source": peaks["source"] + " (sustained bf16)",
-            "note": "per-launch figures are the mean over the stack's layers (three different token counts)"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["frac_of_nominal"] = roof["achieved"] / roof["peak_nominal"]
+    # bytes per launch of the dominant kernel, mean over the layers (every expert counted as touched)
+    lc = sc.layer
+    e = 2
+    H, E, I_, Ns, Is = lc.hidden, lc.n_experts, lc.inter, lc.n_shared, lc.shared_inter
+    if dom == "gemm1":
+        bytes_per_launch = sum(E * 2 * H * I_ * e + Ns * 2 * H * Is * e + T * H * e + (P * I_ + Ns * T * Is) * e for T, P in shapes) / n_layers
+    elif dom == "gemm2":
+        bytes_per_launch = sum(E * H * I_ * e + Ns * H * Is * e + (P * I_ + Ns * T * Is) * e + T * H * e for T, P in shapes) / n_layers
+    else:
+        bytes_per_launch = 0.0
+    roof = roofline_of(dom, bytes_per_launch, flops_per_launch, per_launch_s, peaks, NCU_TRAFFIC_BYTES.get(label, {}).get(dom))
+    roof["note"] = "per-launch figures are the mean over the stack's layers (their token counts differ)"
     t_bound = max((g1 + g2 + rt) / (peaks["tf_sustained"] * 1e12), n_layers * weight_bytes(sc.layer) / (peaks["hbm_gbs"] * 1e9))
     t_bound_nom = max((g1 + g2 + rt) / (NOMINAL["bf16_tflops"] * 1e12), n_layers * weight_bytes(sc.layer) / (NOMINAL["hbm_gbs"] * 1e9))
     tot_ms = max(sum(x["ms"] for x in prof.values()), 1e-12)
@@ -714,7 +723,8 @@ def measure_stack(args, D, rank, local, world, peaks, with_cpu, sc=None, label="
                    "d2h_bytes_per_step": wl.d2h_bytes(), "batches_in_flight": wl.PIPE_DEPTH, "batches_timed": n_e2e,
                    "value_one_batch_at_a_time": e2e_serial},
            "gpu_launches": int(launches * K), "roofline": roof,
-           "step_roofline": {"frac": t_bound / step_s, "frac_of_nominal": t_bound_nom / step_s, "bound": "tensor",
+           "step_roofline": {"frac": t_bound / step_s, "frac_of_nominal": t_bound_nom / step_s,
+                             "bound": "tensor" if (g1 + g2 + rt) / (peaks["tf_sustained"] * 1e12) >= n_layers * weight_bytes(sc.layer) / (peaks["hbm_gbs"] * 1e9) else "hbm",
                              "t_bound_us": t_bound * 1e6, "activated_flops": g1 + g2 + rt, "peak_source": peaks["source"]},
            "kernels": kernels, "dense_k_unpruned": dense}
     if with_cpu:

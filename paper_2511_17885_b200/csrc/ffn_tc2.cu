@@ -1,13 +1,12 @@
 // Expert FFNs on the tcgen05 tensor cores with CTA pairs (cta_group::2), for batches whose experts hold
 // several hundred rows.
 //
-// At that size the grouped GEMMs of Eq. 4 are a dense contraction and should run at the tensor cores' rate, but
-// a single CTA computing a 128 x 256 tile has to bring 48 KB into shared memory per 64-deep k-block (128 rows of
-// activations, 256 rows of weights) for 512 tensor-core cycles of work: 96 bytes per cycle, where an SM takes in
-// 64 (measured: the one-CTA kernel moves 64 B/clk/SM and keeps the tensor pipe 73 % busy).  Two CTAs of
-// a cluster that share one MMA of M = 256 halve the weight traffic: each loads its own 128 activation rows and
-// HALF of the 256 weight rows, 32 KB per k-block, 64 bytes per cycle - the balance point - and its ring holds
-// six stages instead of four.
+// At that size the grouped GEMMs of Eq. 4 are a dense contraction.  A single CTA computing a 128 x 256 tile brings
+// 48 KB into shared memory per 64-deep k-block (128 rows of activations, 256 rows of weights) for 512
+// tensor-core cycles of work, 96 bytes per cycle if the pipe were to stay busy; the one-CTA kernel is measured
+// at 62-79 B/clk/SM with the tensor pipe 67-84 % busy.  Two CTAs of a cluster that share one MMA of M = 256
+// halve the weight traffic: each loads its own 128 activation rows and HALF of the 256 weight rows, 32 KB per
+// k-block, and its ring holds six stages instead of four.
 //
 //   cluster rank r (0 = leader, 1 = partner), tile = (256 grouped rows of one expert) x (256 output columns):
 //     A  rows  row0 + 128 r .. + 127 of the tile                      (own shared memory, own TMA loads)
