@@ -141,10 +141,10 @@ __device__ __forceinline__ void emit_block_ranks(const uint32_t* emask, long lon
 }
 
 // ---------------------------------------------------------------------------------------
-// bf16 router on the tcgen05 tensor cores.  A CTA of 8 warps owns 128 tokens:
+// bf16 router on the tcgen05 tensor cores.  A CTA of 16 warps owns 128 tokens:
 //   warp 0    : TMA producer  (X tile 128x64 and the router matrix tile e_pad x 64 per stage)
 //   warp 1    : UMMA issuer   (128 x e_pad x 16 tcgen05.mma; the logits tile lives in TMEM)
-//   warps 4-7 : once the accumulator is complete, copy it (+ bias) from TMEM to shared memory,
+//   warps 4-11: once the accumulator is complete, copy it (+ bias) from TMEM to shared memory,
 //               reusing the pipeline's stage buffers
 //   cluster   : with few token tiles the contraction is split over a cluster of 2 or 4 CTAs
 //               (more SMs pulling X); every CTA then owns 128/split rows of the tile and adds
@@ -157,7 +157,7 @@ __device__ __forceinline__ void emit_block_ranks(const uint32_t* emask, long lon
 // ---------------------------------------------------------------------------------------
 constexpr int RT_BM = 128;
 constexpr int RT_BK = 64;
-constexpr int RT_THREADS = 256;
+constexpr int RT_THREADS = 512;
 constexpr int RT_A_BYTES = RT_BM * RT_BK * 2;
 constexpr int RT_MAX_STAGES = 8;
 
@@ -187,9 +187,10 @@ __device__ __forceinline__ void route_tail_group8(const float* Lr, int ldl, long
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 3, l8 = lane & 7;
   const int E = a.E;
-  for (int it = 0; it < n_rows / 32; ++it) {
-    // rows of one warp are 8 apart: with an odd row pitch the four groups hit distinct banks
-    const int rl = it * 32 + g * 8 + warp;
+  for (int base = (warp >> 3) * 32; base < n_rows; base += 32 * (RT_THREADS / 256)) {
+    // eight warps share 32 rows; rows of one warp are 8 apart: with an odd row pitch the four groups hit
+    // distinct banks
+    const int rl = base + g * 8 + (warp & 7);
     const long long t = t_first + rl;
     const bool tok_ok = t < a.T;
     float z[NV];
@@ -346,7 +347,7 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       else { atomicCAS(status, 0, DEV_TIMEOUT); *abort_flag = 1; }
     }
   } else {
-    // warps 2-7 have nothing to do while the GEMM streams: clear this CTA's rows of the layer's
+    // warps 2-15 have nothing to do while the GEMM streams: clear this CTA's rows of the layer's
     // fp32 combine accumulator (and, once, the tile schedulers' counters)
     if (a.misc_zero && blockIdx.x == 0 && threadIdx.x == 64)
       for (int i = 1; i < 8; ++i) a.misc_zero[i] = 0;
@@ -362,14 +363,15 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       }
     }
   }
-  if (warp >= 4) {
+  if (warp >= 4 && warp < 12) {
     // accumulator complete => every stage buffer has been consumed: reuse them for the logits
+    // (two warps per TMEM lane quarter, alternate 32-column chunks)
     const int q = warp & 3;
     if (mbar_wait(tfull_bar, 0, abort_flag)) {
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
       float* dst = Ls + (q * 32 + lane) * ldl;
-      for (int c = 0; c < nch; ++c) {
+      for (int c = (warp - 4) >> 2; c < nch; c += 2) {
         uint32_t v[32];
         tmem_ld32(taddr + c * 32, v);
         tmem_ld_wait();
