@@ -435,6 +435,7 @@ __global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const Pr
   __shared__ float s_red[8][MAXW + 1];
   __shared__ float s_scale;
   __shared__ unsigned s_merged;                  // bit w: row w of this block is a merged window
+  __shared__ long long s_mem[CP_ROWS][MAXW];     // member tokens of the block's merged rows (validated)
   pdl_launch_dependents();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) s_merged = 0;
@@ -459,7 +460,18 @@ __global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const Pr
         // count (reported through the status word).  Never index x with it.
         for (int i = lane; i < vec; i += 32) dst[i] = make_uint4(0u, 0u, 0u, 0u);
         my_kind = -1;
-      } else if (my_kind != 2) {
+      } else if (my_kind == 2) {
+        // a merged window: look its member tokens up now, so that the dependent index loads are behind the
+        // block's copies when the whole CTA turns to this row
+        int v0 = a.vrank[t0];
+        if (v0 < 0 || v0 + a.W > sq.n_vis[b]) v0 = 0;   // inconsistent mask / count (status word set): stay inside the list
+        const long long s_lo = sq.seq_off[b], s_hi = sq.seq_off[b + 1];
+        if (lane < MAXW) {
+          long long tkn = lane < a.W ? a.vis_list[s_lo + v0 + lane] : s_lo;
+          if (tkn < s_lo || tkn >= s_hi) tkn = s_lo;
+          s_mem[warp][lane] = tkn;
+        }
+      } else {
         const uint4* src = reinterpret_cast<const uint4*>(X + t0 * a.H);
         for (int i0 = 0; i0 < vec; i0 += 256) {
           uint4 v[8];
@@ -479,19 +491,9 @@ __global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const Pr
     if (!((merged_mask >> w) & 1)) continue;
     const long long row = row_base + blk_row0 + w;
     T* O = static_cast<T*>(a.x_out) + row * a.H;
-    int b = 0;
-    while (b + 1 < sq.n_seq && row >= sq.out_off[b + 1]) ++b;
-    const long long t0 = a.keep_idx_ws[row];
-    int v0 = a.vrank[t0];
-    if (v0 < 0 || v0 + a.W > sq.n_vis[b]) v0 = 0;   // inconsistent mask / count (status word set): stay inside the list
-    const long long s_lo = sq.seq_off[b], s_hi = sq.seq_off[b + 1];
     long long mem[MAXW];
 #pragma unroll
-    for (int k = 0; k < MAXW; ++k) {
-      long long tkn = k < a.W ? a.vis_list[s_lo + v0 + k] : s_lo;
-      if (tkn < s_lo || tkn >= s_hi) tkn = s_lo;
-      mem[k] = tkn;
-    }
+    for (int k = 0; k < MAXW; ++k) mem[k] = s_mem[w][k];
     const float invW = 1.f / (float)a.W;
     float part[MAXW + 1];
 #pragma unroll
