@@ -121,12 +121,14 @@ typedef struct fmmoe_handle fmmoe_handle;   /* opaque: device, SM count, status 
  * built-in scratch array of fmmoe_prune_visual_static onto the device).  Not thread-safe
  * per handle.  Environment, read once here: FMMOE_DEBUG_SYNC=1 synchronises after every
  * kernel and reports the first failing one on stderr; FMMOE_GATHER_MIN_TOKENS=n moves the
- * token count from which GEMM-1 gathers the routed rows itself (default 12288);
+ * token count from which GEMM-1 gathers the routed rows itself instead of reading an
+ * expert-ordered copy of x (default 256);
  * FMMOE_SMALL_M_MAX_TOKENS=n moves the token count below which the expert GEMMs run with the
- * token rows as the MMA's N dimension (default 12288; 0 turns that form off);
+ * token rows as the MMA's N dimension (default 256: decode-sized batches; 0 turns that form
+ * off; layers with FP8 weights always run in it);
  * FMMOE_CTA_PAIR_MIN_TOKENS=n makes them run on CTA pairs with 256-row tiles from n tokens on
- * (off by default: measured no faster than the one-CTA form on a power-capped B200); FMMOE_PAIR_ROWS_MIN_TOKENS=n the token count from which the combine goes
- * through per-pair bf16 rows instead of atomic adds (default 8192). */
+ * (off by default: measured no faster than the one-CTA form on a power-capped B200); FMMOE_PAIR_ROWS_MIN_TOKENS=n keeps the atomic fp32 combine below n tokens
+ * (default 0: the combine always goes through per-pair bf16 rows summed in a fixed order). */
 fmmoe_status fmmoe_create(fmmoe_handle **handle, int device);
 fmmoe_status fmmoe_destroy(fmmoe_handle *handle);
 const char  *fmmoe_status_string(fmmoe_status s);
@@ -364,8 +366,8 @@ fmmoe_status fmmoe_stack_forward(fmmoe_handle *handle, const fmmoe_layer_desc *d
  * wait of a kernel on a barrier has a time budget; when it runs out the kernel records
  * FMMOE_ERR_TIMEOUT in the status word, releases its tensor memory and returns, so that a protocol
  * error ends as a status code with the context intact.  This call ARMS that path for the next
- * fmmoe_moe_forward on the handle (bf16 layer in its small-M form, i.e. fewer tokens than
- * FMMOE_SMALL_M_MAX_TOKENS, default 12288): that call's GEMM-1 runs as a single CTA whose
+ * fmmoe_moe_forward on the handle (a bf16 layer; the armed call runs in the small-M form
+ * whatever its token count): that call's GEMM-1 runs as a single CTA whose
  * producer stops before it issues any copy or arrival for k-block number `k_block` (0 = the first),
  * and all of that call's waits use `budget_ns` (1 us .. 1 s) instead of the default 2 s.  Nothing
  * faults and nothing spins without a limit: the issuing thread's wait for the missing stage

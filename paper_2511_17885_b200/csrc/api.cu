@@ -186,7 +186,7 @@ extern "C" __attribute__((visibility("default"))) fmmoe_status fmmoe_create(fmmo
   }
   h->wait_budget_ns = 2000000000ull;
   h->sm_attr_set = false; h->smq_attr_set = false; h->tc2_attr_set = false;
-  h->small_m_max_tokens = kGatherMinTokensDefault;
+  h->small_m_max_tokens = kSmallMMaxTokensDefault;
   if (const char* g = getenv("FMMOE_SMALL_M_MAX_TOKENS")) {
     char* end = nullptr;
     const long long v = strtoll(g, &end, 10);
@@ -305,7 +305,9 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   // bf16 at small batch: the permutation's scatter pass also writes the expert-grouped copy of x
   const bool pair = use_pair_rows(h, *d, T, flags);
   const bool cta_pairs = use_cta_pairs(h, *d, T);
-  const bool copy_rows = d->dtype == FMMOE_BF16 && (cta_pairs || use_small_m(h, *d, T) || !gather_rows_in_gemm(h, T));
+  // an armed wait self-test runs on the small-M form whatever the size thresholds say
+  const bool small_m = !cta_pairs && (use_small_m(h, *d, T) || (h->test_withhold_stage >= 0 && d->dtype == FMMOE_BF16));
+  const bool copy_rows = d->dtype == FMMOE_BF16 && (cta_pairs || small_m || !gather_rows_in_gemm(h, T));
   st = run_route(h, *d, *w, x, is_visual, T, flags, r, true, (det || pair) ? nullptr : reinterpret_cast<float*>(ws + pl.acc_off), s,
                  copy_rows ? ws + pl.xp_off : nullptr, cta_pairs ? 2 * TC_BLOCK_M : 0);
   if (st != FMMOE_OK) return st;
@@ -330,7 +332,7 @@ static fmmoe_status forward_impl(fmmoe_handle* h, const fmmoe_layer_desc* d, con
   fa.test_withhold_stage = -1; fa.grid_override = 0;
   if (cta_pairs) {
     st = launch_ffn_tc2(h, fa, s);
-  } else if (use_small_m(h, *d, T)) {
+  } else if (small_m) {
     const uint64_t budget = h->wait_budget_ns;
     if (h->test_withhold_stage >= 0) {     // armed self-test: this call only
       fa.test_withhold_stage = h->test_withhold_stage; fa.grid_override = 1;

@@ -18,6 +18,8 @@
 //           token to the fp32 accumulator with one 128-byte reduction (or stores them, fixed-order mode).
 // The transposed accumulator needs no shared-memory staging: for a fixed token the lanes of a warp already
 // hold consecutive output features.
+// When it runs: bf16 layers below 256 tokens (decode-sized batches; from there on the rows-as-M form with
+// the in-GEMM row gather measured faster) and every layer with FP8 weights.
 // FP8 weight stream (WQ = 1): the expert matrices arrive as FP8 E4M3 bytes with one power-of-two scale per
 // 128 x 128 block.  TMA brings the bytes (half the HBM traffic of bf16) into a ring of raw stages; eight more
 // warps expand every weight box to bf16 in the 128-byte-swizzled layout the MMA reads (exactly: an E4M3 value

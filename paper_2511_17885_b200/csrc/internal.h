@@ -222,11 +222,14 @@ struct FfnArgs {   // both paths
   int test_withhold_stage;   // small-M form, self-test only (-1: off)
   int grid_override;         // small-M form, self-test only: CTAs to launch (0: one per SM)
 };
-// Large batches: skip the expert-ordered copy of x and let GEMM-1's loader warps gather the rows.
-// Small batches are bound by the weight stream, where the copy + plain TMA boxes are faster.
-// The threshold is a property of the handle (default 12,288 tokens; FMMOE_GATHER_MIN_TOKENS, read once
+// From a few hundred tokens on GEMM-1's loader warps gather the routed rows of x themselves and no
+// expert-ordered copy of x is written (measured faster than the copy + plain TMA boxes from 256 tokens on,
+// by 3-12 % of a step between 2,432 and 14,336 tokens).  Below that the small-M form runs on the copy.
+// The threshold is a property of the handle (default 256 tokens; FMMOE_GATHER_MIN_TOKENS, read once
 // in fmmoe_create, overrides it so that either path can be exercised at any size).
-constexpr int64_t kGatherMinTokensDefault = 12288;
+constexpr int64_t kGatherMinTokensDefault = 256;
+// Decode-sized batches: token rows as the MMA's N dimension (FMMOE_SMALL_M_MAX_TOKENS).
+constexpr int64_t kSmallMMaxTokensDefault = 256;
 static inline bool gather_rows_in_gemm(const fmmoe_handle* h, int64_t T) { return T >= h->gather_min_tokens; }
 fmmoe_status launch_ffn_tc(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05, token rows as M
 fmmoe_status launch_ffn_sm(fmmoe_handle* h, const FfnArgs& a, cudaStream_t s);    // bf16, tcgen05, token rows as N (reads xp)
@@ -236,9 +239,12 @@ static inline bool use_cta_pairs(const fmmoe_handle* h, const fmmoe_layer_desc& 
   return d.dtype == FMMOE_BF16 && d.weight_format == FMMOE_WEIGHTS_AS_DTYPE && T >= h->cta_pair_min_tokens;
 }
 // Which form runs: below small_m_max_tokens (and below the in-GEMM gather threshold) the small-M form.
-// The fp32 accumulator of the atomic combine is T*H*4 bytes; once it no longer fits the L2 cache next to the
-// activations its read-modify-writes page through HBM, and writing every pair's row once in bf16 is cheaper.
-constexpr int64_t kPairMinTokensDefault = 8192;
+// Combine: every pair's gate-scaled row is written once in bf16 and summed per token in a fixed order
+// (no atomics, reproducible bit for bit).  Measured against the atomic fp32 accumulator it is equal below
+// 512 tokens and 2-4 % of a step faster from there on (the accumulator, T*H*4 bytes, stops fitting the L2
+// cache next to the activations around 8,192 tokens and then pages through HBM), so it is the default at
+// every size; FMMOE_PAIR_ROWS_MIN_TOKENS=n keeps the atomic combine below n tokens.
+constexpr int64_t kPairMinTokensDefault = 0;
 static inline bool use_pair_rows(const fmmoe_handle* h, const fmmoe_layer_desc& d, int64_t T, uint32_t flags) {
   return d.dtype == FMMOE_BF16 && !(flags & FMMOE_FLAG_DETERMINISTIC) && T >= h->pair_min_tokens;
 }

@@ -318,16 +318,19 @@ def _rows_per_expert_case(counts, n_text_extra, H=128, I_=192, seed=41):
     return I.round_to_storage(x, "bf16"), mask, w, E
 
 
+_SMALL_M = {"FMMOE_SMALL_M_MAX_TOKENS": "1000000", "FMMOE_GATHER_MIN_TOKENS": "1000000"}
+_ATOMIC = {"FMMOE_PAIR_ROWS_MIN_TOKENS": "1000000"}       # the atomic fp32 combine (optional; the default is pair rows)
 ROW_PATHS = {
     # name: environment read by fmmoe_create -> which kernels the expert GEMMs run as at this size
-    "small_m": {},                                                        # default below 12,288 tokens: rows as the MMA's N
-    "rows_as_m_copy": {"FMMOE_SMALL_M_MAX_TOKENS": "0"},                  # rows as M, expert-ordered copy of x
-    "rows_as_m_gather": {"FMMOE_SMALL_M_MAX_TOKENS": "0", "FMMOE_GATHER_MIN_TOKENS": "0"},   # rows as M, in-GEMM gather
-    # 256-row tiles on CTA pairs (default from 12,288 tokens on), with the atomic and the per-pair combine
-    "cta_pairs": {"FMMOE_CTA_PAIR_MIN_TOKENS": "0"},
+    "default": {},                                        # rows as N below 256 tokens, rows as M + gather above; pair rows
+    "small_m": dict(_SMALL_M, **_ATOMIC),                 # rows as the MMA's N at every size
+    "rows_as_m_copy": dict({"FMMOE_SMALL_M_MAX_TOKENS": "0", "FMMOE_GATHER_MIN_TOKENS": "1000000"}, **_ATOMIC),   # rows as M, expert-ordered copy of x
+    "rows_as_m_gather": dict({"FMMOE_SMALL_M_MAX_TOKENS": "0", "FMMOE_GATHER_MIN_TOKENS": "0"}, **_ATOMIC),   # rows as M, in-GEMM gather
+    # 256-row tiles on CTA pairs (optional form), with the atomic and the per-pair combine
+    "cta_pairs": dict({"FMMOE_CTA_PAIR_MIN_TOKENS": "0"}, **_ATOMIC),
     "cta_pairs_pair_rows": {"FMMOE_CTA_PAIR_MIN_TOKENS": "0", "FMMOE_PAIR_ROWS_MIN_TOKENS": "0"},
-    # the combine through per-pair bf16 rows (default from 8,192 tokens on), under both forms
-    "small_m_pair_rows": {"FMMOE_PAIR_ROWS_MIN_TOKENS": "0"},
+    # the combine through per-pair bf16 rows (the default), under both forms
+    "small_m_pair_rows": dict(_SMALL_M, FMMOE_PAIR_ROWS_MIN_TOKENS="0"),
     "rows_as_m_gather_pair_rows": {"FMMOE_SMALL_M_MAX_TOKENS": "0", "FMMOE_GATHER_MIN_TOKENS": "0",
                                    "FMMOE_PAIR_ROWS_MIN_TOKENS": "0"},
 }
@@ -346,8 +349,8 @@ def handle_with_env(monkeypatch, env):
 def test_rows_per_expert_boundaries_on_every_gemm_form(path, monkeypatch):
     """Experts holding 0, 1, 15, 16, 17, 33, 64, 65, 96, 97, 128 and 129 rows (and two with several hundred), EVERY
     output row against the oracle, on each form of the expert GEMMs: token rows as the MMA's N dimension (the
-    default below 12,288 tokens), rows as M reading the expert-ordered copy written by the scatter pass, and rows
-    as M with the in-GEMM gather by token (otherwise only reached from 12,288 tokens on)."""
+    default below 256 tokens), rows as M reading the expert-ordered copy written by the scatter pass, and rows
+    as M with the in-GEMM gather by token (the default from 256 tokens on)."""
     counts = [0, 1, 15, 16, 17, 33, 64, 65, 96, 97, 128, 129]
     x, mask, w, E = _rows_per_expert_case(counts, n_text_extra=300)
     h = handle_with_env(monkeypatch, ROW_PATHS[path])
