@@ -380,6 +380,14 @@ def test_decode_sized_batches_with_shared_experts(T):
     check_layer("bf16", T, 128, 8, 64, 2, 1, 0, 0, flags=B.FLAG_REDUCE_ON | B.FLAG_DETERMINISTIC, seed=60 + T)
 
 
+@pytest.mark.parametrize("T", [255, 256, 257])
+def test_default_form_on_both_sides_of_its_size_threshold(T):
+    """With the handle's defaults a bf16 layer runs with the token rows as the MMA's N dimension below 256 tokens
+    and as its M dimension, gathering its rows, from 256 on: the last size of the one and the first two of the
+    other, shared experts and residual included, against the oracle."""
+    check_layer("bf16", T, 256, 8, 192, 4, 2, Ns=1, Is=128, flags=B.FLAG_REDUCE_ON | B.FLAG_RESIDUAL, seed=300 + T)
+
+
 def test_small_m_form_equals_rows_as_m_form_bit_for_bit_in_fixed_order_mode(monkeypatch):
     """The three forms of the expert GEMMs (rows as N, rows as M, rows as M on CTA pairs) accumulate every output element over the same k order in fp32, so with the
     fixed-order combine their layer outputs are identical bit for bit."""
