@@ -6,7 +6,7 @@
 //                        merge set = m highest C (Eq. 15), drop set = d smallest A_bar among
 //                        the rest (both by an in-CTA bitonic sort of (score, window) keys),
 //                        then the stable compaction map (scan of keep flags)
-//   compact_kernel     : copies kept rows (a warp per row, eight rows per CTA); a merged window becomes
+//   compact_kernel     : copies kept rows (a warp per row, four rows per CTA); a merged window becomes
 //                        mean(rows) rescaled to the largest member norm (Eq. 16-18) at its first token's
 //                        position, formed by the whole CTA
 // Ranks come from sorting unique (value, window index) keys, so the keep-set does not depend
@@ -426,8 +426,11 @@ template <> struct Row8<float> {
 
 // Rows per CTA of compact_kernel: one warp copies one kept row (the common case: with the paper's merge
 // rates about 3 % of the output rows are merged windows), then the whole CTA forms the block's merged rows
-// one after another, so that a merge still has 256 threads behind it.
-constexpr int CP_ROWS = 8;
+// one after another, so that a merge still has 256 threads behind it.  Four rows per CTA (warps 0-3 copy):
+// a CTA then rarely holds more than one merged row, whose dependent steps set the kernel's duration
+// (measured 23.9 / 10.2 us with four, 26.9 / 15.2 us with eight and 25.2 / 10.1 us with two rows per CTA on
+// 14,336 / 2,432 tokens).
+constexpr int CP_ROWS = 4;
 
 template <typename T>
 __global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const PruneSeqs sq, long long row_base, long long n_rows) {
@@ -448,7 +451,7 @@ __global__ void __launch_bounds__(256) compact_kernel(const PruneDev a, const Pr
   int my_kind = -1;
   {
     const long long rel = blk_row0 + warp;
-    if (rel < n_rows) {
+    if (warp < CP_ROWS && rel < n_rows) {
       const long long row = row_base + rel;
       int b = 0;
       while (b + 1 < sq.n_seq && row >= sq.out_off[b + 1]) ++b;
