@@ -55,6 +55,7 @@ NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # the nominal peaks the m
 NCU_TRAFFIC_BYTES = {
     "C2x4": {"gemm1": 1101.6e6, "gemm2": 723.2e6, "route": 60.4e6, "finalize": 296.1e6},   # ffn_tc_kernel<0/1>, route_tc, finalize_pair
     "C1": {"gemm1": 824.8e6, "gemm2": 469.9e6, "finalize": 51.6e6},                         # ffn_tc_kernel<0/1>, finalize_pair
+    "C2": {"gemm1": 870.4e6, "gemm2": 477.2e6},                                             # ffn_tc_kernel<0/1>
     "C1_fp8": {"gemm1": 501.7e6, "gemm2": 293.8e6},                                         # ffn_sm_kernel<0/1, 1>
 }
 
